@@ -1,0 +1,160 @@
+/*
+ * libasap -- the ASAP visual-token prune step (arXiv 2603.14549, Sec. 4) for one B200 (sm_100a).
+ *
+ * The step runs between two decoder layers during prefill.  For every sequence of a packed
+ * batch, laid out as [ prefix (system prompt) | visual span I | suffix (text) ], it
+ *   1a. sums the pre-softmax alignment W = Q K^T / sqrt(d) over the visual queries to get the
+ *       attention mass s_j of every visual key                                   (Sec. 4.1, Eq. 1)
+ *   1b. min-max normalises s to the salience s_hat and forms the mask vector
+ *       m_j = ln max(lambda_max * s_hat_j, eps)                                  (Eq. 2, Eq. 3)
+ *   1c. evaluates A = Softmax(W + M_bidir) on the ranking query rows            (Eq. 3, Eq. 4)
+ *   2.  averages A over heads and ranking rows into one score r_j per visual key
+ *   3.  keeps the keep_k visual tokens of largest r_j (ties: lower index)        (Fig. 3)
+ *   4a. sends every dropped token to the kept token of highest cosine similarity (Sec. 4.2)
+ *   4b. replaces every kept token by the salience-weighted mean of itself and the tokens
+ *       sent to it                                                               (Eq. 5)
+ *   5.  writes the shortened sequence [ prefix | kept visual, ascending | suffix ] with its
+ *       gathered position ids                                                    (Fig. 3)
+ *
+ * Conventions for every entry point
+ *   - Pointers inside asap_inputs / asap_outputs are DEVICE pointers owned by the caller; the
+ *     structs themselves and the asap_params struct live in HOST memory.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work: they never
+ *     synchronise the stream, never read device memory on the host and never allocate (all
+ *     scratch memory is taken by asap_init).
+ *   - Every function returns an asap_status and never throws or aborts.  On ASAP_ERR_* no
+ *     kernel has been launched by that call and the outputs are untouched.  The text of the
+ *     last error is available from asap_last_error.
+ *   - Host-side checks cover what the host can see (null pointers, 16-byte alignment of
+ *     q / k / hidden / out_hidden, head_dim == 128, D == H * head_dim, 0 < keep_k <= min_vis,
+ *     0 < lambda_max <= 1, eps > 0, sizes within the asap_init capacities).  The per-sample
+ *     arrays live on the device; the first kernel of each call checks them (spans inside the
+ *     sequence, vis_len within [min_vis, max_vis], ascending cu_seqlens, ...) and records a
+ *     violation in a device status word that asap_check reads.  A kernel never traps or
+ *     spins without bound; every wait in the tensor-core kernels has an iteration limit after
+ *     which the status word is set and the block leaves.
+ *   - bf16 tensors are row-major with the stated shapes and no padding.
+ *   - A context serves one stream at a time: two calls on the same context that overlap on
+ *     the GPU race on its scratch memory.
+ */
+#ifndef ASAP_H
+#define ASAP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct asap_ctx asap_ctx; /* opaque: scratch memory, device status word, error text */
+
+typedef enum {
+  ASAP_OK = 0,
+  ASAP_ERR_INVALID = -1,     /* bad argument visible to the host */
+  ASAP_ERR_ALIGN = -2,       /* a tensor pointer is not 16-byte aligned */
+  ASAP_ERR_WORKSPACE = -3,   /* the problem exceeds the capacities given to asap_init */
+  ASAP_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed */
+  ASAP_ERR_UNSUPPORTED = -5, /* head_dim != 128, D not a multiple of 8, ... */
+  ASAP_ERR_DEVICE = -6       /* asap_check: a kernel flagged bad device-side data or a timed-out wait */
+} asap_status;
+
+/* Problem description.  Sequence b owns packed rows cu_seqlens[b] .. cu_seqlens[b+1]-1.  Span
+ * starts are relative to the start of their sequence. */
+typedef struct {
+  int32_t B;            /* sequences in the batch */
+  int32_t H;            /* attention heads */
+  int32_t head_dim;     /* must be 128 */
+  int32_t D;            /* hidden size, == H * head_dim */
+  int32_t total_tokens; /* rows of q / k / hidden / pos_ids == cu_seqlens[B] */
+  int32_t min_vis;      /* host-known bounds: min_vis <= vis_len[b] <= max_vis */
+  int32_t max_vis;
+  int32_t max_seq;      /* bound on the length of any sequence */
+  int32_t max_rank;     /* bound on rank_len[b] (on text_len[b] when rank_start is NULL) */
+  const int32_t *cu_seqlens; /* [B+1] */
+  const int32_t *vis_start;  /* [B] image span I */
+  const int32_t *vis_len;    /* [B] */
+  const int32_t *text_start; /* [B] text span, text_start >= vis_start + vis_len */
+  const int32_t *text_len;   /* [B] */
+  const int32_t *rank_start; /* [B] query rows whose Eq. 4 probabilities rank the visual keys; */
+  const int32_t *rank_len;   /* [B] both NULL => the text span.  rank_len[b] >= 1.             */
+  const void *q;             /* bf16 [total_tokens, H, head_dim], rotary embedding applied */
+  const void *k;             /* bf16 [total_tokens, H, head_dim], rotary embedding applied */
+  const void *hidden;        /* bf16 [total_tokens, D], hidden states after the pruning layer */
+  const int32_t *pos_ids;    /* [total_tokens] */
+} asap_inputs;
+
+typedef struct {
+  int32_t keep_k;       /* visual tokens kept per sequence, 0 < keep_k <= min_vis */
+  float lambda_max;     /* Eq. 3 leak budget, in (0, 1] */
+  float eps;            /* Eq. 2 / Eq. 3 / Eq. 5 epsilon, the paper uses 1e-6 */
+  float sim_threshold;  /* Sec. 4.2 threshold t: merge only if cosine similarity > t; -INFINITY = always */
+  int32_t mask_enable;  /* 0: Eq. 3 is replaced by the causal mask of Sec. 3.2 */
+  int32_t merge_enable; /* 0: kept tokens are copied unmerged, assign = -1 */
+} asap_params;
+
+/* Results.  Per-sequence arrays are padded to the stated pitch; entries past vis_len[b]
+ * (or past vis_len[b] - keep_k) are 0 for floats and -1 for indices.  Visual indices are
+ * relative to the start of the image span. */
+typedef struct {
+  float *mass;       /* [B, max_vis] s_j       (Eq. 1, mean over heads)            */
+  float *salience;   /* [B, max_vis] s_hat_j   (Eq. 2)                             */
+  float *mask_log;   /* [B, max_vis] m_j       (Eq. 3)                             */
+  float *rank_score; /* [B, max_vis] r_j       (mean over heads, ranking rows of Eq. 4) */
+  int32_t *keep_idx; /* [B, keep_k]            kept visual indices, ascending      */
+  int32_t *drop_idx; /* [B, max_vis - keep_k]  dropped visual indices, ascending   */
+  int32_t *assign;   /* [B, max_vis - keep_k]  kept SLOT (0..keep_k-1) a dropped token merges into, or -1 */
+  float *best_sim;   /* [B, max_vis - keep_k]  its cosine similarity to that slot; may be NULL */
+  void *out_hidden;  /* bf16 [out_rows, D]     shortened sequences, packed         */
+  int32_t *out_pos;  /* [out_rows]             position ids gathered from pos_ids  */
+  int32_t *src_row;  /* [out_rows]             packed input row each output row came from */
+  int32_t *out_cu_seqlens; /* [B+1]            row offsets of the shortened sequences */
+  int32_t out_rows_capacity; /* rows available in out_hidden / out_pos / src_row; the step needs
+                                total_tokens - sum_b vis_len[b] + B * keep_k, which is at most
+                                total_tokens - B * (min_vis - keep_k) */
+} asap_outputs;
+
+/* Creates a context on `device` and takes all scratch memory the step will ever need for
+ * problems with total_tokens <= max_total_tokens, B <= max_B, H <= max_H, D <= max_D and
+ * B * keep_k <= max_keep_rows (0 = max_total_tokens).  The only call that allocates. */
+asap_status asap_init(asap_ctx **ctx, int device, size_t max_total_tokens, int max_B, int max_H,
+                      int max_D, size_t max_keep_rows);
+
+/* Steps 1a-2 (Sec. 4.1, Eq. 1-4).  Writes out->mass, salience, mask_log, rank_score. */
+asap_status asap_score(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                       const asap_outputs *out, void *stream);
+
+/* Step 3 (Fig. 3: top-k retained).  Reads `rank_score` [B, max_vis]; writes out->keep_idx,
+ * out->drop_idx. */
+asap_status asap_select(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                        const float *rank_score, const asap_outputs *out, void *stream);
+
+/* Steps 4a-5 (Sec. 4.2, Eq. 5; hand-off of Fig. 3).  Reads `salience`, `keep_idx`, `drop_idx`
+ * (layouts as in asap_outputs); writes out->assign, best_sim (if non-NULL), out_hidden,
+ * out_pos, src_row, out_cu_seqlens. */
+asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                       const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
+                       const asap_outputs *out, void *stream);
+
+/* Steps 1a-5 back to back on `stream`; fills every field of `out`. */
+asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                            const asap_outputs *out, void *stream);
+
+/* Reads the device status word (one 4-byte copy after synchronising `stream`).  ASAP_OK, or
+ * ASAP_ERR_DEVICE with the reason in asap_last_error; the word is cleared. */
+asap_status asap_check(asap_ctx *ctx, void *stream);
+
+/* Text of the last error recorded on this context (empty string if none).  Valid until the
+ * next call on the context.  asap_last_error(NULL) describes a failed asap_init. */
+const char *asap_last_error(const asap_ctx *ctx);
+
+/* Number of kernel launches the library has enqueued through this context so far. */
+uint64_t asap_launch_count(const asap_ctx *ctx);
+
+/* Releases the context and its scratch memory.  NULL is allowed. */
+void asap_free(asap_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASAP_H */

@@ -112,21 +112,25 @@ def mask_matrix(n: int, rows: np.ndarray, v0: int, nv: int, m: Optional[np.ndarr
     Eq. 3: 0 on and below the diagonal.  Above the diagonal the causal -inf stays,
     except inside the image span (query AND key visual) where it is overwritten by
     m_j.  With the mask disabled this is the causal mask of Sec. 3.2."""
-    M = np.full((len(rows), n), -np.inf, dtype=np.float64)
-    for a, i in enumerate(rows):
-        for j in range(n):
-            if j <= i:
-                M[a, j] = 0.0
-            elif mask_enable and v0 <= i < v0 + nv and v0 <= j < v0 + nv:
-                M[a, j] = m[j - v0]
+    i = np.asarray(rows)[:, None]                 # query position
+    j = np.arange(n)[None, :]                     # key position
+    M = np.where(j <= i, 0.0, -np.inf)
+    if mask_enable:
+        m_of_key = np.full(n, -np.inf)
+        m_of_key[v0:v0 + nv] = m
+        in_span = (i >= v0) & (i < v0 + nv) & (j >= v0) & (j < v0 + nv)
+        M = np.where(in_span & (i < j), m_of_key[None, :], M)
     return M
 
 
 def attention_probs(q: np.ndarray, k: np.ndarray, h: int, rows: np.ndarray, v0: int, nv: int,
-                    m: Optional[np.ndarray], mask_enable: bool) -> np.ndarray:
-    """Eq. 4: A = Softmax(W + M_bidir), rows `rows` of one head, over all keys."""
+                    m: Optional[np.ndarray], mask_enable: bool, M: Optional[np.ndarray] = None) -> np.ndarray:
+    """Eq. 4: A = Softmax(W + M_bidir), rows `rows` of one head, over all keys.
+    (M may be passed in when several heads share it; it is the same for every head.)"""
     W = alignment(q[rows], k, h)
-    Z = W + mask_matrix(k.shape[0], rows, v0, nv, m, mask_enable)
+    if M is None:
+        M = mask_matrix(k.shape[0], rows, v0, nv, m, mask_enable)
+    Z = W + M
     Z = Z - Z.max(axis=1, keepdims=True)
     E = np.exp(Z)
     return E / E.sum(axis=1, keepdims=True)
@@ -139,8 +143,9 @@ def rank_scores(q: np.ndarray, k: np.ndarray, v0: int, nv: int, r0: int, nr: int
     H = q.shape[1]
     rows = np.arange(r0, r0 + nr)
     r = np.zeros(nv, dtype=np.float64)
+    M = mask_matrix(k.shape[0], rows, v0, nv, m, mask_enable)
     for h in range(H):
-        A = attention_probs(q, k, h, rows, v0, nv, m, mask_enable)
+        A = attention_probs(q, k, h, rows, v0, nv, m, mask_enable, M)
         r += A[:, v0:v0 + nv].sum(axis=0)
     return r / (H * nr)
 

@@ -1,0 +1,417 @@
+// Host side of libasap: context and scratch memory, argument validation, tensor-map
+// creation and the launch sequence of each C-ABI entry point declared in include/asap.h.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/asap.h"
+#include "kernels_stream.cuh"
+#include "kernels_tc.cuh"
+
+using namespace asap;
+
+namespace {
+
+char g_init_error[256] = "";
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+struct asap_ctx {
+  int device = 0;
+  size_t cap_tokens = 0, cap_keep_rows = 0;
+  int cap_B = 0, cap_H = 0, cap_D = 0;
+  size_t cap_chunks = 0;      // rows of the query-sum partial buffer
+  uint8_t *arena = nullptr;   // one allocation, carved below
+  SampleDesc *desc = nullptr;
+  float *qsum_partial = nullptr, *qbar = nullptr, *score_partial = nullptr, *inv_norm = nullptr,
+        *kept_inv = nullptr;
+  unsigned int *cnt_qsum = nullptr, *cnt_mass = nullptr, *cnt_score = nullptr;
+  int32_t *role = nullptr, *seg = nullptr, *members = nullptr;
+  __nv_bfloat16 *kept_rows = nullptr;
+  uint32_t *status = nullptr;
+  EncodeTiledFn encode = nullptr;
+  uint64_t launches = 0;
+  char err[512] = "";
+};
+
+namespace {
+
+asap_status fail(asap_ctx *ctx, asap_status st, const char *fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(ctx ? ctx->err : g_init_error, ctx ? sizeof(ctx->err) : sizeof(g_init_error), fmt, ap);
+  va_end(ap);
+  return st;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// 2-D bf16 tensor [rows, cols] row-major, box = 64 columns x box_rows rows, 128-byte swizzle.
+bool make_map(asap_ctx *ctx, CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols,
+              uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims,
+                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// ---- validation of everything the host can see -------------------------------------------
+enum Need : unsigned {
+  NEED_QK = 1u, NEED_HIDDEN = 2u, NEED_SCORE_OUT = 4u, NEED_SELECT_OUT = 8u, NEED_MERGE_OUT = 16u
+};
+
+asap_status validate(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                     const asap_outputs *out, unsigned need) {
+  if (!ctx) return fail(nullptr, ASAP_ERR_INVALID, "null context");
+  ctx->err[0] = 0;
+  if (!in || !p || !out) return fail(ctx, ASAP_ERR_INVALID, "null inputs / params / outputs struct");
+  if (in->B <= 0 || in->H <= 0 || in->total_tokens <= 0)
+    return fail(ctx, ASAP_ERR_INVALID, "B, H and total_tokens must be positive");
+  if (in->head_dim != 128) return fail(ctx, ASAP_ERR_UNSUPPORTED, "head_dim must be 128, got %d", in->head_dim);
+  if (in->D != in->H * in->head_dim) return fail(ctx, ASAP_ERR_INVALID, "D != H * head_dim");
+  if (in->D > 8192) return fail(ctx, ASAP_ERR_UNSUPPORTED, "D > 8192 is not supported");
+  if (in->min_vis <= 0 || in->max_vis < in->min_vis || in->max_seq < in->max_vis)
+    return fail(ctx, ASAP_ERR_INVALID, "need 0 < min_vis <= max_vis <= max_seq");
+  if (in->max_vis > 57344) return fail(ctx, ASAP_ERR_UNSUPPORTED, "max_vis > 57344 is not supported");
+  if (in->max_rank <= 0 || in->max_rank > in->max_seq)
+    return fail(ctx, ASAP_ERR_INVALID, "need 0 < max_rank <= max_seq");
+  if (p->keep_k <= 0 || p->keep_k > in->min_vis)
+    return fail(ctx, ASAP_ERR_INVALID, "need 0 < keep_k <= min_vis (keep_k=%d, min_vis=%d)", p->keep_k, in->min_vis);
+  if (!(p->lambda_max > 0.f && p->lambda_max <= 1.f))
+    return fail(ctx, ASAP_ERR_INVALID, "lambda_max must be in (0, 1]");
+  if (!(p->eps > 0.f)) return fail(ctx, ASAP_ERR_INVALID, "eps must be positive");
+  if (p->sim_threshold != p->sim_threshold) return fail(ctx, ASAP_ERR_INVALID, "sim_threshold is NaN");
+  if (!in->cu_seqlens || !in->vis_start || !in->vis_len || !in->text_start || !in->text_len)
+    return fail(ctx, ASAP_ERR_INVALID, "null per-sample array");
+  if ((in->rank_start == nullptr) != (in->rank_len == nullptr))
+    return fail(ctx, ASAP_ERR_INVALID, "rank_start and rank_len must both be given or both be NULL");
+  if ((need & NEED_QK) && (!in->q || !in->k)) return fail(ctx, ASAP_ERR_INVALID, "null q / k");
+  if ((need & NEED_QK) && (!aligned16(in->q) || !aligned16(in->k)))
+    return fail(ctx, ASAP_ERR_ALIGN, "q / k must be 16-byte aligned");
+  if (need & NEED_HIDDEN) {
+    if (!in->hidden || !in->pos_ids) return fail(ctx, ASAP_ERR_INVALID, "null hidden / pos_ids");
+    if (!aligned16(in->hidden)) return fail(ctx, ASAP_ERR_ALIGN, "hidden must be 16-byte aligned");
+  }
+  if ((need & NEED_SCORE_OUT) && (!out->mass || !out->salience || !out->mask_log || !out->rank_score))
+    return fail(ctx, ASAP_ERR_INVALID, "null score output (mass / salience / mask_log / rank_score)");
+  if ((need & NEED_SELECT_OUT) && (!out->keep_idx || !out->drop_idx))
+    return fail(ctx, ASAP_ERR_INVALID, "null keep_idx / drop_idx");
+  if (need & NEED_MERGE_OUT) {
+    if (!out->assign || !out->out_hidden || !out->out_pos || !out->src_row || !out->out_cu_seqlens)
+      return fail(ctx, ASAP_ERR_INVALID, "null merge output");
+    if (!aligned16(out->out_hidden)) return fail(ctx, ASAP_ERR_ALIGN, "out_hidden must be 16-byte aligned");
+    const long long bound = (long long)in->total_tokens - (long long)in->B * (in->min_vis - p->keep_k);
+    if (out->out_rows_capacity <= 0 || bound <= 0)
+      return fail(ctx, ASAP_ERR_INVALID, "out_rows_capacity must be positive");
+  }
+  // capacities
+  if ((size_t)in->total_tokens > ctx->cap_tokens || in->B > ctx->cap_B || in->H > ctx->cap_H ||
+      in->D > ctx->cap_D)
+    return fail(ctx, ASAP_ERR_WORKSPACE, "problem exceeds the capacities given to asap_init");
+  if ((size_t)in->B * (size_t)in->max_vis > ctx->cap_tokens)
+    return fail(ctx, ASAP_ERR_WORKSPACE, "B * max_vis exceeds max_total_tokens");
+  if ((size_t)in->B * (size_t)p->keep_k > ctx->cap_keep_rows)
+    return fail(ctx, ASAP_ERR_WORKSPACE, "B * keep_k exceeds max_keep_rows");
+  const size_t chunks = (size_t)in->B * ((in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS);
+  if (chunks > ctx->cap_chunks) return fail(ctx, ASAP_ERR_WORKSPACE, "query-sum scratch too small for B * max_vis");
+  return ASAP_OK;
+}
+
+asap_status after_launch(asap_ctx *ctx, const char *what) {
+  ctx->launches += 1;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "%s launch failed: %s", what, cudaGetErrorString(e));
+  return ASAP_OK;
+}
+
+#define ASAP_TRY(expr)                   \
+  do {                                   \
+    asap_status st__ = (expr);           \
+    if (st__ != ASAP_OK) return st__;    \
+  } while (0)
+
+// ---- stage launchers -------------------------------------------------------------------------
+asap_status launch_prepare(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                           int32_t *out_cu, int out_capacity, cudaStream_t st) {
+  PrepareArgs a;
+  a.B = in->B; a.total_tokens = in->total_tokens; a.min_vis = in->min_vis; a.max_vis = in->max_vis;
+  a.max_seq = in->max_seq; a.max_rank = in->max_rank; a.keep_k = p->keep_k; a.out_capacity = out_capacity;
+  a.cu_seqlens = in->cu_seqlens; a.vis_start = in->vis_start; a.vis_len = in->vis_len;
+  a.text_start = in->text_start; a.text_len = in->text_len; a.rank_start = in->rank_start;
+  a.rank_len = in->rank_len; a.desc = ctx->desc; a.out_cu_seqlens = out_cu; a.status = ctx->status;
+  prepare_kernel<<<1, 256, 0, st>>>(a);
+  return after_launch(ctx, "prepare");
+}
+
+asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                         const asap_outputs *out, cudaStream_t st) {
+  const int D = in->D, B = in->B;
+  const int max_chunks = (in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS;
+  const int col_blocks = (D + QSUM_COLS - 1) / QSUM_COLS;
+  qsum_kernel<<<dim3(max_chunks, col_blocks, B), QSUM_THREADS, 0, st>>>(
+      static_cast<const __nv_bfloat16 *>(in->q), ctx->desc, D, max_chunks, ctx->qsum_partial, ctx->qbar,
+      ctx->cnt_qsum);
+  ASAP_TRY(after_launch(ctx, "qsum"));
+
+  const float scale = 1.0f / ((float)in->H * sqrtf((float)in->head_dim));
+  const int row_blocks = (in->max_vis + MASS_ROWS - 1) / MASS_ROWS;
+  mass_salience_kernel<<<dim3(row_blocks, B), MASS_THREADS, (size_t)D * sizeof(float), st>>>(
+      static_cast<const __nv_bfloat16 *>(in->k), ctx->desc, D, in->max_vis, scale, p->lambda_max, p->eps,
+      ctx->qbar, out->mass, out->salience, out->mask_log, ctx->cnt_mass);
+  ASAP_TRY(after_launch(ctx, "mass_salience"));
+
+  CUtensorMap map_q, map_k;
+  if (!make_map(ctx, &map_q, in->q, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
+      !make_map(ctx, &map_k, in->k, (uint64_t)in->total_tokens, (uint64_t)D, 128))
+    return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for q / k");
+  ScoreArgs sa;
+  sa.desc = ctx->desc; sa.H = in->H; sa.max_vis = in->max_vis; sa.mask_enable = p->mask_enable ? 1 : 0;
+  sa.scale_log2 = 1.4426950408889634f / sqrtf((float)in->head_dim);
+  sa.mask_log = out->mask_log; sa.partial = ctx->score_partial; sa.rank_score = out->rank_score;
+  sa.counters = ctx->cnt_score; sa.status = ctx->status;
+  score_kernel<<<dim3(in->H, B), SC_THREADS, SC_SMEM_BYTES, st>>>(map_q, map_k, sa);
+  return after_launch(ctx, "score");
+}
+
+asap_status launch_select(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                          const float *rank_score, const asap_outputs *out, cudaStream_t st) {
+  select_kernel<<<in->B, SELECT_THREADS, (size_t)in->max_vis * sizeof(uint32_t), st>>>(
+      rank_score, ctx->desc, in->max_vis, p->keep_k, out->keep_idx, out->drop_idx, ctx->role);
+  return after_launch(ctx, "select");
+}
+
+__global__ void fill_assign_kernel(int32_t *assign, float *best_sim, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    assign[i] = -1;
+    if (best_sim) best_sim[i] = 0.f;
+  }
+}
+
+asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                         const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
+                         const asap_outputs *out, cudaStream_t st) {
+  const int B = in->B, D = in->D, k = p->keep_k;
+  const size_t nd_total = (size_t)B * (size_t)(in->max_vis - k);
+  if (nd_total > 0) {
+    const int blocks = (int)((nd_total + 255) / 256 < 1024 ? (nd_total + 255) / 256 : 1024);
+    fill_assign_kernel<<<blocks, 256, 0, st>>>(out->assign, out->best_sim, nd_total);
+    ASAP_TRY(after_launch(ctx, "fill_assign"));
+  }
+  const bool do_merge = p->merge_enable && in->max_vis > k;
+  if (do_merge) {
+    norm_gather_kernel<<<dim3((in->max_vis + 7) / 8, B), NORM_THREADS, 0, st>>>(
+        static_cast<const __nv_bfloat16 *>(in->hidden), ctx->desc, D, in->max_vis, k, ctx->role,
+        ctx->inv_norm, ctx->kept_rows, ctx->kept_inv);
+    ASAP_TRY(after_launch(ctx, "norm_gather"));
+
+    const int n_nt = (k + 255) / 256;
+    const int n_tile = (((k + n_nt - 1) / n_nt) + 15) & ~15;
+    const int stage_bytes = SIM_A_BYTES + n_tile * 128;
+    int stages = (200 * 1024) / stage_bytes;
+    if (stages > SIM_MAX_STAGES) stages = SIM_MAX_STAGES;
+    const size_t smem = (size_t)stages * stage_bytes + SIM_BOOK_BYTES + 1024;
+    CUtensorMap map_h, map_kept;
+    if (!make_map(ctx, &map_h, in->hidden, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
+        !make_map(ctx, &map_kept, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, (uint32_t)n_tile))
+      return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for hidden / kept rows");
+    SimArgs sa;
+    sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = n_tile;
+    sa.n_nt = n_nt; sa.stages = stages; sa.threshold = p->sim_threshold; sa.role = ctx->role;
+    sa.inv_norm = ctx->inv_norm; sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
+    sa.best_sim = out->best_sim; sa.status = ctx->status;
+    sim_kernel<<<dim3((in->max_vis + 127) / 128, B), SIM_THREADS, smem, st>>>(map_h, map_kept, sa);
+    ASAP_TRY(after_launch(ctx, "sim"));
+
+    csr_kernel<<<B, CSR_THREADS, (size_t)k * sizeof(int), st>>>(ctx->desc, in->max_vis, k, out->assign,
+                                                                 ctx->seg, ctx->members);
+    ASAP_TRY(after_launch(ctx, "csr"));
+  }
+  const long long bound_ll = (long long)in->total_tokens - (long long)B * (in->min_vis - k);
+  int bound = (int)(bound_ll < out->out_rows_capacity ? bound_ll : out->out_rows_capacity);
+  int blocks = bound < 148 * 8 ? bound : 148 * 8;
+  merge_compact_kernel<<<blocks, MERGE_THREADS, 0, st>>>(
+      static_cast<const __nv_bfloat16 *>(in->hidden), in->pos_ids, ctx->desc, B, D, in->max_vis, k, bound,
+      p->eps, do_merge ? 1 : 0, salience, keep_idx, drop_idx, ctx->seg, ctx->members,
+      static_cast<__nv_bfloat16 *>(out->out_hidden), out->out_pos, out->src_row);
+  return after_launch(ctx, "merge_compact");
+}
+
+}  // namespace
+
+// =================================================================================================
+// C ABI
+// =================================================================================================
+extern "C" {
+
+asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, int max_B, int max_H,
+                      int max_D, size_t max_keep_rows) {
+  g_init_error[0] = 0;
+  if (!ctx_out) return fail(nullptr, ASAP_ERR_INVALID, "asap_init: null ctx pointer");
+  *ctx_out = nullptr;
+  if (max_total_tokens == 0 || max_B <= 0 || max_H <= 0 || max_D <= 0 || max_D % 8 != 0)
+    return fail(nullptr, ASAP_ERR_INVALID, "asap_init: capacities must be positive, max_D a multiple of 8");
+  if (max_total_tokens > 0x7fffffffULL) return fail(nullptr, ASAP_ERR_INVALID, "asap_init: max_total_tokens too large");
+  if (max_keep_rows == 0) max_keep_rows = max_total_tokens;
+  cudaError_t e = cudaSetDevice(device);
+  if (e != cudaSuccess) return fail(nullptr, ASAP_ERR_CUDA, "cudaSetDevice(%d): %s", device, cudaGetErrorString(e));
+  cudaDeviceProp prop;
+  e = cudaGetDeviceProperties(&prop, device);
+  if (e != cudaSuccess) return fail(nullptr, ASAP_ERR_CUDA, "cudaGetDeviceProperties: %s", cudaGetErrorString(e));
+  if (prop.major != 10)
+    return fail(nullptr, ASAP_ERR_UNSUPPORTED, "libasap is built for sm_100a only; device %d is sm_%d%d", device,
+                prop.major, prop.minor);
+  asap_ctx *ctx = new (std::nothrow) asap_ctx();
+  if (!ctx) return fail(nullptr, ASAP_ERR_CUDA, "out of host memory");
+  ctx->device = device;
+  ctx->cap_tokens = max_total_tokens; ctx->cap_B = max_B; ctx->cap_H = max_H; ctx->cap_D = max_D;
+  ctx->cap_keep_rows = max_keep_rows;
+  ctx->cap_chunks = max_total_tokens / QSUM_ROWS + 2 * (size_t)max_B;
+
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+    delete ctx;
+    return fail(nullptr, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  }
+  ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+
+  const size_t T = max_total_tokens, Bc = (size_t)max_B, Hc = (size_t)max_H, Dc = (size_t)max_D;
+  const size_t col_blocks = (Dc + QSUM_COLS - 1) / QSUM_COLS;
+  size_t off = 0;
+  auto carve = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t o_desc = carve(Bc * sizeof(SampleDesc));
+  const size_t o_qpart = carve(ctx->cap_chunks * Dc * sizeof(float));
+  const size_t o_qbar = carve(Bc * Dc * sizeof(float));
+  const size_t o_spart = carve(Hc * T * sizeof(float));
+  const size_t o_inv = carve(T * sizeof(float));
+  const size_t o_kinv = carve(max_keep_rows * sizeof(float));
+  const size_t o_cnt = carve((Bc * col_blocks + 2 * Bc) * sizeof(unsigned int));
+  const size_t o_role = carve(T * sizeof(int32_t));
+  const size_t o_seg = carve((max_keep_rows + Bc) * sizeof(int32_t));
+  const size_t o_mem = carve(T * sizeof(int32_t));
+  const size_t o_kept = carve(max_keep_rows * Dc * sizeof(__nv_bfloat16));
+  const size_t o_status = carve(sizeof(uint32_t));
+  e = cudaMalloc(&ctx->arena, off);
+  if (e != cudaSuccess) {
+    delete ctx;
+    return fail(nullptr, ASAP_ERR_CUDA, "cudaMalloc of %zu scratch bytes: %s", off, cudaGetErrorString(e));
+  }
+  ctx->desc = reinterpret_cast<SampleDesc *>(ctx->arena + o_desc);
+  ctx->qsum_partial = reinterpret_cast<float *>(ctx->arena + o_qpart);
+  ctx->qbar = reinterpret_cast<float *>(ctx->arena + o_qbar);
+  ctx->score_partial = reinterpret_cast<float *>(ctx->arena + o_spart);
+  ctx->inv_norm = reinterpret_cast<float *>(ctx->arena + o_inv);
+  ctx->kept_inv = reinterpret_cast<float *>(ctx->arena + o_kinv);
+  ctx->cnt_qsum = reinterpret_cast<unsigned int *>(ctx->arena + o_cnt);
+  ctx->cnt_mass = ctx->cnt_qsum + Bc * col_blocks;
+  ctx->cnt_score = ctx->cnt_mass + Bc;
+  ctx->role = reinterpret_cast<int32_t *>(ctx->arena + o_role);
+  ctx->seg = reinterpret_cast<int32_t *>(ctx->arena + o_seg);
+  ctx->members = reinterpret_cast<int32_t *>(ctx->arena + o_mem);
+  ctx->kept_rows = reinterpret_cast<__nv_bfloat16 *>(ctx->arena + o_kept);
+  ctx->status = reinterpret_cast<uint32_t *>(ctx->arena + o_status);
+  e = cudaMemset(ctx->arena + o_cnt, 0, (Bc * col_blocks + 2 * Bc) * sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
+  // kernels whose dynamic shared memory exceeds the 48 KB default
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(csr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    cudaFree(ctx->arena);
+    delete ctx;
+    return fail(nullptr, ASAP_ERR_CUDA, "asap_init set-up: %s", cudaGetErrorString(e));
+  }
+  *ctx_out = ctx;
+  return ASAP_OK;
+}
+
+asap_status asap_score(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const asap_outputs *out,
+                       void *stream) {
+  ASAP_TRY(validate(ctx, in, p, out, NEED_QK | NEED_SCORE_OUT));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ASAP_TRY(launch_prepare(ctx, in, p, nullptr, 0x7fffffff, st));
+  return launch_score(ctx, in, p, out, st);
+}
+
+asap_status asap_select(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *rank_score,
+                        const asap_outputs *out, void *stream) {
+  ASAP_TRY(validate(ctx, in, p, out, NEED_SELECT_OUT));
+  if (!rank_score) return fail(ctx, ASAP_ERR_INVALID, "null rank_score");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ASAP_TRY(launch_prepare(ctx, in, p, nullptr, 0x7fffffff, st));
+  return launch_select(ctx, in, p, rank_score, out, st);
+}
+
+asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *salience,
+                       const int32_t *keep_idx, const int32_t *drop_idx, const asap_outputs *out,
+                       void *stream) {
+  ASAP_TRY(validate(ctx, in, p, out, NEED_HIDDEN | NEED_MERGE_OUT));
+  if (!salience || !keep_idx || (!drop_idx && in->max_vis > p->keep_k))
+    return fail(ctx, ASAP_ERR_INVALID, "null salience / keep_idx / drop_idx");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
+  role_map_kernel<<<dim3((in->max_vis + 255) / 256, in->B), 256, 0, st>>>(ctx->desc, in->max_vis, p->keep_k,
+                                                                         keep_idx, drop_idx, ctx->role);
+  ASAP_TRY(after_launch(ctx, "role_map"));
+  return launch_merge(ctx, in, p, salience, keep_idx, drop_idx, out, st);
+}
+
+asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const asap_outputs *out,
+                            void *stream) {
+  ASAP_TRY(validate(ctx, in, p, out, NEED_QK | NEED_HIDDEN | NEED_SCORE_OUT | NEED_SELECT_OUT | NEED_MERGE_OUT));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
+  ASAP_TRY(launch_score(ctx, in, p, out, st));
+  ASAP_TRY(launch_select(ctx, in, p, out->rank_score, out, st));
+  return launch_merge(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st);
+}
+
+asap_status asap_check(asap_ctx *ctx, void *stream) {
+  if (!ctx) return fail(nullptr, ASAP_ERR_INVALID, "null context");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, ctx->status, sizeof(word), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "asap_check: %s", cudaGetErrorString(e));
+  if (word == 0) { ctx->err[0] = 0; return ASAP_OK; }
+  cudaMemsetAsync(ctx->status, 0, sizeof(uint32_t), st);
+  cudaStreamSynchronize(st);
+  return fail(ctx, ASAP_ERR_DEVICE, "device status 0x%x:%s%s%s%s", word,
+              (word & STATUS_BAD_SAMPLE) ? " a per-sample span failed validation (sample skipped);" : "",
+              (word & STATUS_OUT_CAPACITY) ? " shortened batch exceeds out_rows_capacity (nothing written);" : "",
+              (word & STATUS_SCORE_TIMEOUT) ? " a wait timed out in the score kernel;" : "",
+              (word & STATUS_SIM_TIMEOUT) ? " a wait timed out in the similarity kernel;" : "");
+}
+
+const char *asap_last_error(const asap_ctx *ctx) { return ctx ? ctx->err : g_init_error; }
+
+uint64_t asap_launch_count(const asap_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+void asap_free(asap_ctx *ctx) {
+  if (!ctx) return;
+  cudaSetDevice(ctx->device);
+  cudaFree(ctx->arena);
+  delete ctx;
+}
+
+}  // extern "C"

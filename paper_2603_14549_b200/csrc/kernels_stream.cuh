@@ -1,0 +1,656 @@
+// The memory-bound and latency-bound kernels of the ASAP prune step:
+//   prepare        device-side validation, per-sample descriptors, output row offsets
+//   qsum           sum of the visual query rows                       (Eq. 1, summed over i first)
+//   mass_salience  s_j, then s_hat_j and m_j                          (Eq. 1, Eq. 2, Eq. 3)
+//   select         stable radix top-k of the ranking scores           (Fig. 3)
+//   role_map       kept slot / dropped position of every visual token
+//   norm_gather    inverse row norms; kept rows gathered for the similarity GEMM (Sec. 4.2)
+//   csr            dropped tokens grouped by destination slot
+//   merge_compact  Eq. 5 and the hand-off of Fig. 3
+#pragma once
+
+#include "common.cuh"
+
+namespace asap {
+
+// =======================================================================================
+// prepare
+// =======================================================================================
+struct PrepareArgs {
+  int32_t B, total_tokens, min_vis, max_vis, max_seq, max_rank, keep_k, out_capacity;
+  const int32_t *cu_seqlens, *vis_start, *vis_len, *text_start, *text_len, *rank_start, *rank_len;
+  SampleDesc *desc;          // [B]
+  int32_t *out_cu_seqlens;   // [B+1] or nullptr
+  uint32_t *status;
+};
+
+__global__ void prepare_kernel(PrepareArgs a) {
+  __shared__ int s_bad;
+  if (threadIdx.x == 0) s_bad = 0;
+  __syncthreads();
+  for (int b = threadIdx.x; b < a.B; b += blockDim.x) {
+    const int lo = a.cu_seqlens[b], hi = a.cu_seqlens[b + 1];
+    const int n = hi - lo;
+    const int v0 = a.vis_start[b], nv = a.vis_len[b];
+    const int t0 = a.text_start[b], tl = a.text_len[b];
+    const int r0 = a.rank_start ? a.rank_start[b] : t0;
+    const int nr = a.rank_len ? a.rank_len[b] : tl;
+    bool ok = lo >= 0 && n > 0 && n <= a.max_seq && hi <= a.total_tokens;
+    ok = ok && v0 >= 0 && nv >= a.min_vis && nv <= a.max_vis && v0 + nv <= n;
+    ok = ok && tl >= 0 && t0 >= v0 + nv && t0 + tl <= n;
+    ok = ok && r0 >= 0 && nr >= 1 && nr <= a.max_rank && r0 + nr <= n;
+    ok = ok && a.keep_k <= nv;
+    if (b == 0) ok = ok && lo == 0;
+    if (b == a.B - 1) ok = ok && hi == a.total_tokens;
+    SampleDesc d;
+    d.row0 = lo; d.n = n; d.v0 = v0; d.nv = nv; d.r0 = r0; d.nr = nr; d.out_row0 = 0;
+    d.valid = ok ? 1 : 0;
+    a.desc[b] = d;
+    if (!ok) s_bad = 1;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int acc = 0;
+    for (int b = 0; b < a.B; ++b) {
+      a.desc[b].out_row0 = acc;
+      if (a.out_cu_seqlens) a.out_cu_seqlens[b] = acc;
+      if (a.desc[b].valid) acc += a.desc[b].n - a.desc[b].nv + a.keep_k;
+    }
+    if (a.out_cu_seqlens) a.out_cu_seqlens[a.B] = acc;
+    uint32_t bits = 0;
+    if (s_bad) bits |= STATUS_BAD_SAMPLE;
+    if (acc > a.out_capacity) {
+      bits |= STATUS_OUT_CAPACITY;
+      for (int b = 0; b < a.B; ++b) a.desc[b].valid = 0;   // nothing may be written
+    }
+    if (bits) atomicOr(a.status, bits);
+  }
+}
+
+// =======================================================================================
+// qsum: qbar[b, c] = sum over visual rows i of q[i, c]   (fp32, fixed summation order)
+// grid (chunks, column blocks, B); a block sums QSUM_ROWS rows of 2048 columns and the block
+// that finishes last for (b, column block) adds the chunk partials in chunk order.
+// =======================================================================================
+constexpr int QSUM_ROWS = 32;
+constexpr int QSUM_THREADS = 256;
+constexpr int QSUM_COLS = QSUM_THREADS * 8;
+
+__global__ void __launch_bounds__(QSUM_THREADS)
+qsum_kernel(const __nv_bfloat16 *__restrict__ q, const SampleDesc *__restrict__ desc, int D,
+            int max_chunks, float *__restrict__ partial /*[B, max_chunks, D]*/,
+            float *__restrict__ qbar /*[B, D]*/, unsigned int *__restrict__ counters) {
+  const int b = blockIdx.z, cb = blockIdx.y, chunk = blockIdx.x;
+  const SampleDesc d = desc[b];
+  if (!d.valid) return;
+  const int nchunks = (d.nv + QSUM_ROWS - 1) / QSUM_ROWS;
+  if (chunk >= nchunks) return;
+  const int col = cb * QSUM_COLS + threadIdx.x * 8;
+  const bool active = col < D;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (active) {
+    const int r_lo = chunk * QSUM_ROWS;
+    const int r_hi = min(d.nv, r_lo + QSUM_ROWS);
+    const uint4 *base =
+        reinterpret_cast<const uint4 *>(q + (size_t)(d.row0 + d.v0) * D + col);
+    const size_t pitch = (size_t)D / 8;
+    int r = r_lo;
+    for (; r + 4 <= r_hi; r += 4) {
+      uint4 v0 = __ldg(base + (size_t)r * pitch);
+      uint4 v1 = __ldg(base + (size_t)(r + 1) * pitch);
+      uint4 v2 = __ldg(base + (size_t)(r + 2) * pitch);
+      uint4 v3 = __ldg(base + (size_t)(r + 3) * pitch);
+      float f[8];
+      unpack8(v0, f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] += f[e];
+      unpack8(v1, f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] += f[e];
+      unpack8(v2, f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] += f[e];
+      unpack8(v3, f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] += f[e];
+    }
+    for (; r < r_hi; ++r) {
+      uint4 v = __ldg(base + (size_t)r * pitch);
+      float f[8];
+      unpack8(v, f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] += f[e];
+    }
+    float4 *dst = reinterpret_cast<float4 *>(partial + ((size_t)b * max_chunks + chunk) * D + col);
+    dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+  }
+  // last block for (b, cb) reduces the chunk partials
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned int *c = counters + (size_t)b * gridDim.y + cb;
+    unsigned int old = atomicAdd(c, 1u);
+    s_last = (old == (unsigned int)(nchunks - 1));
+    if (s_last) *c = 0u;   // ready for the next call
+  }
+  __syncthreads();
+  if (!s_last || !active) return;
+  __threadfence();
+  float tot[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int c = 0; c < nchunks; ++c) {
+    const float4 *src =
+        reinterpret_cast<const float4 *>(partial + ((size_t)b * max_chunks + c) * D + col);
+    float4 a0 = __ldcg(src), a1 = __ldcg(src + 1);
+    tot[0] += a0.x; tot[1] += a0.y; tot[2] += a0.z; tot[3] += a0.w;
+    tot[4] += a1.x; tot[5] += a1.y; tot[6] += a1.z; tot[7] += a1.w;
+  }
+  float4 *dst = reinterpret_cast<float4 *>(qbar + (size_t)b * D + col);
+  dst[0] = make_float4(tot[0], tot[1], tot[2], tot[3]);
+  dst[1] = make_float4(tot[4], tot[5], tot[6], tot[7]);
+}
+
+// =======================================================================================
+// mass_salience: s_j = qbar . k_j / (H sqrt(d))  (Eq. 1 with the sum over queries taken first
+// and the mean over heads folded in); the block that finishes last for a sample then does the
+// min-max normalisation (Eq. 2) and the mask vector (Eq. 3).
+// grid (row blocks, B); 8 warps x 4 rows each.
+// =======================================================================================
+constexpr int MASS_THREADS = 256;
+constexpr int MASS_ROWS_PER_WARP = 4;
+constexpr int MASS_ROWS = (MASS_THREADS / 32) * MASS_ROWS_PER_WARP;
+
+__global__ void __launch_bounds__(MASS_THREADS)
+mass_salience_kernel(const __nv_bfloat16 *__restrict__ k, const SampleDesc *__restrict__ desc,
+                     int D, int max_vis, float scale, float lambda_max, float eps,
+                     const float *__restrict__ qbar, float *__restrict__ mass,
+                     float *__restrict__ salience, float *__restrict__ mask_log,
+                     unsigned int *__restrict__ counters) {
+  extern __shared__ float s_q[];   // [D]
+  __shared__ float s_red[2 * (MASS_THREADS / 32)];
+  __shared__ int s_last;
+  const int b = blockIdx.y;
+  const SampleDesc d = desc[b];
+  float *mass_b = mass + (size_t)b * max_vis;
+  if (!d.valid) {
+    for (int j = blockIdx.x * MASS_THREADS + threadIdx.x; j < max_vis; j += gridDim.x * MASS_THREADS) {
+      mass_b[j] = 0.f; salience[(size_t)b * max_vis + j] = 0.f; mask_log[(size_t)b * max_vis + j] = 0.f;
+    }
+    return;
+  }
+  const int nblocks = (d.nv + MASS_ROWS - 1) / MASS_ROWS;
+  if ((int)blockIdx.x >= nblocks) return;
+  for (int c = threadIdx.x * 4; c < D; c += MASS_THREADS * 4)
+    *reinterpret_cast<float4 *>(s_q + c) = __ldcg(reinterpret_cast<const float4 *>(qbar + (size_t)b * D + c));
+  __syncthreads();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int j0 = blockIdx.x * MASS_ROWS + warp * MASS_ROWS_PER_WARP;
+  const int nvec = D / 8;
+  float acc[MASS_ROWS_PER_WARP];
+  const uint4 *rowp[MASS_ROWS_PER_WARP];
+#pragma unroll
+  for (int r = 0; r < MASS_ROWS_PER_WARP; ++r) {
+    acc[r] = 0.f;
+    const int j = min(j0 + r, d.nv - 1);   // clamp: duplicates are discarded below
+    rowp[r] = reinterpret_cast<const uint4 *>(k + (size_t)(d.row0 + d.v0 + j) * D);
+  }
+  for (int v = lane; v < nvec; v += 32) {
+    uint4 kv[MASS_ROWS_PER_WARP];
+#pragma unroll
+    for (int r = 0; r < MASS_ROWS_PER_WARP; ++r) kv[r] = __ldg(rowp[r] + v);
+    const float4 qa = *reinterpret_cast<const float4 *>(s_q + v * 8);
+    const float4 qb = *reinterpret_cast<const float4 *>(s_q + v * 8 + 4);
+#pragma unroll
+    for (int r = 0; r < MASS_ROWS_PER_WARP; ++r) {
+      float f[8];
+      unpack8(kv[r], f);
+      acc[r] += f[0] * qa.x + f[1] * qa.y + f[2] * qa.z + f[3] * qa.w + f[4] * qb.x + f[5] * qb.y +
+                f[6] * qb.z + f[7] * qb.w;
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < MASS_ROWS_PER_WARP; ++r) {
+    const float tot = warp_sum(acc[r]);
+    if (lane == 0 && j0 + r < d.nv) mass_b[j0 + r] = tot * scale;
+  }
+
+  // ---- last block of the sample: Eq. 2 and Eq. 3 over the whole image span ----
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned int old = atomicAdd(counters + b, 1u);
+    s_last = (old == (unsigned int)(nblocks - 1));
+    if (s_last) counters[b] = 0u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  float lo = INFINITY, hi = -INFINITY;
+  for (int j = threadIdx.x; j < d.nv; j += MASS_THREADS) {
+    const float s = __ldcg(mass_b + j);
+    lo = fminf(lo, s); hi = fmaxf(hi, s);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+  }
+  if (lane == 0) { s_red[warp] = lo; s_red[MASS_THREADS / 32 + warp] = hi; }
+  __syncthreads();
+  lo = s_red[0]; hi = s_red[MASS_THREADS / 32];
+#pragma unroll
+  for (int w = 1; w < MASS_THREADS / 32; ++w) {
+    lo = fminf(lo, s_red[w]); hi = fmaxf(hi, s_red[MASS_THREADS / 32 + w]);
+  }
+  const float inv = 1.0f / ((hi - lo) + eps);
+  float *sal_b = salience + (size_t)b * max_vis, *msk_b = mask_log + (size_t)b * max_vis;
+  for (int j = threadIdx.x; j < max_vis; j += MASS_THREADS) {
+    if (j < d.nv) {
+      const float sh = (__ldcg(mass_b + j) - lo) * inv;
+      sal_b[j] = sh;
+      msk_b[j] = logf(fmaxf(lambda_max * sh, eps));
+    } else {
+      mass_b[j] = 0.f; sal_b[j] = 0.f; msk_b[j] = 0.f;
+    }
+  }
+}
+
+// =======================================================================================
+// select: exact top-k by radix select over order-preserving 32-bit keys, equal scores resolved
+// toward the lower index, outputs in ascending index order.  One block per sample.
+// =======================================================================================
+constexpr int SELECT_THREADS = 1024;
+
+__device__ __forceinline__ uint32_t score_key(float f) {
+  if (f != f) return 0u;                       // NaN ranks below everything
+  uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// exclusive prefix sum of one int per thread across the block; returns the block total in `total`
+__device__ __forceinline__ int block_exclusive_scan(int v, int *s_warp /*[32]*/, int &total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();   // s_warp may still be read from a previous scan
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int w = (lane < (int)(blockDim.x >> 5)) ? s_warp[lane] : 0;
+    int winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int t = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += t;
+    }
+    s_warp[lane] = winc - w;             // exclusive warp offsets
+    if (lane == 31) s_warp[32] = winc;   // block total
+  }
+  __syncthreads();
+  total = s_warp[32];
+  return s_warp[warp] + inc - v;
+}
+
+__global__ void __launch_bounds__(SELECT_THREADS)
+select_kernel(const float *__restrict__ rank_score, const SampleDesc *__restrict__ desc,
+              int max_vis, int keep_k, int32_t *__restrict__ keep_idx, int32_t *__restrict__ drop_idx,
+              int32_t *__restrict__ role /*[B, max_vis]*/) {
+  extern __shared__ uint32_t s_key[];   // [max_vis]
+  __shared__ int s_hist[256];
+  __shared__ int s_scan[33];
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_remaining;
+  const int b = blockIdx.x;
+  const SampleDesc d = desc[b];
+  const int nd_max = max_vis - keep_k;
+  int32_t *keep_b = keep_idx + (size_t)b * keep_k;
+  int32_t *drop_b = drop_idx + (size_t)b * nd_max;
+  int32_t *role_b = role + (size_t)b * max_vis;
+  if (!d.valid) {
+    for (int j = threadIdx.x; j < keep_k; j += blockDim.x) keep_b[j] = -1;
+    for (int j = threadIdx.x; j < nd_max; j += blockDim.x) drop_b[j] = -1;
+    for (int j = threadIdx.x; j < max_vis; j += blockDim.x) role_b[j] = 0;
+    return;
+  }
+  const int nv = d.nv;
+  for (int j = threadIdx.x; j < nv; j += blockDim.x)
+    s_key[j] = score_key(rank_score[(size_t)b * max_vis + j]);
+  if (threadIdx.x == 0) { s_prefix = 0u; s_remaining = keep_k; }
+  __syncthreads();
+
+  // four 8-bit digits, most significant first: find the key of the keep_k-th largest score
+  uint32_t known = 0u;   // mask of the digits fixed so far
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_hist[i] = 0;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    for (int j = threadIdx.x; j < nv; j += blockDim.x) {
+      const uint32_t key = s_key[j];
+      if ((key & known) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      const int lane = threadIdx.x;
+      // lane L owns digits 255-8L .. 248-8L (descending); find where the running count reaches `remaining`
+      int mine = 0;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mine += s_hist[255 - 8 * lane - e];
+      int inc = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+      }
+      const int remaining = s_remaining;
+      __syncwarp();   // every lane has read s_remaining before one of them rewrites it
+      const int before = inc - mine;
+      if (before < remaining && remaining <= inc) {
+        int run = before;
+        for (int e = 0; e < 8; ++e) {
+          const int digit = 255 - 8 * lane - e;
+          const int c = s_hist[digit];
+          if (run + c >= remaining) {
+            s_prefix = prefix | ((uint32_t)digit << shift);
+            s_remaining = remaining - run;
+            break;
+          }
+          run += c;
+        }
+      }
+    }
+    known |= 255u << shift;
+    __syncthreads();
+  }
+  const uint32_t kth = s_prefix;      // key of the keep_k-th largest score
+  const int take_equal = s_remaining; // how many tokens with exactly that key are kept (lowest indices)
+
+  // ordered emission: thread t owns the contiguous indices [t*per, (t+1)*per)
+  const int per = (nv + blockDim.x - 1) / blockDim.x;
+  const int lo = min(nv, (int)threadIdx.x * per), hi = min(nv, lo + per);
+  int n_eq = 0;
+  for (int j = lo; j < hi; ++j) n_eq += (s_key[j] == kth);
+  int tot;
+  int eq_before = block_exclusive_scan(n_eq, s_scan, tot);
+  int n_keep = 0;
+  {
+    int e = eq_before;
+    for (int j = lo; j < hi; ++j) {
+      const uint32_t key = s_key[j];
+      n_keep += (key > kth) || (key == kth && e < take_equal);
+      e += (key == kth);
+    }
+  }
+  int keep_before = block_exclusive_scan(n_keep, s_scan, tot);
+  {
+    int e = eq_before, kp = keep_before;
+    for (int j = lo; j < hi; ++j) {
+      const uint32_t key = s_key[j];
+      const bool kept = (key > kth) || (key == kth && e < take_equal);
+      e += (key == kth);
+      if (kept) {
+        keep_b[kp] = j; role_b[j] = kp; ++kp;
+      } else {
+        const int dp = j - kp;
+        drop_b[dp] = j; role_b[j] = -(dp + 1);
+      }
+    }
+  }
+  for (int j = nv - keep_k + threadIdx.x; j < nd_max; j += blockDim.x) drop_b[j] = -1;
+  for (int j = nv + threadIdx.x; j < max_vis; j += blockDim.x) role_b[j] = 0;
+}
+
+// role map from caller-provided keep / drop lists (entry point asap_merge)
+__global__ void role_map_kernel(const SampleDesc *__restrict__ desc, int max_vis, int keep_k,
+                                const int32_t *__restrict__ keep_idx,
+                                const int32_t *__restrict__ drop_idx, int32_t *__restrict__ role) {
+  const int b = blockIdx.y;
+  const SampleDesc d = desc[b];
+  if (!d.valid) return;
+  const int nd_max = max_vis - keep_k;
+  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < d.nv; t += gridDim.x * blockDim.x) {
+    if (t < keep_k) {
+      const int j = keep_idx[(size_t)b * keep_k + t];
+      if (j >= 0 && j < d.nv) role[(size_t)b * max_vis + j] = t;
+    } else {
+      const int dp = t - keep_k;
+      const int j = drop_idx[(size_t)b * nd_max + dp];
+      if (j >= 0 && j < d.nv) role[(size_t)b * max_vis + j] = -(dp + 1);
+    }
+  }
+}
+
+// =======================================================================================
+// norm_gather: one warp per visual row.  inv_norm = 1/||h|| (0 if ||h|| < 1e-12, which makes
+// every similarity of that row 0); kept rows are also copied to their slot of the dense
+// [B*keep_k, D] operand of the similarity GEMM together with their inverse norm.
+// =======================================================================================
+constexpr int NORM_THREADS = 256;
+
+__global__ void __launch_bounds__(NORM_THREADS)
+norm_gather_kernel(const __nv_bfloat16 *__restrict__ hidden, const SampleDesc *__restrict__ desc,
+                   int D, int max_vis, int keep_k, const int32_t *__restrict__ role,
+                   float *__restrict__ inv_norm /*[B, max_vis]*/,
+                   __nv_bfloat16 *__restrict__ kept_rows /*[B*keep_k, D]*/,
+                   float *__restrict__ kept_inv /*[B*keep_k]*/) {
+  const int b = blockIdx.y;
+  const SampleDesc d = desc[b];
+  if (!d.valid) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int j = blockIdx.x * (NORM_THREADS / 32) + warp;
+  if (j >= d.nv) return;
+  const int slot = role[(size_t)b * max_vis + j];
+  const uint4 *src = reinterpret_cast<const uint4 *>(hidden + (size_t)(d.row0 + d.v0 + j) * D);
+  uint4 *dst = slot >= 0 ? reinterpret_cast<uint4 *>(kept_rows + ((size_t)b * keep_k + slot) * D) : nullptr;
+  const int nvec = D / 8;
+  float ss = 0.f;
+  for (int v = lane; v < nvec; v += 128) {
+    uint4 x[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (v + 32 * u < nvec) x[u] = __ldg(src + v + 32 * u);
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (v + 32 * u < nvec) {
+        float f[8];
+        unpack8(x[u], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ss += f[e] * f[e];
+        if (dst) dst[v + 32 * u] = x[u];
+      }
+  }
+  ss = warp_sum(ss);
+  if (lane == 0) {
+    const float nrm = sqrtf(ss);
+    const float inv = nrm >= 1e-12f ? 1.0f / nrm : 0.f;
+    inv_norm[(size_t)b * max_vis + j] = inv;
+    if (slot >= 0) kept_inv[(size_t)b * keep_k + slot] = inv;
+  }
+}
+
+// =======================================================================================
+// csr: group the dropped tokens by destination slot (counting sort, stable in dropped order so
+// the merge adds its members in a fixed order).  One block per sample.
+// seg [B, keep_k+1], members [B, max_vis-keep_k] (dropped POSITIONS, ascending inside a slot).
+// =======================================================================================
+constexpr int CSR_THREADS = 1024;
+
+__global__ void __launch_bounds__(CSR_THREADS)
+csr_kernel(const SampleDesc *__restrict__ desc, int max_vis, int keep_k,
+           const int32_t *__restrict__ assign, int32_t *__restrict__ seg,
+           int32_t *__restrict__ members) {
+  extern __shared__ int s_cnt[];   // [keep_k] counts, then cursors
+  __shared__ int s_scan[33];
+  const int b = blockIdx.x;
+  const SampleDesc d = desc[b];
+  int32_t *seg_b = seg + (size_t)b * (keep_k + 1);
+  if (!d.valid) {
+    for (int i = threadIdx.x; i <= keep_k; i += blockDim.x) seg_b[i] = 0;
+    return;
+  }
+  const int nd_max = max_vis - keep_k, nd = d.nv - keep_k;
+  const int32_t *as_b = assign + (size_t)b * nd_max;
+  int32_t *mem_b = members + (size_t)b * nd_max;
+  for (int i = threadIdx.x; i < keep_k; i += blockDim.x) s_cnt[i] = 0;
+  __syncthreads();
+  for (int p = threadIdx.x; p < nd; p += blockDim.x) {
+    const int a = as_b[p];
+    if (a >= 0 && a < keep_k) atomicAdd(&s_cnt[a], 1);
+  }
+  __syncthreads();
+  // exclusive scan over slots; thread t owns a contiguous range of slots
+  const int per = (keep_k + blockDim.x - 1) / blockDim.x;
+  const int lo = min(keep_k, (int)threadIdx.x * per), hi = min(keep_k, lo + per);
+  int mine = 0;
+  for (int i = lo; i < hi; ++i) mine += s_cnt[i];
+  int tot;
+  int run = block_exclusive_scan(mine, s_scan, tot);
+  for (int i = lo; i < hi; ++i) {
+    const int c = s_cnt[i];
+    seg_b[i] = run;
+    s_cnt[i] = run;      // becomes the slot's write cursor
+    run += c;
+  }
+  if (threadIdx.x == 0) seg_b[keep_k] = tot;
+  __syncthreads();
+  // stable fill by one warp, 32 dropped positions at a time in ascending order
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    for (int base = 0; base < nd; base += 32) {
+      const int p = base + lane;
+      int a = (p < nd) ? as_b[p] : -1;
+      if (a >= keep_k) a = -1;
+      const unsigned peers = __match_any_sync(0xffffffffu, a);
+      const int rank = __popc(peers & ((1u << lane) - 1u));
+      int cur = 0;
+      if (a >= 0) cur = s_cnt[a];
+      __syncwarp();
+      if (a >= 0) {
+        mem_b[cur + rank] = p;
+        if (rank == 0) s_cnt[a] = cur + __popc(peers);
+      }
+      __syncwarp();
+    }
+  }
+}
+
+// =======================================================================================
+// merge_compact: one block per output row (grid-stride).  Prefix and suffix rows are copied;
+// a kept visual row becomes (s_hat_i h_i + sum_j s_hat_j h_j) / (s_hat_i + sum_j s_hat_j)
+// over the dropped tokens j assigned to it (Eq. 5), accumulated in fp32 in a fixed order and
+// rounded to bf16 once.  A row without members, or whose total weight is <= eps, is copied.
+// =======================================================================================
+constexpr int MERGE_THREADS = 256;
+constexpr int MERGE_MAX_VEC = 4;   // 16-byte vectors per thread: D <= 256*4*8 = 8192
+
+__global__ void __launch_bounds__(MERGE_THREADS)
+merge_compact_kernel(const __nv_bfloat16 *__restrict__ hidden, const int32_t *__restrict__ pos_ids,
+                     const SampleDesc *__restrict__ desc, int B, int D, int max_vis, int keep_k,
+                     int out_rows_bound, float eps, int merge_enable,
+                     const float *__restrict__ salience, const int32_t *__restrict__ keep_idx,
+                     const int32_t *__restrict__ drop_idx, const int32_t *__restrict__ seg,
+                     const int32_t *__restrict__ members, __nv_bfloat16 *__restrict__ out_hidden,
+                     int32_t *__restrict__ out_pos, int32_t *__restrict__ src_row) {
+  const int nvec = D / 8;
+  const int nd_max = max_vis - keep_k;
+  for (int orow = blockIdx.x; orow < out_rows_bound; orow += gridDim.x) {
+    // sample that owns this output row: last b with out_row0 <= orow
+    int lo = 0, hi = B - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (desc[mid].out_row0 <= orow) lo = mid; else hi = mid - 1;
+    }
+    const int b = lo;
+    const SampleDesc d = desc[b];
+    const int local = orow - d.out_row0;
+    const int out_len = d.n - d.nv + keep_k;
+    if (!d.valid || local >= out_len) continue;   // past the end of the shortened batch
+    int srow;         // sequence-relative source row
+    int slot = -1;
+    if (local < d.v0) srow = local;
+    else if (local < d.v0 + keep_k) {
+      slot = local - d.v0;
+      srow = d.v0 + min(max(keep_idx[(size_t)b * keep_k + slot], 0), d.nv - 1);
+    } else srow = local - keep_k + d.nv;
+    const size_t grow = (size_t)(d.row0 + srow);
+    if (threadIdx.x == 0) {
+      out_pos[orow] = pos_ids[grow];
+      src_row[orow] = (int32_t)grow;
+    }
+    const uint4 *src = reinterpret_cast<const uint4 *>(hidden + grow * D);
+    uint4 *dst = reinterpret_cast<uint4 *>(out_hidden + (size_t)orow * D);
+    int m_lo = 0, m_hi = 0;
+    if (slot >= 0 && merge_enable) {
+      m_lo = seg[(size_t)b * (keep_k + 1) + slot];
+      m_hi = seg[(size_t)b * (keep_k + 1) + slot + 1];
+    }
+    if (m_hi == m_lo) {
+#pragma unroll
+      for (int u = 0; u < MERGE_MAX_VEC; ++u) {
+        const int v = threadIdx.x + u * MERGE_THREADS;
+        if (v < nvec) dst[v] = __ldg(src + v);
+      }
+      continue;
+    }
+    const float *sal_b = salience + (size_t)b * max_vis;
+    const float w_self = sal_b[srow - d.v0];
+    float acc[MERGE_MAX_VEC][8];
+#pragma unroll
+    for (int u = 0; u < MERGE_MAX_VEC; ++u) {
+      const int v = threadIdx.x + u * MERGE_THREADS;
+      if (v < nvec) {
+        float f[8];
+        unpack8(__ldg(src + v), f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[u][e] = w_self * f[e];
+      }
+    }
+    float den = w_self;
+    const int32_t *mem_b = members + (size_t)b * nd_max;
+    const int32_t *drop_b = drop_idx + (size_t)b * nd_max;
+    for (int m = m_lo; m < m_hi; ++m) {
+      const int j = min(max(drop_b[mem_b[m]], 0), d.nv - 1);   // visual index of the member
+      const float w = sal_b[j];
+      den += w;
+      const uint4 *msrc = reinterpret_cast<const uint4 *>(hidden + (size_t)(d.row0 + d.v0 + j) * D);
+#pragma unroll
+      for (int u = 0; u < MERGE_MAX_VEC; ++u) {
+        const int v = threadIdx.x + u * MERGE_THREADS;
+        if (v < nvec) {
+          float f[8];
+          unpack8(__ldg(msrc + v), f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[u][e] += w * f[e];
+        }
+      }
+    }
+    if (den <= eps) {
+#pragma unroll
+      for (int u = 0; u < MERGE_MAX_VEC; ++u) {
+        const int v = threadIdx.x + u * MERGE_THREADS;
+        if (v < nvec) dst[v] = __ldg(src + v);
+      }
+    } else {
+      const float inv = 1.0f / den;
+#pragma unroll
+      for (int u = 0; u < MERGE_MAX_VEC; ++u) {
+        const int v = threadIdx.x + u * MERGE_THREADS;
+        if (v < nvec) {
+          uint4 o;
+          o.x = pack2_rn(acc[u][0] * inv, acc[u][1] * inv);
+          o.y = pack2_rn(acc[u][2] * inv, acc[u][3] * inv);
+          o.z = pack2_rn(acc[u][4] * inv, acc[u][5] * inv);
+          o.w = pack2_rn(acc[u][6] * inv, acc[u][7] * inv);
+          dst[v] = o;
+        }
+      }
+    }
+  }
+}
+
+}  // namespace asap

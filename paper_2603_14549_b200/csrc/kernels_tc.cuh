@@ -1,0 +1,537 @@
+// The two dense contractions of the ASAP prune step on the sm_100a tensor cores
+// (tcgen05.mma, operands staged by TMA into 128-byte-swizzled shared memory, fp32
+// accumulators in tensor memory):
+//
+//   score_kernel  Eq. 3 / Eq. 4: masked softmax of the ranking rows' logits, reduced over
+//                 ranking rows; the logits never leave the SM.
+//   sim_kernel    Sec. 4.2: cosine similarity of every visual row against the kept rows with
+//                 the arg-max over kept slots taken in the epilogue.
+//
+// Both use one TMA-producer warp, one MMA-issuer warp (a single elected lane) and four
+// epilogue warps that read tensor memory (warp w may touch lanes 32*(w%4) .. 32*(w%4)+31).
+// Every mbarrier wait is bounded (see WaitCtx); after an abort the block keeps walking its
+// uniform control flow so that every named barrier and the final teardown are still reached.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace asap {
+
+constexpr long long TC_WAIT_LIMIT = 1500000000LL;   // clock cycles, roughly one second
+constexpr float LOG2E_F = 1.4426950408889634f;
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// =======================================================================================
+// score_kernel
+//
+// One block per (head h, sample b).  For each tile of up to 128 ranking rows:
+//   pass 1  D = Q_rows K_tile^T   (M = 128 rows,  N = 128 keys): thread-per-row running
+//           max / sum over all admitted keys  ->  off_i = max_i + log2(sum_i)   (log2 units)
+//   pass 2  D = K_tile Q_rows^T   (M = 128 keys,  N = rows):     thread-per-key sum over rows
+//           of exp2(logit + mask - off_i), i.e. of the Eq. 4 probabilities A[i, j]
+// Pass 2 walks the key tiles in reverse so that the tiles still resident in the shared-memory
+// ring (a direct-mapped cache of key tiles, stage = tile mod stages) are reused without a
+// reload; tiles that were evicted come back from L2.
+// Additive mask (Eq. 3), logits in log2 units: 0 for key j <= row position p; m_j*log2(e) for
+// j > p when both are in the image span (mask enabled); -inf otherwise.
+// =======================================================================================
+constexpr int SC_THREADS = 192;
+constexpr int SC_STAGES = 5;
+constexpr int SC_HALF_BYTES = 128 * 128;        // 128 rows x 64 bf16
+constexpr int SC_TILE_BYTES = 2 * SC_HALF_BYTES;
+constexpr int SC_SMEM_MAIN = (1 + SC_STAGES) * SC_TILE_BYTES;
+constexpr int SC_SMEM_BYTES = SC_SMEM_MAIN + 2048 + 1024;   // + bookkeeping + alignment slack
+constexpr uint32_t SC_TMEM_COLS = 256;
+
+struct ScoreArgs {
+  const SampleDesc *desc;
+  int H, max_vis, mask_enable;
+  float scale_log2;           // log2(e) / sqrt(head_dim)
+  const float *mask_log;      // [B, max_vis]  m_j (natural log)
+  float *partial;             // [B, H, max_vis] per-head sums over ranking rows
+  float *rank_score;          // [B, max_vis]
+  unsigned int *counters;     // [B]
+  uint32_t *status;
+};
+
+struct ScoreBook {             // bookkeeping block placed after the tiles in shared memory
+  uint64_t full[SC_STAGES], empty[SC_STAGES], q_full, q_empty, acc_full[2], acc_empty[2];
+  float off[128];              // per ranking row: max + log2(sum), +inf for rows past the tile
+  float soft[128];             // per key of the current tile: m_j*log2(e) or -inf
+  int sim_res[2][SC_STAGES];   // [role][stage] tile resident in the stage (producer / issuer copies)
+  int sim_fill[2][SC_STAGES];
+  int sim_use[2][SC_STAGES];
+  uint32_t tmem_base;
+  int abort_flag;
+  int is_last;
+};
+
+struct RowTile {
+  int R0, nrows, n_kt, t_lo, t_hi;
+  bool use_soft;
+};
+
+__device__ __forceinline__ RowTile score_row_tile(const SampleDesc &d, int rt, int mask_enable) {
+  RowTile r;
+  r.R0 = d.r0 + rt * 128;
+  r.nrows = min(128, d.nr - rt * 128);
+  const int p_max = r.R0 + r.nrows - 1;
+  r.use_soft = mask_enable && (r.R0 < d.v0 + d.nv) && (p_max >= d.v0);
+  int jmax = p_max;
+  if (r.use_soft) jmax = max(jmax, d.v0 + d.nv - 1);
+  r.n_kt = jmax / 128 + 1;
+  r.t_lo = d.v0 / 128;
+  r.t_hi = min((d.v0 + d.nv - 1) / 128, r.n_kt - 1);
+  return r;
+}
+
+__global__ void __launch_bounds__(SC_THREADS, 1)
+score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+             ScoreArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const int h = blockIdx.x, b = blockIdx.y;
+  const SampleDesc d = a.desc[b];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float *rank_b = a.rank_score + (size_t)b * a.max_vis;
+  if (!d.valid) {
+    if (h == 0)
+      for (int j = threadIdx.x; j < a.max_vis; j += SC_THREADS) rank_b[j] = 0.f;
+    return;
+  }
+  if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SCORE_TIMEOUT) return;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_smem = base;
+  const uint32_t k_smem = base + SC_TILE_BYTES;
+  ScoreBook *bk = reinterpret_cast<ScoreBook *>(base_ptr + SC_SMEM_MAIN);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < SC_STAGES; ++s) {
+      mbar_init(smem_u32(&bk->full[s]), 1);
+      mbar_init(smem_u32(&bk->empty[s]), 1);
+      for (int r = 0; r < 2; ++r) { bk->sim_res[r][s] = -1; bk->sim_fill[r][s] = 0; bk->sim_use[r][s] = 0; }
+    }
+    mbar_init(smem_u32(&bk->q_full), 1);
+    mbar_init(smem_u32(&bk->q_empty), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&bk->acc_full[i]), 1);
+      mbar_init(smem_u32(&bk->acc_empty[i]), 4);
+    }
+    bk->abort_flag = 0;
+    bk->is_last = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bk->tmem_base), SC_TMEM_COLS);
+    tmem_relinquish();
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bk->tmem_base;
+  WaitCtx wc{&bk->abort_flag, a.status, STATUS_SCORE_TIMEOUT, TC_WAIT_LIMIT};
+  const int n_rt = (d.nr + 127) / 128;
+  const int grow0 = d.row0;   // packed row of the sequence start
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tmap_q);
+      tma_prefetch_desc(&tmap_k);
+      int *res = bk->sim_res[0], *fill = bk->sim_fill[0], *use = bk->sim_use[0];
+      for (int rt = 0; rt < n_rt; ++rt) {
+        const RowTile T = score_row_tile(d, rt, a.mask_enable);
+        if (rt > 0) mbar_wait(smem_u32(&bk->q_empty), (rt - 1) & 1, wc);
+        if (!bk->abort_flag) {
+          mbar_expect_tx(smem_u32(&bk->q_full), SC_TILE_BYTES);
+          tma_load_2d(q_smem, &tmap_q, smem_u32(&bk->q_full), h * 128, grow0 + T.R0);
+          tma_load_2d(q_smem + SC_HALF_BYTES, &tmap_q, smem_u32(&bk->q_full), h * 128 + 64, grow0 + T.R0);
+        }
+        const int n_p2 = T.t_hi >= T.t_lo ? T.t_hi - T.t_lo + 1 : 0;
+        for (int u = 0; u < T.n_kt + n_p2; ++u) {
+          const int t = u < T.n_kt ? u : T.t_hi - (u - T.n_kt);
+          const int s = t % SC_STAGES;
+          if (res[s] != t) {
+            if (use[s] > 0) mbar_wait(smem_u32(&bk->empty[s]), (use[s] - 1) & 1, wc);
+            if (!bk->abort_flag) {
+              const uint32_t dst = k_smem + s * SC_TILE_BYTES;
+              mbar_expect_tx(smem_u32(&bk->full[s]), SC_TILE_BYTES);
+              tma_load_2d(dst, &tmap_k, smem_u32(&bk->full[s]), h * 128, grow0 + t * 128);
+              tma_load_2d(dst + SC_HALF_BYTES, &tmap_k, smem_u32(&bk->full[s]), h * 128 + 64, grow0 + t * 128);
+              fill[s] += 1;
+            }
+            res[s] = t;
+          }
+          use[s] += 1;
+        }
+      }
+      // every copy this thread issued must have landed before the block may leave
+      for (int s = 0; s < SC_STAGES; ++s)
+        if (fill[s] > 0) mbar_wait_drain(smem_u32(&bk->full[s]), (fill[s] - 1) & 1, TC_WAIT_LIMIT);
+      mbar_wait_drain(smem_u32(&bk->q_full), (n_rt - 1) & 1, TC_WAIT_LIMIT);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int *res = bk->sim_res[1], *fill = bk->sim_fill[1];
+      int g = 0;
+      for (int rt = 0; rt < n_rt; ++rt) {
+        const RowTile T = score_row_tile(d, rt, a.mask_enable);
+        const int n2 = (T.nrows + 15) & ~15;
+        const uint32_t idesc1 = umma_idesc_bf16(128, 128);
+        const uint32_t idesc2 = umma_idesc_bf16(128, n2);
+        mbar_wait(smem_u32(&bk->q_full), rt & 1, wc);
+        const int n_p2 = T.t_hi >= T.t_lo ? T.t_hi - T.t_lo + 1 : 0;
+        for (int u = 0; u < T.n_kt + n_p2; ++u, ++g) {
+          const bool pass1 = u < T.n_kt;
+          const int t = pass1 ? u : T.t_hi - (u - T.n_kt);
+          const int s = t % SC_STAGES, buf = g & 1;
+          if (g >= 2) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((g >> 1) - 1) & 1, wc);
+          if (res[s] != t) {
+            res[s] = t;
+            fill[s] += 1;
+            mbar_wait(smem_u32(&bk->full[s]), (fill[s] - 1) & 1, wc);
+          }
+          tc_fence_after();
+          if (!bk->abort_flag) {
+            const uint32_t ks = k_smem + s * SC_TILE_BYTES;
+            const uint32_t dcol = tmem_base + buf * 128;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+              const uint32_t o = (kk >> 2) * SC_HALF_BYTES + (kk & 3) * 32;
+              const uint64_t dq = umma_desc_sw128(q_smem + o), dk = umma_desc_sw128(ks + o);
+              if (pass1) tc_mma_bf16(dcol, dq, dk, idesc1, kk > 0);
+              else       tc_mma_bf16(dcol, dk, dq, idesc2, kk > 0);
+            }
+            tc_commit(smem_u32(&bk->empty[s]));
+            tc_commit(smem_u32(&bk->acc_full[buf]));
+          }
+        }
+        if (!bk->abort_flag) tc_commit(smem_u32(&bk->q_empty));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (4 warps)
+    const int quarter = warp & 3;
+    const int lrow = quarter * 32 + lane;          // tensor-memory lane owned by this thread
+    const int et = (warp - 2) * 32 + lane;         // 0..127 among the epilogue threads
+    float *part = a.partial + ((size_t)b * a.H + h) * a.max_vis;
+    for (int j = et; j < d.nv; j += 128) part[j] = 0.f;
+    epi_bar_sync();
+    const float *mlog = a.mask_log + (size_t)b * a.max_vis;
+    const float scale = a.scale_log2;
+    const int v_end = d.v0 + d.nv;
+    int g = 0;
+    for (int rt = 0; rt < n_rt; ++rt) {
+      const RowTile T = score_row_tile(d, rt, a.mask_enable);
+      const int n_p2 = T.t_hi >= T.t_lo ? T.t_hi - T.t_lo + 1 : 0;
+      // ---------------- pass 1: thread = ranking row
+      const bool row_ok = lrow < T.nrows;
+      const bool warp_rows = quarter * 32 < T.nrows;
+      const int p_i = T.R0 + lrow;
+      const bool row_vis = T.use_soft && p_i >= d.v0 && p_i < v_end;
+      float m = -INFINITY, l = 0.f;
+      for (int t = 0; t < T.n_kt; ++t, ++g) {
+        const int buf = g & 1, j0 = t * 128;
+        const bool fast = (j0 + 127 <= T.R0);
+        const bool stage_soft = T.use_soft && !fast;
+        if (stage_soft) {
+          const int j = j0 + lrow;
+          bk->soft[lrow] = (j >= d.v0 && j < v_end) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
+          epi_bar_sync();
+        }
+        mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 1) & 1, wc);
+        tc_fence_after();
+        if (warp_rows) {
+          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 128;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c * 32, r);
+            tmem_wait_ld();
+            float x[32];
+            float cmax = -INFINITY;
+            if (fast) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) { x[e] = __uint_as_float(r[e]) * scale; cmax = fmaxf(cmax, x[e]); }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) {
+                const int j = j0 + c * 32 + e;
+                float add;
+                if (j <= p_i) add = 0.f;
+                else add = (row_vis && stage_soft) ? bk->soft[c * 32 + e] : -INFINITY;
+                x[e] = __uint_as_float(r[e]) * scale + add;
+                cmax = fmaxf(cmax, x[e]);
+              }
+            }
+            const float m_new = fmaxf(m, cmax);
+            if (row_ok && m_new > -INFINITY) {
+              float sum = 0.f;
+#pragma unroll
+              for (int e = 0; e < 32; ++e) sum += fast_exp2(x[e] - m_new);
+              l = l * fast_exp2(m - m_new) + sum;
+              m = m_new;
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
+        if (stage_soft) epi_bar_sync();
+      }
+      // per-row offset: exp2(x - off) = exp2(x - max) / sum
+      bk->off[lrow] = row_ok ? (m + __log2f(l)) : INFINITY;
+      epi_bar_sync();
+      // ---------------- pass 2: thread = key
+      const int n2 = (T.nrows + 15) & ~15;
+      for (int u = 0; u < n_p2; ++u, ++g) {
+        const int t = T.t_hi - u, buf = g & 1, j0 = t * 128;
+        const int j = j0 + lrow;
+        const bool key_ok = j >= d.v0 && j < v_end;
+        const bool fast = (j0 + 127 <= T.R0);
+        const bool warp_keys = (j0 + quarter * 32 + 31 >= d.v0) && (j0 + quarter * 32 < v_end);
+        const float soft_j = (T.use_soft && key_ok) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
+        mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 1) & 1, wc);
+        tc_fence_after();
+        if (warp_keys) {
+          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 128;
+          float sum = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < n2; c += 16) {
+            uint32_t r[16];
+            tmem_ld16(taddr + c, r);
+            tmem_wait_ld();
+            if (fast) {
+#pragma unroll
+              for (int e = 0; e < 16; ++e) sum += fast_exp2(__uint_as_float(r[e]) * scale - bk->off[c + e]);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                const int p = T.R0 + c + e;
+                float add;
+                if (j <= p) add = 0.f;
+                else add = (p >= d.v0 && p < v_end) ? soft_j : -INFINITY;
+                sum += fast_exp2(__uint_as_float(r[e]) * scale + add - bk->off[c + e]);
+              }
+            }
+          }
+          if (key_ok) part[j - d.v0] += sum;
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
+      }
+      epi_bar_sync();   // off[] is rewritten by the next row tile
+    }
+    __threadfence();
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, SC_TMEM_COLS);
+  }
+  // the block that finishes last for this sample adds the heads in head order
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned int old = atomicAdd(a.counters + b, 1u);
+    bk->is_last = (old == (unsigned int)(a.H - 1));
+    if (bk->is_last) a.counters[b] = 0u;
+  }
+  __syncthreads();
+  if (!bk->is_last) return;
+  __threadfence();
+  const float inv = 1.0f / ((float)a.H * (float)d.nr);
+  for (int j = threadIdx.x; j < a.max_vis; j += SC_THREADS) {
+    float tot = 0.f;
+    if (j < d.nv) {
+      const float *p = a.partial + (size_t)b * a.H * a.max_vis + j;
+      for (int hh = 0; hh < a.H; ++hh) tot += __ldcg(p + (size_t)hh * a.max_vis);
+      tot *= inv;
+    }
+    rank_b[j] = tot;
+  }
+}
+
+// =======================================================================================
+// sim_kernel
+//
+// One block per (128 visual rows, sample).  D = V_tile Kept^T with M = 128 visual rows,
+// N = n_tile kept slots per accumulator, K = the hidden size in steps of 64.  The epilogue
+// scales column s by 1/||kept_s||, keeps the running maximum and the first slot attaining it,
+// and finally writes, for rows that were dropped, the slot (or -1 if the cosine similarity is
+// not above the threshold) and the similarity.  Rows that were kept, or lie past the image
+// span, are computed but not written.
+// =======================================================================================
+constexpr int SIM_THREADS = 192;
+constexpr int SIM_A_BYTES = 128 * 128;           // 128 rows x 64 bf16
+constexpr int SIM_BOOK_BYTES = 1024;
+constexpr uint32_t SIM_TMEM_COLS = 512;
+constexpr int SIM_MAX_STAGES = 8;
+
+struct SimArgs {
+  const SampleDesc *desc;
+  int D, max_vis, keep_k, n_tile, n_nt, stages;
+  float threshold;
+  const int32_t *role;       // [B, max_vis]
+  const float *inv_norm;     // [B, max_vis]
+  const float *kept_inv;     // [B*keep_k]
+  int32_t *assign;           // [B, max_vis-keep_k]
+  float *best_sim;           // [B, max_vis-keep_k] or nullptr
+  uint32_t *status;
+};
+
+struct SimBook {
+  uint64_t full[SIM_MAX_STAGES], empty[SIM_MAX_STAGES], acc_full[2], acc_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(SIM_THREADS, 1)
+sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_kept,
+           SimArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const int mt = blockIdx.x, b = blockIdx.y;
+  const SampleDesc d = a.desc[b];
+  if (!d.valid || mt * 128 >= d.nv) return;
+  if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SIM_TIMEOUT) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const int b_bytes = a.n_tile * 128;
+  const int stage_bytes = SIM_A_BYTES + b_bytes;
+  SimBook *bk = reinterpret_cast<SimBook *>(base_ptr + (size_t)a.stages * stage_bytes);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < a.stages; ++s) {
+      mbar_init(smem_u32(&bk->full[s]), 1);
+      mbar_init(smem_u32(&bk->empty[s]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&bk->acc_full[i]), 1);
+      mbar_init(smem_u32(&bk->acc_empty[i]), 4);
+    }
+    bk->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bk->tmem_base), SIM_TMEM_COLS);
+    tmem_relinquish();
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bk->tmem_base;
+  WaitCtx wc{&bk->abort_flag, a.status, STATUS_SIM_TIMEOUT, TC_WAIT_LIMIT};
+  const int n_kb = a.D / 64;
+  const int total_it = a.n_nt * n_kb;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tmap_h);
+      tma_prefetch_desc(&tmap_kept);
+      const int row_a = d.row0 + d.v0 + mt * 128;
+      const int row_b = b * a.keep_k;
+      int issued = 0;
+      for (int it = 0; it < total_it; ++it) {
+        const int s = it % a.stages, nt = it / n_kb, kb = it - nt * n_kb;
+        if (it >= a.stages) mbar_wait(smem_u32(&bk->empty[s]), ((it / a.stages) - 1) & 1, wc);
+        if (bk->abort_flag) break;
+        const uint32_t dst = base + s * stage_bytes;
+        mbar_expect_tx(smem_u32(&bk->full[s]), stage_bytes);
+        tma_load_2d(dst, &tmap_h, smem_u32(&bk->full[s]), kb * 64, row_a);
+        tma_load_2d(dst + SIM_A_BYTES, &tmap_kept, smem_u32(&bk->full[s]), kb * 64, row_b + nt * a.n_tile);
+        issued = it + 1;
+      }
+      // drain: the last fill of every stage must have landed before the block leaves
+      for (int s = 0; s < a.stages; ++s) {
+        // last iteration index < issued that maps to stage s
+        if (issued > s) {
+          const int last = ((issued - 1 - s) / a.stages) * a.stages + s;
+          mbar_wait_drain(smem_u32(&bk->full[s]), (last / a.stages) & 1, TC_WAIT_LIMIT);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(128, a.n_tile);
+      int it = 0;
+      for (int nt = 0; nt < a.n_nt; ++nt) {
+        const int buf = nt & 1;
+        if (nt >= 2) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((nt >> 1) - 1) & 1, wc);
+        const uint32_t dcol = tmem_base + buf * 256;
+        for (int kb = 0; kb < n_kb; ++kb, ++it) {
+          const int s = it % a.stages;
+          mbar_wait(smem_u32(&bk->full[s]), (it / a.stages) & 1, wc);
+          tc_fence_after();
+          if (!bk->abort_flag) {
+            const uint32_t sa = base + s * stage_bytes, sb = sa + SIM_A_BYTES;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              tc_mma_bf16(dcol, umma_desc_sw128(sa + kk * 32), umma_desc_sw128(sb + kk * 32), idesc,
+                          (kb > 0 || kk > 0) ? 1u : 0u);
+            tc_commit(smem_u32(&bk->empty[s]));
+          }
+        }
+        if (!bk->abort_flag) tc_commit(smem_u32(&bk->acc_full[buf]));
+      }
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int v = mt * 128 + quarter * 32 + lane;       // visual index of this thread's row
+    const float *kinv = a.kept_inv + (size_t)b * a.keep_k;
+    float best = -INFINITY;
+    int best_slot = 0;
+    for (int nt = 0; nt < a.n_nt; ++nt) {
+      const int buf = nt & 1;
+      mbar_wait(smem_u32(&bk->acc_full[buf]), (nt >> 1) & 1, wc);
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 256;
+      const int slot0 = nt * a.n_tile;
+      const int ncol = min(a.n_tile, a.keep_k - slot0);   // kept slots in this accumulator
+#pragma unroll 1
+      for (int c = 0; c < ncol; c += 16) {
+        uint32_t r[16];
+        tmem_ld16(taddr + c, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const int slot = slot0 + c + e;
+          if (c + e < ncol) {
+            const float val = __uint_as_float(r[e]) * __ldg(kinv + slot);
+            if (val > best) { best = val; best_slot = slot; }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
+    }
+    if (v < d.nv && !bk->abort_flag) {
+      const int role = a.role[(size_t)b * a.max_vis + v];
+      if (role < 0) {
+        const int dp = -role - 1;
+        const float sim = best * a.inv_norm[(size_t)b * a.max_vis + v];
+        const size_t o = (size_t)b * (a.max_vis - a.keep_k) + dp;
+        a.assign[o] = (sim > a.threshold) ? best_slot : -1;
+        if (a.best_sim) a.best_sim[o] = sim;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, SIM_TMEM_COLS);
+  }
+}
+
+}  // namespace asap

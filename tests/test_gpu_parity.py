@@ -1,0 +1,159 @@
+"""GPU parity: the CUDA prune step, called through the C ABI, against the CPU oracle on the
+same seeded inputs.  Sizes span several 128-wide tiles with ragged tails; the benchmark shapes
+run at full size with the oracle evaluated on a sample of the sequences."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_14549_b200 import binding as A
+from paper_2603_14549_b200 import workloads as W
+from tests.parity import compare_sample
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = A.asap_init(0, max_total_tokens=80000, max_B=32, max_H=40, max_D=5120, max_keep_rows=40000)
+    yield c
+    A.asap_free(c)
+
+
+def run_step(ctx, batch, params, rank_start=None, rank_len=None, samples=None, stats=None):
+    inp = A.make_inputs(batch, DEV, rank_start, rank_len)
+    out = A.alloc_outputs(inp, params.keep_k, fill=True)
+    A.asap_prune_step(ctx, inp, params, out)
+    torch.cuda.synchronize()
+    A.asap_check(ctx)
+    for b in (range(batch.B) if samples is None else samples):
+        compare_sample(batch, b, params, out, rank_start, rank_len, stats)
+    return inp, out
+
+
+def test_ragged_multi_tile(ctx):
+    batch = W.tiny(B=3, n_vis=[130, 257, 64], text_lens=[5, 17, 33], H=2, keep_k=16, seed=101, centres=6)
+    run_step(ctx, batch, A.Params(keep_k=16))
+
+
+def test_text_longer_than_one_row_tile(ctx):
+    batch = W.tiny(B=2, n_vis=[200, 140], text_lens=[150, 129], H=2, keep_k=40, seed=102, centres=8)
+    run_step(ctx, batch, A.Params(keep_k=40))
+
+
+@pytest.mark.parametrize("lambda_max", [1.0, 0.5, 0.1])
+def test_visual_ranking_rows_use_the_soft_mask(ctx, lambda_max):
+    batch = W.tiny(B=2, n_vis=[300, 129], text_lens=[20, 7], H=2, keep_k=32, seed=103, centres=8)
+    rs = batch.vis_start.clone()
+    rl = batch.vis_len + batch.text_len            # ranking rows = image span + text span
+    run_step(ctx, batch, A.Params(keep_k=32, lambda_max=lambda_max), rs, rl)
+
+
+def test_ranking_rows_partly_visual_and_mask_off(ctx):
+    batch = W.tiny(B=2, n_vis=[260, 131], text_lens=[9, 30], H=1, keep_k=20, seed=104)
+    rs = batch.vis_start + 100
+    rl = batch.vis_len - 100 + batch.text_len
+    run_step(ctx, batch, A.Params(keep_k=20, lambda_max=0.7), rs, rl)
+    run_step(ctx, batch, A.Params(keep_k=20, mask_enable=False), rs, rl)
+
+
+def test_identity_when_k_equals_visual_count(ctx):
+    batch = W.tiny(B=2, n_vis=[150, 150], text_lens=[4, 40], H=2, keep_k=150, seed=105)
+    inp, out = run_step(ctx, batch, A.Params(keep_k=150))
+    assert torch.equal(out.out_hidden.cpu(), batch.hidden)
+    assert torch.equal(out.out_pos.cpu(), batch.pos_ids)
+
+
+def test_mask_off_merge_off_is_plain_topk_gather(ctx):
+    batch = W.tiny(B=2, n_vis=[190, 133], text_lens=[12, 31], H=2, keep_k=24, seed=106)
+    inp, out = run_step(ctx, batch, A.Params(keep_k=24, mask_enable=False, merge_enable=False))
+    src = out.src_row.cpu().long()
+    assert torch.equal(out.out_hidden.cpu(), batch.hidden[src])
+
+
+@pytest.mark.parametrize("t", [0.8, 0.95, 1.0])
+def test_similarity_threshold(ctx, t):
+    batch = W.tiny(B=2, n_vis=[180, 140], text_lens=[10, 20], H=2, keep_k=30, seed=107, centres=5)
+    inp, out = run_step(ctx, batch, A.Params(keep_k=30, sim_threshold=t))
+    if t >= 1.0:
+        assert int((out.assign >= 0).sum()) == 0
+
+
+@pytest.mark.parametrize("nv", [1, 2, 3, 5, 8, 127, 128, 129])
+@pytest.mark.parametrize("tl", [1, 16, 17])
+def test_edge_sizes(ctx, nv, tl):
+    ks = sorted({1, max(1, nv - 1), nv})
+    for k in ks:
+        batch = W.tiny(B=2, n_vis=[nv, nv], text_lens=[tl, tl + 1], H=1, keep_k=k, seed=200 + nv, centres=2)
+        run_step(ctx, batch, A.Params(keep_k=k))
+
+
+def test_duplicate_token_merges_into_its_twin(ctx):
+    batch = W.tiny(B=1, n_vis=[140], text_lens=[8], H=2, keep_k=20, seed=108, centres=50)
+    inp = A.make_inputs(batch, DEV)
+    out = A.alloc_outputs(inp, 20, fill=True)
+    p = A.Params(keep_k=20)
+    A.asap_prune_step(ctx, inp, p, out)
+    torch.cuda.synchronize()
+    keep = out.keep_idx[0].cpu()
+    drop = out.drop_idx[0].cpu()
+    v0 = int(batch.vis_start[0])
+    # overwrite one dropped token with a copy of kept token #3 and rerun: it must land on slot 3
+    victim = int(drop[5])
+    batch.hidden[v0 + victim] = batch.hidden[v0 + int(keep[3])]
+    inp2, out2 = run_step(ctx, batch, p)
+    pos = (out2.drop_idx[0] == victim).nonzero()
+    if len(pos):     # the twin is still dropped (ranking does not depend on hidden states)
+        dp = int(pos[0])
+        assert int(out2.assign[0, dp]) == 3
+        assert abs(float(out2.best_sim[0, dp]) - 1.0) < 1e-5
+
+
+def test_c1_full(ctx):
+    stats = {}
+    batch = W.config("c1")
+    run_step(ctx, batch, A.Params(keep_k=batch.keep_k), stats=stats)
+    print("c1 parity maxima", stats)
+
+
+def test_c2_full_size_sampled(ctx):
+    stats = {}
+    batch = W.config("c2")
+    run_step(ctx, batch, A.Params(keep_k=batch.keep_k), samples=[0, 7, 15], stats=stats)
+    print("c2 parity maxima", stats)
+
+
+@pytest.mark.parametrize("k", [320, 160])
+def test_c3_prefix_with_outliers(ctx, k):
+    stats = {}
+    batch = W.config("c3", B=2, keep_k=k)
+    run_step(ctx, batch, A.Params(keep_k=k), samples=[1], stats=stats)
+    print("c3 parity maxima", stats)
+
+
+def test_c4_prefix_sampled(ctx):
+    stats = {}
+    batch = W.config("c4", B=6)
+    run_step(ctx, batch, A.Params(keep_k=batch.keep_k), samples=[5], stats=stats)
+    print("c4 parity maxima", stats)
+
+
+def test_c5_progressive_three_steps(ctx):
+    """13B-shaped schedule 2304 -> 1152 -> 576 -> 288: every step consumes the previous step's
+    hidden states and gathered position ids, with Q/K re-drawn at those positions."""
+    batch = W.config("c5", B=2)
+    cur = batch
+    for step, k in enumerate(W.C5_SCHEDULE):
+        p = A.Params(keep_k=k)
+        cur.keep_k = k
+        inp, out = run_step(ctx, cur, p, samples=[1])
+        ocu = out.out_cu_seqlens.cpu()
+        hidden = out.out_hidden[: int(ocu[-1])].cpu()
+        pos = out.out_pos[: int(ocu[-1])].cpu()
+        q, kk = W.redraw_qk(pos, ocu, cur.H, cur.head_dim, cur.seed, step + 1)
+        cur = W.Batch(name="c5", B=cur.B, H=cur.H, head_dim=cur.head_dim, D=cur.D, keep_k=k, cu_seqlens=ocu,
+                      vis_start=cur.vis_start, vis_len=torch.full_like(cur.vis_len, k),
+                      text_start=cur.vis_start + k, text_len=cur.text_len, q=q, k=kk, hidden=hidden,
+                      pos_ids=pos, seed=cur.seed)
