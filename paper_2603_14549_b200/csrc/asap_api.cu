@@ -98,6 +98,16 @@ asap_status validate(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
     return fail(ctx, ASAP_ERR_INVALID, "lambda_max must be in (0, 1]");
   if (!(p->eps > 0.f)) return fail(ctx, ASAP_ERR_INVALID, "eps must be positive");
   if (p->sim_threshold != p->sim_threshold) return fail(ctx, ASAP_ERR_INVALID, "sim_threshold is NaN");
+  // capacities
+  if ((size_t)in->total_tokens > ctx->cap_tokens || in->B > ctx->cap_B || in->H > ctx->cap_H ||
+      in->D > ctx->cap_D)
+    return fail(ctx, ASAP_ERR_WORKSPACE, "problem exceeds the capacities given to asap_init");
+  if ((size_t)in->B * (size_t)in->max_vis > ctx->cap_tokens)
+    return fail(ctx, ASAP_ERR_WORKSPACE, "B * max_vis exceeds max_total_tokens");
+  if ((size_t)in->B * (size_t)p->keep_k > ctx->cap_keep_rows)
+    return fail(ctx, ASAP_ERR_WORKSPACE, "B * keep_k exceeds max_keep_rows");
+  const size_t chunks = (size_t)in->B * ((in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS);
+  if (chunks > ctx->cap_chunks) return fail(ctx, ASAP_ERR_WORKSPACE, "query-sum scratch too small for B * max_vis");
   if (!in->cu_seqlens || !in->vis_start || !in->vis_len || !in->text_start || !in->text_len)
     return fail(ctx, ASAP_ERR_INVALID, "null per-sample array");
   if ((in->rank_start == nullptr) != (in->rank_len == nullptr))
@@ -111,26 +121,17 @@ asap_status validate(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
   }
   if ((need & NEED_SCORE_OUT) && (!out->mass || !out->salience || !out->mask_log || !out->rank_score))
     return fail(ctx, ASAP_ERR_INVALID, "null score output (mass / salience / mask_log / rank_score)");
-  if ((need & NEED_SELECT_OUT) && (!out->keep_idx || !out->drop_idx))
+  const bool has_drops = in->max_vis > p->keep_k;   // otherwise the dropped-token arrays are empty
+  if ((need & NEED_SELECT_OUT) && (!out->keep_idx || (!out->drop_idx && has_drops)))
     return fail(ctx, ASAP_ERR_INVALID, "null keep_idx / drop_idx");
   if (need & NEED_MERGE_OUT) {
-    if (!out->assign || !out->out_hidden || !out->out_pos || !out->src_row || !out->out_cu_seqlens)
+    if ((!out->assign && has_drops) || !out->out_hidden || !out->out_pos || !out->src_row || !out->out_cu_seqlens)
       return fail(ctx, ASAP_ERR_INVALID, "null merge output");
     if (!aligned16(out->out_hidden)) return fail(ctx, ASAP_ERR_ALIGN, "out_hidden must be 16-byte aligned");
     const long long bound = (long long)in->total_tokens - (long long)in->B * (in->min_vis - p->keep_k);
     if (out->out_rows_capacity <= 0 || bound <= 0)
       return fail(ctx, ASAP_ERR_INVALID, "out_rows_capacity must be positive");
   }
-  // capacities
-  if ((size_t)in->total_tokens > ctx->cap_tokens || in->B > ctx->cap_B || in->H > ctx->cap_H ||
-      in->D > ctx->cap_D)
-    return fail(ctx, ASAP_ERR_WORKSPACE, "problem exceeds the capacities given to asap_init");
-  if ((size_t)in->B * (size_t)in->max_vis > ctx->cap_tokens)
-    return fail(ctx, ASAP_ERR_WORKSPACE, "B * max_vis exceeds max_total_tokens");
-  if ((size_t)in->B * (size_t)p->keep_k > ctx->cap_keep_rows)
-    return fail(ctx, ASAP_ERR_WORKSPACE, "B * keep_k exceeds max_keep_rows");
-  const size_t chunks = (size_t)in->B * ((in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS);
-  if (chunks > ctx->cap_chunks) return fail(ctx, ASAP_ERR_WORKSPACE, "query-sum scratch too small for B * max_vis");
   return ASAP_OK;
 }
 

@@ -155,8 +155,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         for (int u = 0; u < T.n_kt + n_p2; ++u) {
           const int t = u < T.n_kt ? u : T.t_hi - (u - T.n_kt);
           const int s = t % SC_STAGES;
+          // The previous use of this stage must have finished, both before a refill and
+          // before a reuse is booked: an mbarrier wait only tells phases apart by parity, so
+          // the producer may never fall two completions behind on a stage.
+          if (use[s] > 0) mbar_wait(smem_u32(&bk->empty[s]), (use[s] - 1) & 1, wc);
           if (res[s] != t) {
-            if (use[s] > 0) mbar_wait(smem_u32(&bk->empty[s]), (use[s] - 1) & 1, wc);
             if (!bk->abort_flag) {
               const uint32_t dst = k_smem + s * SC_TILE_BYTES;
               mbar_expect_tx(smem_u32(&bk->full[s]), SC_TILE_BYTES);
