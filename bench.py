@@ -1,0 +1,401 @@
+"""Benchmark of the ASAP prune step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1..c5] [--impl reference]
+
+A step is one pass of the whole prune step (attention mass, salience, mask, masked ranking
+scores, top-k, cosine assignment, weighted merge, compaction) over one synthetic batch.  The
+default workload is the LLaVA-1.5-7B-shaped batch of 16 sequences (576 visual tokens, ragged
+text, keep 64).  One JSON line is printed by rank 0:
+
+  value          visual tokens per second, inputs resident in HBM, all ranks together
+  e2e            the same with inputs in pinned host memory: every step copies them to the
+                 device, runs the step through the C ABI and reads the shortened batch back
+  roofline       the kernel with the largest share of the step, against the measured peak
+  kernels        per-kernel device time (CUDA events recorded by the library on its stream)
+  cpu_baseline   the float64 CPU oracle timed on this host's cores on a few sequences
+
+With --impl reference the CPU oracle alone is timed (rank 0 only).
+With N > 1 every rank prunes its own batch of the same shape (sequences are independent, there
+is no exchange step): the ranks only meet at the barriers around the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2603_14549_b200 import replicas as R
+from paper_2603_14549_b200 import workloads as W
+
+METRIC = "visual_tokens_per_sec"
+UNIT = "tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+WORKLOADS = {
+    "c1": "LLaVA-1.5-7B single sequence: 35 system + 576 visual + 32 text, D=4096, 32x128 heads, keep 192",
+    "c2": "LLaVA-1.5-7B batch 16: 35 system + 576 visual + text U[16,128], D=4096, 32x128 heads, keep 64",
+    "c3": "LLaVA-NeXT-7B batch 8: 35 system + 2304 visual + 64 text, D=4096, 32x128 heads, keep 320",
+    "c4": "LLaVA-NeXT AnyRes batch 64: 35 system + 2880 visual + text U[32,256], D=4096, 32x128 heads, keep 576",
+    "c5": "13B-shaped batch 32, first step of 2304->1152: 35 system + 2304 visual + 128 text, D=5120, 40x128 heads",
+}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------------------
+# algorithmic traffic / work of each kernel for one launch over the whole batch
+# ------------------------------------------------------------------------------------------
+def algorithmic(batch, keep_k):
+    """Bytes each kernel must move and flops it must do, from the problem sizes alone:
+    every operand it consumes read once, every result written once (bf16 = 2 bytes)."""
+    D = batch.D
+    out = {name: {"bytes": 0, "flops": 0} for name in
+           ("qsum", "mass_salience", "score", "select", "norm_gather", "sim", "csr", "merge_compact",
+            "prepare", "fill_assign")}
+    for b in range(batch.B):
+        n = int(batch.cu_seqlens[b + 1] - batch.cu_seqlens[b])
+        nv, tl = int(batch.vis_len[b]), int(batch.text_len[b])
+        t0 = int(batch.text_start[b])
+        row = D * 2
+        out["qsum"]["bytes"] += nv * row
+        out["qsum"]["flops"] += nv * D
+        out["mass_salience"]["bytes"] += nv * row + nv * 12
+        out["mass_salience"]["flops"] += 2 * nv * D
+        # ranking rows = text span: queries once, every key they may attend to once
+        out["score"]["bytes"] += tl * row + (t0 + tl) * row + nv * 4
+        out["score"]["flops"] += 2 * tl * (t0 + (tl + 1) // 2) * D
+        out["select"]["bytes"] += nv * 4 + nv * 4
+        out["norm_gather"]["bytes"] += nv * row
+        out["norm_gather"]["flops"] += 2 * nv * D
+        out["sim"]["bytes"] += nv * row
+        out["sim"]["flops"] += 2 * (nv - keep_k) * keep_k * D
+        out["csr"]["bytes"] += (nv - keep_k) * 8
+        out["merge_compact"]["bytes"] += n * row + (n - nv + keep_k) * row
+        out["merge_compact"]["flops"] += 2 * nv * D
+    return out
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.path = tempfile.mktemp(prefix="asap_clocks_", suffix=".csv")
+        self.proc = None
+        self.index = device_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    parts = [p.strip() for p in line.split(",")]
+                    if len(parts) < 7:
+                        continue
+                    try:
+                        sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+                    except ValueError:
+                        continue
+                    for nm, v in zip(names, parts[3:7]):
+                        if v.lower().startswith("active"):
+                            reasons.add(nm)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle legs (the only places that touch oracle/)
+# ------------------------------------------------------------------------------------------
+def time_oracle(batch, keep_k, budget_s=12.0, max_samples=None):
+    """Runs the float64 oracle sequence by sequence until `budget_s` of CPU time is used or the
+    batch is exhausted; returns (visual tokens per second, seconds, sequences, threads)."""
+    from oracle import asap_oracle as O
+    import numpy as np
+
+    def bits(t):   # bf16 tensor -> uint16 bit patterns, the form the oracle takes
+        return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    done, tokens = 0, 0
+    t_start = time.perf_counter()
+    limit = batch.B if max_samples is None else min(batch.B, max_samples)
+    while done < limit:
+        b = done
+        rows = batch.sample_rows(b)
+        O.prune_sample(bits(batch.q[rows]), bits(batch.k[rows]), bits(batch.hidden[rows]),
+                       batch.pos_ids[rows].numpy(), int(batch.vis_start[b]), int(batch.vis_len[b]),
+                       int(batch.text_start[b]), int(batch.text_len[b]), keep_k)
+        done += 1
+        tokens += int(batch.vis_len[b])
+        if time.perf_counter() - t_start >= budget_s:
+            break
+    secs = time.perf_counter() - t_start
+    return tokens / secs, secs, done, threads
+
+
+def run_reference(args):
+    rank, size, _ = R.world()
+    if rank != 0:
+        return
+    batch = W.config(args.workload, B=args.ref_sequences)
+    keep_k = batch.keep_k
+    for _ in range(args.warmup):
+        time_oracle(batch, keep_k, budget_s=1e9, max_samples=1)
+    t0 = time.perf_counter()
+    tokens = 0
+    threads = 1
+    for _ in range(args.steps):
+        v, secs, done, threads = time_oracle(batch, keep_k, budget_s=1e9)
+        tokens += sum(int(batch.vis_len[b]) for b in range(done))
+    secs = time.perf_counter() - t0
+    value = tokens / secs
+    sample = f"{batch.B} sequence(s) of {args.workload} per step, float64 numpy oracle"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ------------------------------------------------------------------------------------------
+# CUDA arm
+# ------------------------------------------------------------------------------------------
+def device_copies(A, batch, device, n_copies):
+    first = A.make_inputs(batch, device)
+    copies = [first]
+    import dataclasses
+    for _ in range(n_copies - 1):
+        copies.append(dataclasses.replace(first, q=first.q.clone(), k=first.k.clone(),
+                                          hidden=first.hidden.clone(), pos_ids=first.pos_ids.clone()))
+    return copies
+
+
+def run_cuda(args):
+    from paper_2603_14549_b200 import binding as A   # raises if libasap.so is missing: no fallback
+    rank, size, local = R.init("nccl")
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (B200); there is no CPU path")
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    peaks, peak_kind = load_peaks()
+
+    seed = R.replica_seed(W.BASE_SEED + int(args.workload[1]) - 1, rank)
+    batch = W.config(args.workload, seed=seed)
+    keep_k = batch.keep_k
+    params = A.Params(keep_k=keep_k)
+    units = int(batch.vis_len.sum())
+    in_bytes = sum(t.numel() * t.element_size() for t in (batch.q, batch.k, batch.hidden, batch.pos_ids))
+    n_copies = max(2, min(64, -(-(8 * L2_BYTES) // in_bytes)))
+    ctx = A.asap_init(local, max_total_tokens=batch.total, max_B=batch.B, max_H=batch.H, max_D=batch.D,
+                      max_keep_rows=batch.B * keep_k)
+    copies = device_copies(A, batch, device, n_copies)
+    out = A.alloc_outputs(copies[0], keep_k)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        A.asap_prune_step(ctx, copies[i % n_copies], params, out, stream)
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    A.asap_check(ctx)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    launches0 = A.asap_launch_count(ctx)
+    R.barrier(); torch.cuda.synchronize()
+    marks[0].record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i)
+        marks[i + 1].record(stream)
+    torch.cuda.synchronize(); R.barrier()
+    launches = A.asap_launch_count(ctx) - launches0
+    total_ms = marks[0].elapsed_time(marks[-1])
+    per_step = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
+    A.asap_check(ctx)
+    total_ms_max = R.max_over_ranks(total_ms, device)
+    units_all = R.sum_over_ranks(units, device)
+
+    # ---- per-kernel device times: the same steps again with the library's own events on
+    A.asap_profile(ctx, True)
+    for i in range(args.steps):
+        step(args.warmup + i)
+    torch.cuda.synchronize()
+    ktimes = A.asap_profile_read(ctx)
+    A.asap_profile(ctx, False)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end from pinned host memory
+    e2e = None
+    if not args.no_e2e:
+        host = {n: getattr(batch, n).contiguous().pin_memory() for n in ("q", "k", "hidden", "pos_ids")}
+        dev_in = copies[0]
+        n_out_rows = batch.total - units + batch.B * keep_k
+        host_out = {"out_hidden": torch.empty(n_out_rows, batch.D, dtype=torch.bfloat16).pin_memory(),
+                    "out_pos": torch.empty(n_out_rows, dtype=torch.int32).pin_memory(),
+                    "out_cu_seqlens": torch.empty(batch.B + 1, dtype=torch.int32).pin_memory(),
+                    "keep_idx": torch.empty(batch.B, keep_k, dtype=torch.int32).pin_memory()}
+        h2d = sum(t.numel() * t.element_size() for t in host.values())
+        d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+
+        def e2e_step():
+            for n, t in host.items():
+                getattr(dev_in, n).copy_(t, non_blocking=True)
+            A.asap_prune_step(ctx, dev_in, params, out, stream)
+            host_out["out_hidden"].copy_(out.out_hidden[:n_out_rows], non_blocking=True)
+            host_out["out_pos"].copy_(out.out_pos[:n_out_rows], non_blocking=True)
+            host_out["out_cu_seqlens"].copy_(out.out_cu_seqlens, non_blocking=True)
+            host_out["keep_idx"].copy_(out.keep_idx, non_blocking=True)
+            stream.synchronize()            # the caller consumes the shortened batch every step
+
+        e_steps = max(3, min(args.steps, 20))
+        for _ in range(3):
+            e2e_step()
+        R.barrier(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e_steps):
+            e2e_step()
+        e1.record(stream)
+        torch.cuda.synchronize(); R.barrier()
+        e_ms = R.max_over_ranks(e0.elapsed_time(e1), device)
+        e2e = {"value": units_all * e_steps / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": e_steps, "ms_per_step": e_ms / e_steps}
+        A.asap_check(ctx)
+    A.asap_free(ctx)
+
+    if rank != 0:
+        R.shutdown()
+        return
+
+    # ---- roofline of the dominant kernel
+    alg = algorithmic(batch, keep_k)
+    ksum = sum(ms for _, ms in ktimes.values()) or 1.0
+    kernels = {}
+    for name, (n, ms) in sorted(ktimes.items(), key=lambda kv: -kv[1][1]):
+        avg_s = ms / max(n, 1) * 1e-3
+        a = alg.get(name, {"bytes": 0, "flops": 0})
+        kernels[name] = {"launches": n, "avg_us": avg_s * 1e6, "share": ms / ksum,
+                         "alg_GBs": a["bytes"] / avg_s / 1e9 if avg_s > 0 else None,
+                         "alg_TFLOPs": a["flops"] / avg_s / 1e12 if avg_s > 0 else None}
+    top = next(iter(kernels)) if kernels else None
+    roofline = None
+    if top:
+        a, kt = alg[top], kernels[top]
+        hbm_frac = kt["alg_GBs"] / peaks["hbm_gbs"]
+        tc_frac = kt["alg_TFLOPs"] / peaks["bf16_tflops"]
+        if top == "sim" and tc_frac > hbm_frac:
+            roofline = {"kernel": top, "bound": "tensor", "achieved": kt["alg_TFLOPs"], "peak": peaks["bf16_tflops"],
+                        "unit": "TFLOP/s", "frac": tc_frac, "traffic": None, "peak_kind": peak_kind + " (burst)"}
+        else:
+            roofline = {"kernel": top, "bound": "hbm", "achieved": kt["alg_GBs"], "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "frac": hbm_frac, "traffic": None, "peak_kind": peak_kind}
+        roofline["algorithmic_bytes_per_launch"] = a["bytes"]
+        roofline["algorithmic_flops_per_launch"] = a["flops"]
+        roofline["avg_launch_us"] = kt["avg_us"]
+        traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(traffic_path):       # DRAM bytes per launch from the committed ncu capture
+            with open(traffic_path) as f:
+                tr = json.load(f).get(args.workload, {}).get(top)
+            roofline["traffic"] = tr
+
+    # ---- CPU oracle baseline on a bounded sample
+    cpu = None
+    if not args.no_cpu_baseline:
+        v, secs, done, threads = time_oracle(batch, keep_k, budget_s=args.cpu_budget)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"first {done} of {batch.B} sequences of {args.workload}, {secs:.1f} s, float64 numpy"}
+
+    step_s = total_ms_max * 1e-3 / args.steps
+    line = {
+        "metric": METRIC, "value": units_all / step_s, "unit": UNIT, "n_gpus": size, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}", "sequences_per_gpu": batch.B,
+                   "visual_tokens_per_gpu": units, "keep_k": keep_k, "ranking_rows": "text span",
+                   "l2": f"inputs rotate over {n_copies} device copies ({n_copies * in_bytes / 2**20:.0f} MiB) "
+                         f"so no step finds its inputs in the {L2_BYTES // 2**20} MiB L2",
+                   "parallelism": "replicas only (one batch per GPU, no collective)"},
+        "latency_us": {"p10": per_step[len(per_step) // 10] * 1e3, "p50": per_step[len(per_step) // 2] * 1e3,
+                       "p90": per_step[(len(per_step) * 9) // 10] * 1e3},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "kernels": kernels,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    R.shutdown()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
+    ap.add_argument("--ref-sequences", type=int, default=2,
+                    help="--impl reference: sequences of the workload the oracle prunes per step")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

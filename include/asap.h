@@ -148,6 +148,24 @@ asap_status asap_check(asap_ctx *ctx, void *stream);
  * next call on the context.  asap_last_error(NULL) describes a failed asap_init. */
 const char *asap_last_error(const asap_ctx *ctx);
 
+/* Per-kernel device times.  Not part of the method (the paper has no counterpart): a
+ * measurement aid.  asap_profile(ctx, 1) makes every later entry point drop one CUDA event on
+ * its stream before each kernel and one after its last kernel (the first enabling call creates
+ * the events; at most 16384 are used between two reads, later launches go untimed).
+ * asap_profile(ctx, 0) stops that.  Either call clears the accumulated times. */
+typedef struct {
+  char name[32];     /* kernel name: "qsum", "mass_salience", "score", "select", "sim", ... */
+  uint64_t launches; /* launches timed since profiling was enabled */
+  double total_ms;   /* sum over those launches of (next event - this kernel's event) */
+} asap_kernel_time;
+asap_status asap_profile(asap_ctx *ctx, int enable);
+
+/* Waits for the last recorded event, folds the events recorded since the previous read into
+ * the per-kernel totals, copies up to `capacity` totals to `out` (host memory) and returns how
+ * many kernels have a total.  A kernel's time runs to the start of the next kernel of the same
+ * call, so it includes the launch gap behind it. */
+int asap_profile_read(asap_ctx *ctx, asap_kernel_time *out, int capacity);
+
 /* Number of kernel launches the library has enqueued through this context so far. */
 uint64_t asap_launch_count(const asap_ctx *ctx);
 

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "ASAP_OK", -1: "ASAP_ERR_INVALID", -2: "ASAP_ERR_ALIGN", -3: 
                 -4: "ASAP_ERR_CUDA", -5: "ASAP_ERR_UNSUPPORTED", -6: "ASAP_ERR_DEVICE"}
 
 EXPORTS = ("asap_init", "asap_score", "asap_select", "asap_merge", "asap_prune_step", "asap_check",
-           "asap_last_error", "asap_launch_count", "asap_free")
+           "asap_last_error", "asap_launch_count", "asap_free", "asap_profile", "asap_profile_read")
 
 
 class AsapError(RuntimeError):
@@ -45,6 +45,10 @@ class CInputs(C.Structure):
 class CParams(C.Structure):
     _fields_ = [("keep_k", C.c_int32), ("lambda_max", C.c_float), ("eps", C.c_float),
                 ("sim_threshold", C.c_float), ("mask_enable", C.c_int32), ("merge_enable", C.c_int32)]
+
+
+class CKernelTime(C.Structure):
+    _fields_ = [("name", C.c_char * 32), ("launches", C.c_uint64), ("total_ms", C.c_double)]
 
 
 class COutputs(C.Structure):
@@ -86,6 +90,10 @@ def load_library() -> C.CDLL:
     lib.asap_last_error.argtypes = [C.c_void_p]
     lib.asap_launch_count.restype = C.c_uint64
     lib.asap_launch_count.argtypes = [C.c_void_p]
+    lib.asap_profile.restype = C.c_int
+    lib.asap_profile.argtypes = [C.c_void_p, C.c_int]
+    lib.asap_profile_read.restype = C.c_int
+    lib.asap_profile_read.argtypes = [C.c_void_p, C.POINTER(CKernelTime), C.c_int]
     lib.asap_free.restype = None
     lib.asap_free.argtypes = [C.c_void_p]
     _lib = lib
@@ -253,6 +261,17 @@ def asap_launch_count(ctx) -> int:
 def asap_last_error(ctx) -> str:
     text = load_library().asap_last_error(ctx)
     return text.decode() if text else ""
+
+
+def asap_profile(ctx, enable: bool) -> None:
+    _raise(ctx, load_library().asap_profile(ctx, int(bool(enable))))
+
+
+def asap_profile_read(ctx) -> dict:
+    """{kernel name: (launches, total_ms)} accumulated since profiling was enabled."""
+    buf = (CKernelTime * 32)()
+    n = load_library().asap_profile_read(ctx, buf, 32)
+    return {buf[i].name.decode(): (int(buf[i].launches), float(buf[i].total_ms)) for i in range(min(n, 32))}
 
 
 def asap_free(ctx) -> None:

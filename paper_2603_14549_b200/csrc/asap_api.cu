@@ -18,6 +18,8 @@ using namespace asap;
 namespace {
 
 char g_init_error[256] = "";
+constexpr int PROF_MAX_EVENTS = 16384;
+constexpr int PROF_MAX_KERNELS = 32;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
@@ -44,6 +46,13 @@ struct asap_ctx {
   EncodeTiledFn encode = nullptr;
   uint64_t launches = 0;
   char err[512] = "";
+  // per-kernel timing (asap_profile): one event before every launch, one at the end of a call
+  bool prof_on = false;
+  cudaEvent_t *prof_ev = nullptr;
+  const char **prof_name = nullptr;   // kernel that starts at the event; nullptr = end of a call
+  int prof_used = 0;
+  asap_kernel_time prof_acc[PROF_MAX_KERNELS];
+  int prof_nacc = 0;
 };
 
 namespace {
@@ -135,11 +144,24 @@ asap_status validate(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
   return ASAP_OK;
 }
 
+// Called right before a kernel is enqueued (name) and once after the last kernel of an entry
+// point (nullptr): with profiling on, drops a timestamp event on the stream.
+void mark(asap_ctx *ctx, const char *name, cudaStream_t st) {
+  if (!ctx->prof_on || ctx->prof_used >= PROF_MAX_EVENTS) return;
+  if (cudaEventRecord(ctx->prof_ev[ctx->prof_used], st) != cudaSuccess) return;
+  ctx->prof_name[ctx->prof_used++] = name;
+}
+
 asap_status after_launch(asap_ctx *ctx, const char *what) {
   ctx->launches += 1;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "%s launch failed: %s", what, cudaGetErrorString(e));
   return ASAP_OK;
+}
+
+asap_status finish(asap_ctx *ctx, asap_status result, cudaStream_t st) {
+  mark(ctx, nullptr, st);
+  return result;
 }
 
 #define ASAP_TRY(expr)                   \
@@ -157,6 +179,7 @@ asap_status launch_prepare(asap_ctx *ctx, const asap_inputs *in, const asap_para
   a.cu_seqlens = in->cu_seqlens; a.vis_start = in->vis_start; a.vis_len = in->vis_len;
   a.text_start = in->text_start; a.text_len = in->text_len; a.rank_start = in->rank_start;
   a.rank_len = in->rank_len; a.desc = ctx->desc; a.out_cu_seqlens = out_cu; a.status = ctx->status;
+  mark(ctx, "prepare", st);
   prepare_kernel<<<1, 256, 0, st>>>(a);
   return after_launch(ctx, "prepare");
 }
@@ -166,6 +189,7 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
   const int D = in->D, B = in->B;
   const int max_chunks = (in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS;
   const int col_blocks = (D + QSUM_COLS - 1) / QSUM_COLS;
+  mark(ctx, "qsum", st);
   qsum_kernel<<<dim3(max_chunks, col_blocks, B), QSUM_THREADS, 0, st>>>(
       static_cast<const __nv_bfloat16 *>(in->q), ctx->desc, D, max_chunks, ctx->qsum_partial, ctx->qbar,
       ctx->cnt_qsum);
@@ -173,6 +197,7 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
 
   const float scale = 1.0f / ((float)in->H * sqrtf((float)in->head_dim));
   const int row_blocks = (in->max_vis + MASS_ROWS - 1) / MASS_ROWS;
+  mark(ctx, "mass_salience", st);
   mass_salience_kernel<<<dim3(row_blocks, B), MASS_THREADS, (size_t)D * sizeof(float), st>>>(
       static_cast<const __nv_bfloat16 *>(in->k), ctx->desc, D, in->max_vis, scale, p->lambda_max, p->eps,
       ctx->qbar, out->mass, out->salience, out->mask_log, ctx->cnt_mass);
@@ -187,12 +212,14 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
   sa.scale_log2 = 1.4426950408889634f / sqrtf((float)in->head_dim);
   sa.mask_log = out->mask_log; sa.partial = ctx->score_partial; sa.rank_score = out->rank_score;
   sa.counters = ctx->cnt_score; sa.status = ctx->status;
+  mark(ctx, "score", st);
   score_kernel<<<dim3(in->H, B), SC_THREADS, SC_SMEM_BYTES, st>>>(map_q, map_k, sa);
   return after_launch(ctx, "score");
 }
 
 asap_status launch_select(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                           const float *rank_score, const asap_outputs *out, cudaStream_t st) {
+  mark(ctx, "select", st);
   select_kernel<<<in->B, SELECT_THREADS, (size_t)in->max_vis * sizeof(uint32_t), st>>>(
       rank_score, ctx->desc, in->max_vis, p->keep_k, out->keep_idx, out->drop_idx, ctx->role);
   return after_launch(ctx, "select");
@@ -212,11 +239,13 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
   const size_t nd_total = (size_t)B * (size_t)(in->max_vis - k);
   if (nd_total > 0) {
     const int blocks = (int)((nd_total + 255) / 256 < 1024 ? (nd_total + 255) / 256 : 1024);
+    mark(ctx, "fill_assign", st);
     fill_assign_kernel<<<blocks, 256, 0, st>>>(out->assign, out->best_sim, nd_total);
     ASAP_TRY(after_launch(ctx, "fill_assign"));
   }
   const bool do_merge = p->merge_enable && in->max_vis > k;
   if (do_merge) {
+    mark(ctx, "norm_gather", st);
     norm_gather_kernel<<<dim3((in->max_vis + 7) / 8, B), NORM_THREADS, 0, st>>>(
         static_cast<const __nv_bfloat16 *>(in->hidden), ctx->desc, D, in->max_vis, k, ctx->role,
         ctx->inv_norm, ctx->kept_rows, ctx->kept_inv);
@@ -237,9 +266,11 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
     sa.n_nt = n_nt; sa.stages = stages; sa.threshold = p->sim_threshold; sa.role = ctx->role;
     sa.inv_norm = ctx->inv_norm; sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
     sa.best_sim = out->best_sim; sa.status = ctx->status;
+    mark(ctx, "sim", st);
     sim_kernel<<<dim3((in->max_vis + 127) / 128, B), SIM_THREADS, smem, st>>>(map_h, map_kept, sa);
     ASAP_TRY(after_launch(ctx, "sim"));
 
+    mark(ctx, "csr", st);
     csr_kernel<<<B, CSR_THREADS, (size_t)k * sizeof(int), st>>>(ctx->desc, in->max_vis, k, out->assign,
                                                                  ctx->seg, ctx->members);
     ASAP_TRY(after_launch(ctx, "csr"));
@@ -247,6 +278,7 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
   const long long bound_ll = (long long)in->total_tokens - (long long)B * (in->min_vis - k);
   int bound = (int)(bound_ll < out->out_rows_capacity ? bound_ll : out->out_rows_capacity);
   int blocks = bound < 148 * 8 ? bound : 148 * 8;
+  mark(ctx, "merge_compact", st);
   merge_compact_kernel<<<blocks, MERGE_THREADS, 0, st>>>(
       static_cast<const __nv_bfloat16 *>(in->hidden), in->pos_ids, ctx->desc, B, D, in->max_vis, k, bound,
       p->eps, do_merge ? 1 : 0, salience, keep_idx, drop_idx, ctx->seg, ctx->members,
@@ -351,7 +383,7 @@ asap_status asap_score(asap_ctx *ctx, const asap_inputs *in, const asap_params *
   ASAP_TRY(validate(ctx, in, p, out, NEED_QK | NEED_SCORE_OUT));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ASAP_TRY(launch_prepare(ctx, in, p, nullptr, 0x7fffffff, st));
-  return launch_score(ctx, in, p, out, st);
+  return finish(ctx, launch_score(ctx, in, p, out, st), st);
 }
 
 asap_status asap_select(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *rank_score,
@@ -360,7 +392,7 @@ asap_status asap_select(asap_ctx *ctx, const asap_inputs *in, const asap_params 
   if (!rank_score) return fail(ctx, ASAP_ERR_INVALID, "null rank_score");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ASAP_TRY(launch_prepare(ctx, in, p, nullptr, 0x7fffffff, st));
-  return launch_select(ctx, in, p, rank_score, out, st);
+  return finish(ctx, launch_select(ctx, in, p, rank_score, out, st), st);
 }
 
 asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *salience,
@@ -371,10 +403,11 @@ asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *
     return fail(ctx, ASAP_ERR_INVALID, "null salience / keep_idx / drop_idx");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
+  mark(ctx, "role_map", st);
   role_map_kernel<<<dim3((in->max_vis + 255) / 256, in->B), 256, 0, st>>>(ctx->desc, in->max_vis, p->keep_k,
                                                                          keep_idx, drop_idx, ctx->role);
   ASAP_TRY(after_launch(ctx, "role_map"));
-  return launch_merge(ctx, in, p, salience, keep_idx, drop_idx, out, st);
+  return finish(ctx, launch_merge(ctx, in, p, salience, keep_idx, drop_idx, out, st), st);
 }
 
 asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const asap_outputs *out,
@@ -384,7 +417,7 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
   ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
   ASAP_TRY(launch_score(ctx, in, p, out, st));
   ASAP_TRY(launch_select(ctx, in, p, out->rank_score, out, st));
-  return launch_merge(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st);
+  return finish(ctx, launch_merge(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st), st);
 }
 
 asap_status asap_check(asap_ctx *ctx, void *stream) {
@@ -404,6 +437,56 @@ asap_status asap_check(asap_ctx *ctx, void *stream) {
               (word & STATUS_SIM_TIMEOUT) ? " a wait timed out in the similarity kernel;" : "");
 }
 
+asap_status asap_profile(asap_ctx *ctx, int enable) {
+  if (!ctx) return fail(nullptr, ASAP_ERR_INVALID, "null context");
+  cudaSetDevice(ctx->device);
+  if (enable && !ctx->prof_ev) {
+    ctx->prof_ev = new (std::nothrow) cudaEvent_t[PROF_MAX_EVENTS];
+    ctx->prof_name = new (std::nothrow) const char *[PROF_MAX_EVENTS];
+    if (!ctx->prof_ev || !ctx->prof_name) return fail(ctx, ASAP_ERR_CUDA, "out of host memory");
+    for (int i = 0; i < PROF_MAX_EVENTS; ++i) {
+      cudaError_t e = cudaEventCreate(&ctx->prof_ev[i]);
+      if (e != cudaSuccess) {
+        for (int j = 0; j < i; ++j) cudaEventDestroy(ctx->prof_ev[j]);
+        delete[] ctx->prof_ev; delete[] ctx->prof_name;
+        ctx->prof_ev = nullptr; ctx->prof_name = nullptr;
+        return fail(ctx, ASAP_ERR_CUDA, "cudaEventCreate: %s", cudaGetErrorString(e));
+      }
+    }
+  }
+  ctx->prof_on = enable != 0;
+  ctx->prof_used = 0;
+  ctx->prof_nacc = 0;
+  return ASAP_OK;
+}
+
+int asap_profile_read(asap_ctx *ctx, asap_kernel_time *out, int capacity) {
+  if (!ctx || !ctx->prof_ev) return 0;
+  cudaSetDevice(ctx->device);
+  if (ctx->prof_used > 0) cudaEventSynchronize(ctx->prof_ev[ctx->prof_used - 1]);
+  for (int i = 0; i + 1 < ctx->prof_used; ++i) {
+    const char *name = ctx->prof_name[i];
+    if (!name) continue;   // gap between two calls
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->prof_ev[i], ctx->prof_ev[i + 1]) != cudaSuccess) continue;
+    int slot = -1;
+    for (int s = 0; s < ctx->prof_nacc; ++s)
+      if (strcmp(ctx->prof_acc[s].name, name) == 0) { slot = s; break; }
+    if (slot < 0) {
+      if (ctx->prof_nacc >= PROF_MAX_KERNELS) continue;
+      slot = ctx->prof_nacc++;
+      memset(&ctx->prof_acc[slot], 0, sizeof(asap_kernel_time));
+      strncpy(ctx->prof_acc[slot].name, name, sizeof(ctx->prof_acc[slot].name) - 1);
+    }
+    ctx->prof_acc[slot].launches += 1;
+    ctx->prof_acc[slot].total_ms += (double)ms;
+  }
+  ctx->prof_used = 0;
+  const int n = ctx->prof_nacc < capacity ? ctx->prof_nacc : capacity;
+  if (out) memcpy(out, ctx->prof_acc, (size_t)(n > 0 ? n : 0) * sizeof(asap_kernel_time));
+  return ctx->prof_nacc;
+}
+
 const char *asap_last_error(const asap_ctx *ctx) { return ctx ? ctx->err : g_init_error; }
 
 uint64_t asap_launch_count(const asap_ctx *ctx) { return ctx ? ctx->launches : 0; }
@@ -411,6 +494,11 @@ uint64_t asap_launch_count(const asap_ctx *ctx) { return ctx ? ctx->launches : 0
 void asap_free(asap_ctx *ctx) {
   if (!ctx) return;
   cudaSetDevice(ctx->device);
+  if (ctx->prof_ev) {
+    for (int i = 0; i < PROF_MAX_EVENTS; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+    delete[] ctx->prof_ev;
+    delete[] ctx->prof_name;
+  }
   cudaFree(ctx->arena);
   delete ctx;
 }
