@@ -148,6 +148,35 @@ asap_status asap_check(asap_ctx *ctx, void *stream);
  * next call on the context.  asap_last_error(NULL) describes a failed asap_init. */
 const char *asap_last_error(const asap_ctx *ctx);
 
+/* Step 3 once more, for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is the same top-k as asap_select, packaged differently.)
+ *
+ * asap_select needs a context, and asap_init takes its scratch with cudaMalloc.  Some callers
+ * have no such moment: a plug-in that runs inside a host application's already-captured or
+ * memory-budgeted region, a real-time loop that may not touch the allocator, a process whose
+ * device memory is handed out entirely by another component.  For them this entry point keeps
+ * the scratch of the selection (the per-sequence descriptors and the kept / dropped role of
+ * every visual token) in a fixed array that is part of the library image: about 1 MiB on every
+ * GPU that loads libasap, held until the process exits.  It calls no cudaMalloc / cudaFree and
+ * no routine that allocates; the caller passes every input and output.
+ *
+ * Limits: B <= 64 and B * max_vis <= 262144 (ASAP_ERR_WORKSPACE beyond that, nothing launched).
+ * Only the fields of `in` that asap_select reads are used: the sizes and the per-sequence
+ * arrays (q, k, hidden, pos_ids may be NULL).  `rank_score`, `keep_idx`, `drop_idx` are as in
+ * asap_select.  `device_status` may be NULL; otherwise it points to one caller-owned 32-bit
+ * word in device memory that is cleared and then receives bit 0 if a per-sequence array entry
+ * failed validation (that sequence's outputs are all -1).
+ *
+ * The call works on the calling thread's current device; `stream` must belong to it.  The
+ * first call on a device looks the array's device address up and raises the kernel's shared
+ * memory limit; make that first call outside any stream capture.  All calls on a device share
+ * the one array, which keeps what the previous call left: the call clears the status word
+ * itself and overwrites the rest, but two calls that overlap on the GPU (different streams,
+ * different threads) race on it.  Errors are reported through asap_last_error(NULL). */
+asap_status asap_select_static(const asap_inputs *in, const asap_params *p, const float *rank_score,
+                               int32_t *keep_idx, int32_t *drop_idx, uint32_t *device_status,
+                               void *stream);
+
 /* Per-kernel device times.  Not part of the method (the paper has no counterpart): a
  * measurement aid.  asap_profile(ctx, 1) makes every later entry point drop one CUDA event on
  * its stream before each kernel and one after its last kernel (the first enabling call creates

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "ASAP_OK", -1: "ASAP_ERR_INVALID", -2: "ASAP_ERR_ALIGN", -3: 
                 -4: "ASAP_ERR_CUDA", -5: "ASAP_ERR_UNSUPPORTED", -6: "ASAP_ERR_DEVICE"}
 
 EXPORTS = ("asap_init", "asap_score", "asap_select", "asap_merge", "asap_prune_step", "asap_check",
-           "asap_last_error", "asap_launch_count", "asap_free", "asap_profile", "asap_profile_read")
+           "asap_last_error", "asap_launch_count", "asap_free", "asap_profile", "asap_profile_read", "asap_select_static")
 
 
 class AsapError(RuntimeError):
@@ -84,6 +84,9 @@ def load_library() -> C.CDLL:
     lib.asap_merge.restype = C.c_int
     lib.asap_merge.argtypes = [C.c_void_p, C.POINTER(CInputs), C.POINTER(CParams), C.c_void_p, C.c_void_p,
                                C.c_void_p, C.POINTER(COutputs), C.c_void_p]
+    lib.asap_select_static.restype = C.c_int
+    lib.asap_select_static.argtypes = [C.POINTER(CInputs), C.POINTER(CParams), C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.c_void_p, C.c_void_p]
     lib.asap_check.restype = C.c_int
     lib.asap_check.argtypes = [C.c_void_p, C.c_void_p]
     lib.asap_last_error.restype = C.c_char_p
@@ -236,6 +239,16 @@ def asap_select(ctx, inp: Inputs, params: Params, rank_score: torch.Tensor, out:
     ci, cp, co = inp.c_struct(), params.c_struct(), out.c_struct()
     _raise(ctx, load_library().asap_select(ctx, C.byref(ci), C.byref(cp), _ptr(rank_score), C.byref(co),
                                            _stream(stream)))
+
+
+def asap_select_static(inp: Inputs, params: Params, rank_score: torch.Tensor, keep_idx: torch.Tensor,
+                       drop_idx: Optional[torch.Tensor], device_status: Optional[torch.Tensor] = None,
+                       stream=None) -> None:
+    """Top-k selection without a context: the library's fixed device array is the scratch, so
+    nothing is allocated.  Works on the current CUDA device; B <= 64, B * max_vis <= 262144."""
+    ci, cp = inp.c_struct(), params.c_struct()
+    _raise(None, load_library().asap_select_static(C.byref(ci), C.byref(cp), _ptr(rank_score), _ptr(keep_idx),
+                                                   _ptr(drop_idx), _ptr(device_status), _stream(stream)))
 
 
 def asap_merge(ctx, inp: Inputs, params: Params, salience: torch.Tensor, keep_idx: torch.Tensor,

@@ -487,6 +487,97 @@ int asap_profile_read(asap_ctx *ctx, asap_kernel_time *out, int capacity) {
   return ctx->prof_nacc;
 }
 
+// ---- asap_select_static: top-k selection with its scratch in a fixed device array -------------
+namespace {
+
+constexpr int STATIC_MAX_B = 64;                 // sequences per call
+constexpr int STATIC_MAX_ROLE = 256 * 1024;      // B * max_vis per call
+
+struct StaticSelectScratch {
+  SampleDesc desc[STATIC_MAX_B];
+  uint32_t status;
+  uint32_t pad[63];
+  int32_t role[STATIC_MAX_ROLE];
+};
+
+// Lives in every GPU that loads the library, from load to exit (about 1 MiB).  On the host this
+// name is only a handle for cudaGetSymbolAddress; it is never passed to a kernel as it stands.
+static __device__ __align__(256) unsigned char g_static_select[sizeof(StaticSelectScratch)];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+StaticSelectScratch *g_static_ptr[STATIC_MAX_DEVICES] = {};   // device address, per device
+
+// First call on a device: look the array's device address up with that device current and raise
+// the selection kernel's shared-memory limit.  Neither call allocates.
+asap_status static_select_setup(int device, StaticSelectScratch **out) {
+  if (device < 0 || device >= STATIC_MAX_DEVICES)
+    return fail(nullptr, ASAP_ERR_UNSUPPORTED, "asap_select_static: device index %d out of range", device);
+  if (!g_static_ptr[device]) {
+    void *ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_select);
+    if (e != cudaSuccess || !ptr)
+      return fail(nullptr, ASAP_ERR_CUDA, "asap_select_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+    e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+    if (e != cudaSuccess)
+      return fail(nullptr, ASAP_ERR_CUDA, "asap_select_static: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    g_static_ptr[device] = static_cast<StaticSelectScratch *>(ptr);
+  }
+  *out = g_static_ptr[device];
+  return ASAP_OK;
+}
+
+}  // namespace
+
+asap_status asap_select_static(const asap_inputs *in, const asap_params *p, const float *rank_score,
+                               int32_t *keep_idx, int32_t *drop_idx, uint32_t *device_status,
+                               void *stream) {
+  g_init_error[0] = 0;
+  if (!in || !p) return fail(nullptr, ASAP_ERR_INVALID, "asap_select_static: null inputs / params struct");
+  if (in->B <= 0 || in->total_tokens <= 0)
+    return fail(nullptr, ASAP_ERR_INVALID, "asap_select_static: B and total_tokens must be positive");
+  if (in->min_vis <= 0 || in->max_vis < in->min_vis || in->max_seq < in->max_vis)
+    return fail(nullptr, ASAP_ERR_INVALID, "asap_select_static: need 0 < min_vis <= max_vis <= max_seq");
+  if (in->max_rank <= 0 || in->max_rank > in->max_seq)
+    return fail(nullptr, ASAP_ERR_INVALID, "asap_select_static: need 0 < max_rank <= max_seq");
+  if (p->keep_k <= 0 || p->keep_k > in->min_vis)
+    return fail(nullptr, ASAP_ERR_INVALID, "asap_select_static: need 0 < keep_k <= min_vis");
+  if (in->max_vis > 57344)
+    return fail(nullptr, ASAP_ERR_UNSUPPORTED, "asap_select_static: max_vis > 57344 is not supported");
+  if (in->B > STATIC_MAX_B || (long long)in->B * in->max_vis > STATIC_MAX_ROLE)
+    return fail(nullptr, ASAP_ERR_WORKSPACE,
+                "asap_select_static: B = %d, B * max_vis = %lld exceed the fixed scratch (B <= %d, B * max_vis <= %d)",
+                in->B, (long long)in->B * in->max_vis, STATIC_MAX_B, STATIC_MAX_ROLE);
+  if (!in->cu_seqlens || !in->vis_start || !in->vis_len || !in->text_start || !in->text_len)
+    return fail(nullptr, ASAP_ERR_INVALID, "asap_select_static: null per-sample array");
+  if ((in->rank_start == nullptr) != (in->rank_len == nullptr))
+    return fail(nullptr, ASAP_ERR_INVALID, "asap_select_static: rank_start and rank_len go together");
+  if (!rank_score || !keep_idx || (!drop_idx && in->max_vis > p->keep_k))
+    return fail(nullptr, ASAP_ERR_INVALID, "asap_select_static: null rank_score / keep_idx / drop_idx");
+  int device = -1;
+  cudaError_t e = cudaGetDevice(&device);
+  if (e != cudaSuccess) return fail(nullptr, ASAP_ERR_CUDA, "asap_select_static: cudaGetDevice: %s", cudaGetErrorString(e));
+  StaticSelectScratch *scr = nullptr;
+  ASAP_TRY(static_select_setup(device, &scr));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the status word is the one thing that must start at zero; everything else is overwritten
+  uint32_t *status = device_status ? device_status : &scr->status;
+  e = cudaMemsetAsync(status, 0, sizeof(uint32_t), st);
+  if (e != cudaSuccess) return fail(nullptr, ASAP_ERR_CUDA, "asap_select_static: cudaMemsetAsync: %s", cudaGetErrorString(e));
+  asap_ctx view;                 // host-side bookkeeping only; owns nothing
+  view.device = device;
+  view.desc = scr->desc;
+  view.role = scr->role;
+  view.status = status;
+  asap_outputs out;
+  memset(&out, 0, sizeof(out));
+  out.keep_idx = keep_idx;
+  out.drop_idx = drop_idx;
+  asap_status r = launch_prepare(&view, in, p, nullptr, 0x7fffffff, st);
+  if (r == ASAP_OK) r = launch_select(&view, in, p, rank_score, &out, st);
+  if (r != ASAP_OK) snprintf(g_init_error, sizeof(g_init_error), "asap_select_static: %s", view.err);
+  return r;
+}
+
 const char *asap_last_error(const asap_ctx *ctx) { return ctx ? ctx->err : g_init_error; }
 
 uint64_t asap_launch_count(const asap_ctx *ctx) { return ctx ? ctx->launches : 0; }
