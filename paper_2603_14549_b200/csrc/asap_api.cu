@@ -39,7 +39,7 @@ struct asap_ctx {
   SampleDesc *desc = nullptr;
   float *qsum_partial = nullptr, *qbar = nullptr, *score_partial = nullptr, *inv_norm = nullptr,
         *kept_inv = nullptr;
-  unsigned int *cnt_qsum = nullptr, *cnt_mass = nullptr, *cnt_score = nullptr;
+  unsigned int *cnt_qsum = nullptr, *cnt_mass = nullptr, *cnt_score = nullptr, *cnt_sim = nullptr;
   int32_t *role = nullptr, *seg = nullptr, *members = nullptr;
   __nv_bfloat16 *kept_rows = nullptr;
   uint32_t *status = nullptr;
@@ -217,33 +217,24 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
   return after_launch(ctx, "score");
 }
 
+// true when a similarity kernel will run for this call (it then writes assign / best_sim of every
+// dropped token itself)
+bool merging(const asap_inputs *in, const asap_params *p) { return p->merge_enable && in->max_vis > p->keep_k; }
+
 asap_status launch_select(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
-                          const float *rank_score, const asap_outputs *out, cudaStream_t st) {
+                          const float *rank_score, const asap_outputs *out, bool with_merge, cudaStream_t st) {
   mark(ctx, "select", st);
   select_kernel<<<in->B, SELECT_THREADS, (size_t)in->max_vis * sizeof(uint32_t), st>>>(
-      rank_score, ctx->desc, in->max_vis, p->keep_k, out->keep_idx, out->drop_idx, ctx->role);
+      rank_score, ctx->desc, in->max_vis, p->keep_k, out->keep_idx, out->drop_idx, ctx->role,
+      with_merge ? out->assign : nullptr, with_merge ? out->best_sim : nullptr, merging(in, p) ? 1 : 0);
   return after_launch(ctx, "select");
-}
-
-__global__ void fill_assign_kernel(int32_t *assign, float *best_sim, size_t n) {
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-    assign[i] = -1;
-    if (best_sim) best_sim[i] = 0.f;
-  }
 }
 
 asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                          const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
                          const asap_outputs *out, cudaStream_t st) {
   const int B = in->B, D = in->D, k = p->keep_k;
-  const size_t nd_total = (size_t)B * (size_t)(in->max_vis - k);
-  if (nd_total > 0) {
-    const int blocks = (int)((nd_total + 255) / 256 < 1024 ? (nd_total + 255) / 256 : 1024);
-    mark(ctx, "fill_assign", st);
-    fill_assign_kernel<<<blocks, 256, 0, st>>>(out->assign, out->best_sim, nd_total);
-    ASAP_TRY(after_launch(ctx, "fill_assign"));
-  }
-  const bool do_merge = p->merge_enable && in->max_vis > k;
+  const bool do_merge = merging(in, p);
   if (do_merge) {
     mark(ctx, "norm_gather", st);
     norm_gather_kernel<<<dim3((in->max_vis + 7) / 8, B), NORM_THREADS, 0, st>>>(
@@ -257,6 +248,8 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
     int stages = (200 * 1024) / stage_bytes;
     if (stages > SIM_MAX_STAGES) stages = SIM_MAX_STAGES;
     const size_t smem = (size_t)stages * stage_bytes + SIM_BOOK_BYTES + 1024;
+    if ((size_t)k * sizeof(int) > (size_t)stages * stage_bytes)
+      return fail(ctx, ASAP_ERR_UNSUPPORTED, "keep_k = %d is too large for the merge path", k);
     CUtensorMap map_h, map_kept;
     if (!make_map(ctx, &map_h, in->hidden, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
         !make_map(ctx, &map_kept, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, (uint32_t)n_tile))
@@ -265,24 +258,29 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
     sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = n_tile;
     sa.n_nt = n_nt; sa.stages = stages; sa.threshold = p->sim_threshold; sa.role = ctx->role;
     sa.inv_norm = ctx->inv_norm; sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
-    sa.best_sim = out->best_sim; sa.status = ctx->status;
+    sa.best_sim = out->best_sim; sa.seg = ctx->seg; sa.members = ctx->members; sa.counters = ctx->cnt_sim;
+    sa.status = ctx->status;
     mark(ctx, "sim", st);
     sim_kernel<<<dim3((in->max_vis + 127) / 128, B), SIM_THREADS, smem, st>>>(map_h, map_kept, sa);
     ASAP_TRY(after_launch(ctx, "sim"));
 
-    mark(ctx, "csr", st);
-    csr_kernel<<<B, CSR_THREADS, (size_t)k * sizeof(int), st>>>(ctx->desc, in->max_vis, k, out->assign,
-                                                                 ctx->seg, ctx->members);
-    ASAP_TRY(after_launch(ctx, "csr"));
   }
-  const long long bound_ll = (long long)in->total_tokens - (long long)B * (in->min_vis - k);
-  int bound = (int)(bound_ll < out->out_rows_capacity ? bound_ll : out->out_rows_capacity);
-  int blocks = bound < 148 * 8 ? bound : 148 * 8;
+  MergeArgs ma;
+  ma.hidden = static_cast<const __nv_bfloat16 *>(in->hidden); ma.pos_ids = in->pos_ids; ma.desc = ctx->desc;
+  ma.D = D; ma.max_vis = in->max_vis; ma.keep_k = k; ma.merge_enable = do_merge ? 1 : 0; ma.eps = p->eps;
+  ma.salience = salience; ma.keep_idx = keep_idx; ma.drop_idx = drop_idx; ma.seg = ctx->seg;
+  ma.members = ctx->members; ma.out_hidden = static_cast<__nv_bfloat16 *>(out->out_hidden);
+  ma.out_pos = out->out_pos; ma.src_row = out->src_row;
+  const int copy_rows = in->max_seq - in->min_vis;   // prefix + suffix rows of the longest sequence, at most
+  const dim3 grid(k + (copy_rows + MERGE_COPY_ROWS - 1) / MERGE_COPY_ROWS, B);
+  const int nv = (D / 8 + MERGE_THREADS - 1) / MERGE_THREADS;
   mark(ctx, "merge_compact", st);
-  merge_compact_kernel<<<blocks, MERGE_THREADS, 0, st>>>(
-      static_cast<const __nv_bfloat16 *>(in->hidden), in->pos_ids, ctx->desc, B, D, in->max_vis, k, bound,
-      p->eps, do_merge ? 1 : 0, salience, keep_idx, drop_idx, ctx->seg, ctx->members,
-      static_cast<__nv_bfloat16 *>(out->out_hidden), out->out_pos, out->src_row);
+  switch (nv) {
+    case 1: merge_compact_kernel<1><<<grid, MERGE_THREADS, 0, st>>>(ma); break;
+    case 2: merge_compact_kernel<2><<<grid, MERGE_THREADS, 0, st>>>(ma); break;
+    case 3: merge_compact_kernel<3><<<grid, MERGE_THREADS, 0, st>>>(ma); break;
+    default: merge_compact_kernel<4><<<grid, MERGE_THREADS, 0, st>>>(ma); break;
+  }
   return after_launch(ctx, "merge_compact");
 }
 
@@ -336,7 +334,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   const size_t o_spart = carve(Hc * T * sizeof(float));
   const size_t o_inv = carve(T * sizeof(float));
   const size_t o_kinv = carve(max_keep_rows * sizeof(float));
-  const size_t o_cnt = carve((Bc * col_blocks + 2 * Bc) * sizeof(unsigned int));
+  const size_t o_cnt = carve((Bc * col_blocks + 3 * Bc) * sizeof(unsigned int));
   const size_t o_role = carve(T * sizeof(int32_t));
   const size_t o_seg = carve((max_keep_rows + Bc) * sizeof(int32_t));
   const size_t o_mem = carve(T * sizeof(int32_t));
@@ -356,18 +354,18 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   ctx->cnt_qsum = reinterpret_cast<unsigned int *>(ctx->arena + o_cnt);
   ctx->cnt_mass = ctx->cnt_qsum + Bc * col_blocks;
   ctx->cnt_score = ctx->cnt_mass + Bc;
+  ctx->cnt_sim = ctx->cnt_score + Bc;
   ctx->role = reinterpret_cast<int32_t *>(ctx->arena + o_role);
   ctx->seg = reinterpret_cast<int32_t *>(ctx->arena + o_seg);
   ctx->members = reinterpret_cast<int32_t *>(ctx->arena + o_mem);
   ctx->kept_rows = reinterpret_cast<__nv_bfloat16 *>(ctx->arena + o_kept);
   ctx->status = reinterpret_cast<uint32_t *>(ctx->arena + o_status);
-  e = cudaMemset(ctx->arena + o_cnt, 0, (Bc * col_blocks + 2 * Bc) * sizeof(unsigned int));
+  e = cudaMemset(ctx->arena + o_cnt, 0, (Bc * col_blocks + 3 * Bc) * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
   // kernels whose dynamic shared memory exceeds the 48 KB default
   if (e == cudaSuccess) e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(csr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     cudaFree(ctx->arena);
@@ -392,7 +390,7 @@ asap_status asap_select(asap_ctx *ctx, const asap_inputs *in, const asap_params 
   if (!rank_score) return fail(ctx, ASAP_ERR_INVALID, "null rank_score");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ASAP_TRY(launch_prepare(ctx, in, p, nullptr, 0x7fffffff, st));
-  return finish(ctx, launch_select(ctx, in, p, rank_score, out, st), st);
+  return finish(ctx, launch_select(ctx, in, p, rank_score, out, false, st), st);
 }
 
 asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *salience,
@@ -405,7 +403,8 @@ asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *
   ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
   mark(ctx, "role_map", st);
   role_map_kernel<<<dim3((in->max_vis + 255) / 256, in->B), 256, 0, st>>>(ctx->desc, in->max_vis, p->keep_k,
-                                                                         keep_idx, drop_idx, ctx->role);
+                                                                         keep_idx, drop_idx, ctx->role, out->assign,
+                                                                         out->best_sim, merging(in, p) ? 1 : 0);
   ASAP_TRY(after_launch(ctx, "role_map"));
   return finish(ctx, launch_merge(ctx, in, p, salience, keep_idx, drop_idx, out, st), st);
 }
@@ -416,7 +415,7 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
   ASAP_TRY(launch_score(ctx, in, p, out, st));
-  ASAP_TRY(launch_select(ctx, in, p, out->rank_score, out, st));
+  ASAP_TRY(launch_select(ctx, in, p, out->rank_score, out, true, st));
   return finish(ctx, launch_merge(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st), st);
 }
 
@@ -573,7 +572,7 @@ asap_status asap_select_static(const asap_inputs *in, const asap_params *p, cons
   out.keep_idx = keep_idx;
   out.drop_idx = drop_idx;
   asap_status r = launch_prepare(&view, in, p, nullptr, 0x7fffffff, st);
-  if (r == ASAP_OK) r = launch_select(&view, in, p, rank_score, &out, st);
+  if (r == ASAP_OK) r = launch_select(&view, in, p, rank_score, &out, false, st);
   if (r != ASAP_OK) snprintf(g_init_error, sizeof(g_init_error), "asap_select_static: %s", view.err);
   return r;
 }

@@ -5,7 +5,7 @@
 //   select         stable radix top-k of the ranking scores           (Fig. 3)
 //   role_map       kept slot / dropped position of every visual token
 //   norm_gather    inverse row norms; kept rows gathered for the similarity GEMM (Sec. 4.2)
-//   csr            dropped tokens grouped by destination slot
+//   csr_block      dropped tokens grouped by destination slot (tail of the similarity kernel)
 //   merge_compact  Eq. 5 and the hand-off of Fig. 3
 #pragma once
 
@@ -95,24 +95,17 @@ qsum_kernel(const __nv_bfloat16 *__restrict__ q, const SampleDesc *__restrict__ 
         reinterpret_cast<const uint4 *>(q + (size_t)(d.row0 + d.v0) * D + col);
     const size_t pitch = (size_t)D / 8;
     int r = r_lo;
-    for (; r + 4 <= r_hi; r += 4) {
-      uint4 v0 = __ldg(base + (size_t)r * pitch);
-      uint4 v1 = __ldg(base + (size_t)(r + 1) * pitch);
-      uint4 v2 = __ldg(base + (size_t)(r + 2) * pitch);
-      uint4 v3 = __ldg(base + (size_t)(r + 3) * pitch);
-      float f[8];
-      unpack8(v0, f);
+    for (; r + 8 <= r_hi; r += 8) {       // eight independent 16-byte loads in flight per thread
+      uint4 v[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] += f[e];
-      unpack8(v1, f);
+      for (int u = 0; u < 8; ++u) v[u] = __ldg(base + (size_t)(r + u) * pitch);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] += f[e];
-      unpack8(v2, f);
+      for (int u = 0; u < 8; ++u) {
+        float f[8];
+        unpack8(v[u], f);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] += f[e];
-      unpack8(v3, f);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] += f[e];
+        for (int e = 0; e < 8; ++e) acc[e] += f[e];
+      }
     }
     for (; r < r_hi; ++r) {
       uint4 v = __ldg(base + (size_t)r * pitch);
@@ -139,6 +132,7 @@ qsum_kernel(const __nv_bfloat16 *__restrict__ q, const SampleDesc *__restrict__ 
   if (!s_last || !active) return;
   __threadfence();
   float tot[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
   for (int c = 0; c < nchunks; ++c) {
     const float4 *src =
         reinterpret_cast<const float4 *>(partial + ((size_t)b * max_chunks + c) * D + col);
@@ -196,18 +190,27 @@ mass_salience_kernel(const __nv_bfloat16 *__restrict__ k, const SampleDesc *__re
     const int j = min(j0 + r, d.nv - 1);   // clamp: duplicates are discarded below
     rowp[r] = reinterpret_cast<const uint4 *>(k + (size_t)(d.row0 + d.v0 + j) * D);
   }
-  for (int v = lane; v < nvec; v += 32) {
-    uint4 kv[MASS_ROWS_PER_WARP];
+  for (int v0 = lane; v0 < nvec; v0 += 64) {   // two vectors x four rows in flight per lane
+    uint4 kv[2][MASS_ROWS_PER_WARP];
 #pragma unroll
-    for (int r = 0; r < MASS_ROWS_PER_WARP; ++r) kv[r] = __ldg(rowp[r] + v);
-    const float4 qa = *reinterpret_cast<const float4 *>(s_q + v * 8);
-    const float4 qb = *reinterpret_cast<const float4 *>(s_q + v * 8 + 4);
+    for (int t = 0; t < 2; ++t)
 #pragma unroll
-    for (int r = 0; r < MASS_ROWS_PER_WARP; ++r) {
-      float f[8];
-      unpack8(kv[r], f);
-      acc[r] += f[0] * qa.x + f[1] * qa.y + f[2] * qa.z + f[3] * qa.w + f[4] * qb.x + f[5] * qb.y +
-                f[6] * qb.z + f[7] * qb.w;
+      for (int r = 0; r < MASS_ROWS_PER_WARP; ++r)
+        if (v0 + 32 * t < nvec) kv[t][r] = __ldg(rowp[r] + v0 + 32 * t);
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const int v = v0 + 32 * t;
+      if (v < nvec) {
+        const float4 qa = *reinterpret_cast<const float4 *>(s_q + v * 8);
+        const float4 qb = *reinterpret_cast<const float4 *>(s_q + v * 8 + 4);
+#pragma unroll
+        for (int r = 0; r < MASS_ROWS_PER_WARP; ++r) {
+          float f[8];
+          unpack8(kv[t][r], f);
+          acc[r] += f[0] * qa.x + f[1] * qa.y + f[2] * qa.z + f[3] * qa.w + f[4] * qb.x + f[5] * qb.y +
+                    f[6] * qb.z + f[7] * qb.w;
+        }
+      }
     }
   }
 #pragma unroll
@@ -300,7 +303,8 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *s_warp /*[32]*/,
 __global__ void __launch_bounds__(SELECT_THREADS)
 select_kernel(const float *__restrict__ rank_score, const SampleDesc *__restrict__ desc,
               int max_vis, int keep_k, int32_t *__restrict__ keep_idx, int32_t *__restrict__ drop_idx,
-              int32_t *__restrict__ role /*[B, max_vis]*/) {
+              int32_t *__restrict__ role /*[B, max_vis]*/, int32_t *__restrict__ assign /*nullable*/,
+              float *__restrict__ best_sim /*nullable*/, int sim_follows) {
   extern __shared__ uint32_t s_key[];   // [max_vis]
   __shared__ int s_hist[256];
   __shared__ int s_scan[33];
@@ -312,6 +316,15 @@ select_kernel(const float *__restrict__ rank_score, const SampleDesc *__restrict
   int32_t *keep_b = keep_idx + (size_t)b * keep_k;
   int32_t *drop_b = drop_idx + (size_t)b * nd_max;
   int32_t *role_b = role + (size_t)b * max_vis;
+  // assign / best_sim entries the similarity kernel will not write: the padding past the last
+  // dropped token, and everything when no similarity kernel follows or the sample is skipped
+  if (assign) {
+    const int first = (d.valid && sim_follows) ? d.nv - keep_k : 0;
+    for (int j = first + threadIdx.x; j < nd_max; j += blockDim.x) {
+      assign[(size_t)b * nd_max + j] = -1;
+      if (best_sim) best_sim[(size_t)b * nd_max + j] = 0.f;
+    }
+  }
   if (!d.valid) {
     for (int j = threadIdx.x; j < keep_k; j += blockDim.x) keep_b[j] = -1;
     for (int j = threadIdx.x; j < nd_max; j += blockDim.x) drop_b[j] = -1;
@@ -408,11 +421,20 @@ select_kernel(const float *__restrict__ rank_score, const SampleDesc *__restrict
 // role map from caller-provided keep / drop lists (entry point asap_merge)
 __global__ void role_map_kernel(const SampleDesc *__restrict__ desc, int max_vis, int keep_k,
                                 const int32_t *__restrict__ keep_idx,
-                                const int32_t *__restrict__ drop_idx, int32_t *__restrict__ role) {
+                                const int32_t *__restrict__ drop_idx, int32_t *__restrict__ role,
+                                int32_t *__restrict__ assign, float *__restrict__ best_sim,
+                                int sim_follows) {
   const int b = blockIdx.y;
   const SampleDesc d = desc[b];
-  if (!d.valid) return;
   const int nd_max = max_vis - keep_k;
+  {
+    const int first = (d.valid && sim_follows) ? d.nv - keep_k : 0;
+    for (int j = first + blockIdx.x * blockDim.x + threadIdx.x; j < nd_max; j += gridDim.x * blockDim.x) {
+      assign[(size_t)b * nd_max + j] = -1;
+      if (best_sim) best_sim[(size_t)b * nd_max + j] = 0.f;
+    }
+  }
+  if (!d.valid) return;
   for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < d.nv; t += gridDim.x * blockDim.x) {
     if (t < keep_k) {
       const int j = keep_idx[(size_t)b * keep_k + t];
@@ -474,32 +496,23 @@ norm_gather_kernel(const __nv_bfloat16 *__restrict__ hidden, const SampleDesc *_
 }
 
 // =======================================================================================
-// csr: group the dropped tokens by destination slot (counting sort, stable in dropped order so
-// the merge adds its members in a fixed order).  One block per sample.
+// csr_block: group the dropped tokens of one sample by destination slot (counting sort, stable
+// in dropped order so the merge adds its members in a fixed order).  Run by one whole block
+// (any size that is a multiple of 32); s_cnt needs keep_k ints, s_scan 33 ints.
 // seg [B, keep_k+1], members [B, max_vis-keep_k] (dropped POSITIONS, ascending inside a slot).
 // =======================================================================================
-constexpr int CSR_THREADS = 1024;
-
-__global__ void __launch_bounds__(CSR_THREADS)
-csr_kernel(const SampleDesc *__restrict__ desc, int max_vis, int keep_k,
-           const int32_t *__restrict__ assign, int32_t *__restrict__ seg,
-           int32_t *__restrict__ members) {
-  extern __shared__ int s_cnt[];   // [keep_k] counts, then cursors
-  __shared__ int s_scan[33];
-  const int b = blockIdx.x;
-  const SampleDesc d = desc[b];
+__device__ __forceinline__ void csr_block(const SampleDesc &d, int b, int max_vis, int keep_k,
+                                          const int32_t *__restrict__ assign,
+                                          int32_t *__restrict__ seg, int32_t *__restrict__ members,
+                                          int *s_cnt, int *s_scan) {
   int32_t *seg_b = seg + (size_t)b * (keep_k + 1);
-  if (!d.valid) {
-    for (int i = threadIdx.x; i <= keep_k; i += blockDim.x) seg_b[i] = 0;
-    return;
-  }
   const int nd_max = max_vis - keep_k, nd = d.nv - keep_k;
   const int32_t *as_b = assign + (size_t)b * nd_max;
   int32_t *mem_b = members + (size_t)b * nd_max;
   for (int i = threadIdx.x; i < keep_k; i += blockDim.x) s_cnt[i] = 0;
   __syncthreads();
   for (int p = threadIdx.x; p < nd; p += blockDim.x) {
-    const int a = as_b[p];
+    const int a = __ldcg(as_b + p);
     if (a >= 0 && a < keep_k) atomicAdd(&s_cnt[a], 1);
   }
   __syncthreads();
@@ -523,7 +536,7 @@ csr_kernel(const SampleDesc *__restrict__ desc, int max_vis, int keep_k,
     const int lane = threadIdx.x;
     for (int base = 0; base < nd; base += 32) {
       const int p = base + lane;
-      int a = (p < nd) ? as_b[p] : -1;
+      int a = (p < nd) ? __ldcg(as_b + p) : -1;
       if (a >= keep_k) a = -1;
       const unsigned peers = __match_any_sync(0xffffffffu, a);
       const int rank = __popc(peers & ((1u << lane) - 1u));
@@ -540,114 +553,169 @@ csr_kernel(const SampleDesc *__restrict__ desc, int max_vis, int keep_k,
 }
 
 // =======================================================================================
-// merge_compact: one block per output row (grid-stride).  Prefix and suffix rows are copied;
-// a kept visual row becomes (s_hat_i h_i + sum_j s_hat_j h_j) / (s_hat_i + sum_j s_hat_j)
-// over the dropped tokens j assigned to it (Eq. 5), accumulated in fp32 in a fixed order and
-// rounded to bf16 once.  A row without members, or whose total weight is <= eps, is copied.
+// merge_compact: grid (keep_k + copy-row groups, B).
+//   blockIdx.x <  keep_k : the block owns one kept visual row.  Its members (the dropped tokens
+//                          assigned to that slot) are first listed in shared memory with their
+//                          weights, then their rows are streamed four at a time and accumulated
+//                          in fp32 in CSR order:  (s_hat_i h_i + sum_j s_hat_j h_j) / (s_hat_i +
+//                          sum_j s_hat_j)   (Eq. 5), rounded to bf16 once.  No members, merging
+//                          off, or total weight <= eps: the row is copied.
+//   blockIdx.x >= keep_k : each warp copies one prefix / suffix row.
+// Every output row also gets its gathered position id and its source row (hand-off of Fig. 3).
 // =======================================================================================
 constexpr int MERGE_THREADS = 256;
-constexpr int MERGE_MAX_VEC = 4;   // 16-byte vectors per thread: D <= 256*4*8 = 8192
+constexpr int MERGE_COPY_ROWS = MERGE_THREADS / 32;   // copy rows per block
+constexpr int MERGE_LIST = 256;                        // members listed per pass
+constexpr int MERGE_BATCH = 4;                         // member rows in flight per thread
 
+struct MergeArgs {
+  const __nv_bfloat16 *hidden;
+  const int32_t *pos_ids;
+  const SampleDesc *desc;
+  int D, max_vis, keep_k, merge_enable;
+  float eps;
+  const float *salience;
+  const int32_t *keep_idx, *drop_idx, *seg, *members;
+  __nv_bfloat16 *out_hidden;
+  int32_t *out_pos, *src_row;
+};
+
+template <int NV>   // 16-byte vectors per thread: D <= NV * 256 * 8
 __global__ void __launch_bounds__(MERGE_THREADS)
-merge_compact_kernel(const __nv_bfloat16 *__restrict__ hidden, const int32_t *__restrict__ pos_ids,
-                     const SampleDesc *__restrict__ desc, int B, int D, int max_vis, int keep_k,
-                     int out_rows_bound, float eps, int merge_enable,
-                     const float *__restrict__ salience, const int32_t *__restrict__ keep_idx,
-                     const int32_t *__restrict__ drop_idx, const int32_t *__restrict__ seg,
-                     const int32_t *__restrict__ members, __nv_bfloat16 *__restrict__ out_hidden,
-                     int32_t *__restrict__ out_pos, int32_t *__restrict__ src_row) {
-  const int nvec = D / 8;
-  const int nd_max = max_vis - keep_k;
-  for (int orow = blockIdx.x; orow < out_rows_bound; orow += gridDim.x) {
-    // sample that owns this output row: last b with out_row0 <= orow
-    int lo = 0, hi = B - 1;
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (desc[mid].out_row0 <= orow) lo = mid; else hi = mid - 1;
-    }
-    const int b = lo;
-    const SampleDesc d = desc[b];
-    const int local = orow - d.out_row0;
-    const int out_len = d.n - d.nv + keep_k;
-    if (!d.valid || local >= out_len) continue;   // past the end of the shortened batch
-    int srow;         // sequence-relative source row
-    int slot = -1;
-    if (local < d.v0) srow = local;
-    else if (local < d.v0 + keep_k) {
-      slot = local - d.v0;
-      srow = d.v0 + min(max(keep_idx[(size_t)b * keep_k + slot], 0), d.nv - 1);
-    } else srow = local - keep_k + d.nv;
+merge_compact_kernel(MergeArgs a) {
+  __shared__ int s_j[MERGE_LIST];
+  __shared__ float s_w[MERGE_LIST];
+  const int b = blockIdx.y;
+  const SampleDesc d = a.desc[b];
+  if (!d.valid) return;
+  const int nvec = a.D / 8;
+  const int k = a.keep_k;
+  if ((int)blockIdx.x >= k) {
+    // ---------------------------------------------------------------- copy rows, one per warp
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int c = ((int)blockIdx.x - k) * MERGE_COPY_ROWS + warp;     // index among prefix + suffix rows
+    if (c >= d.n - d.nv) return;
+    const int srow = c < d.v0 ? c : c + d.nv;
+    const int orow = d.out_row0 + (c < d.v0 ? c : c + k);
     const size_t grow = (size_t)(d.row0 + srow);
-    if (threadIdx.x == 0) {
-      out_pos[orow] = pos_ids[grow];
-      src_row[orow] = (int32_t)grow;
+    if (lane == 0) {
+      a.out_pos[orow] = a.pos_ids[grow];
+      a.src_row[orow] = (int32_t)grow;
     }
-    const uint4 *src = reinterpret_cast<const uint4 *>(hidden + grow * D);
-    uint4 *dst = reinterpret_cast<uint4 *>(out_hidden + (size_t)orow * D);
-    int m_lo = 0, m_hi = 0;
-    if (slot >= 0 && merge_enable) {
-      m_lo = seg[(size_t)b * (keep_k + 1) + slot];
-      m_hi = seg[(size_t)b * (keep_k + 1) + slot + 1];
-    }
-    if (m_hi == m_lo) {
+    const uint4 *src = reinterpret_cast<const uint4 *>(a.hidden + grow * a.D);
+    uint4 *dst = reinterpret_cast<uint4 *>(a.out_hidden + (size_t)orow * a.D);
+    for (int v = lane; v < nvec; v += 32 * 8) {
+      uint4 x[8];
 #pragma unroll
-      for (int u = 0; u < MERGE_MAX_VEC; ++u) {
-        const int v = threadIdx.x + u * MERGE_THREADS;
-        if (v < nvec) dst[v] = __ldg(src + v);
+      for (int u = 0; u < 8; ++u)
+        if (v + 32 * u < nvec) x[u] = __ldg(src + v + 32 * u);
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (v + 32 * u < nvec) dst[v + 32 * u] = x[u];
+    }
+    return;
+  }
+  // ------------------------------------------------------------------ one kept row
+  const int slot = blockIdx.x;
+  const int vi = min(max(a.keep_idx[(size_t)b * k + slot], 0), d.nv - 1);   // visual index
+  const size_t grow = (size_t)(d.row0 + d.v0 + vi);
+  const int orow = d.out_row0 + d.v0 + slot;
+  if (threadIdx.x == 0) {
+    a.out_pos[orow] = a.pos_ids[grow];
+    a.src_row[orow] = (int32_t)grow;
+  }
+  const uint4 *src = reinterpret_cast<const uint4 *>(a.hidden + grow * a.D);
+  uint4 *dst = reinterpret_cast<uint4 *>(a.out_hidden + (size_t)orow * a.D);
+  const int nd_max = a.max_vis - k;
+  int m_lo = 0, m_hi = 0;
+  if (a.merge_enable) {
+    m_lo = min(max(a.seg[(size_t)b * (k + 1) + slot], 0), nd_max);
+    m_hi = min(max(a.seg[(size_t)b * (k + 1) + slot + 1], m_lo), nd_max);
+  }
+  uint4 self[NV];
+#pragma unroll
+  for (int u = 0; u < NV; ++u) {
+    const int v = threadIdx.x + u * MERGE_THREADS;
+    if (v < nvec) self[u] = __ldg(src + v);
+  }
+  if (m_hi <= m_lo) {
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+      const int v = threadIdx.x + u * MERGE_THREADS;
+      if (v < nvec) dst[v] = self[u];
+    }
+    return;
+  }
+  const float *sal_b = a.salience + (size_t)b * a.max_vis;
+  const int32_t *mem_b = a.members + (size_t)b * nd_max;
+  const int32_t *drop_b = a.drop_idx + (size_t)b * nd_max;
+  const float w_self = sal_b[vi];
+  float acc[NV][8];
+#pragma unroll
+  for (int u = 0; u < NV; ++u) {
+    float f[8];
+    unpack8(self[u], f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[u][e] = w_self * f[e];
+  }
+  float den = w_self;
+  const __nv_bfloat16 *vis0 = a.hidden + (size_t)(d.row0 + d.v0) * a.D;
+  for (int base = m_lo; base < m_hi; base += MERGE_LIST) {
+    const int cnt = min(MERGE_LIST, m_hi - base);
+    __syncthreads();                      // the previous list has been consumed
+    if ((int)threadIdx.x < cnt) {
+      const int j = min(max(drop_b[min(max(mem_b[base + threadIdx.x], 0), nd_max - 1)], 0), d.nv - 1);
+      s_j[threadIdx.x] = j;
+      s_w[threadIdx.x] = sal_b[j];
+    }
+    __syncthreads();
+    for (int m0 = 0; m0 < cnt; m0 += MERGE_BATCH) {
+      uint4 x[MERGE_BATCH][NV];
+#pragma unroll
+      for (int t = 0; t < MERGE_BATCH; ++t) {
+        if (m0 + t < cnt) {
+          const uint4 *msrc = reinterpret_cast<const uint4 *>(vis0 + (size_t)s_j[m0 + t] * a.D);
+#pragma unroll
+          for (int u = 0; u < NV; ++u) {
+            const int v = threadIdx.x + u * MERGE_THREADS;
+            if (v < nvec) x[t][u] = __ldg(msrc + v);
+          }
+        }
       }
-      continue;
-    }
-    const float *sal_b = salience + (size_t)b * max_vis;
-    const float w_self = sal_b[srow - d.v0];
-    float acc[MERGE_MAX_VEC][8];
 #pragma unroll
-    for (int u = 0; u < MERGE_MAX_VEC; ++u) {
+      for (int t = 0; t < MERGE_BATCH; ++t) {
+        if (m0 + t < cnt) {
+          const float w = s_w[m0 + t];
+          den += w;
+#pragma unroll
+          for (int u = 0; u < NV; ++u) {
+            float f[8];
+            unpack8(x[t][u], f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[u][e] += w * f[e];
+          }
+        }
+      }
+    }
+  }
+  if (den <= a.eps) {
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+      const int v = threadIdx.x + u * MERGE_THREADS;
+      if (v < nvec) dst[v] = self[u];
+    }
+  } else {
+    const float inv = 1.0f / den;
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
       const int v = threadIdx.x + u * MERGE_THREADS;
       if (v < nvec) {
-        float f[8];
-        unpack8(__ldg(src + v), f);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[u][e] = w_self * f[e];
-      }
-    }
-    float den = w_self;
-    const int32_t *mem_b = members + (size_t)b * nd_max;
-    const int32_t *drop_b = drop_idx + (size_t)b * nd_max;
-    for (int m = m_lo; m < m_hi; ++m) {
-      const int j = min(max(drop_b[mem_b[m]], 0), d.nv - 1);   // visual index of the member
-      const float w = sal_b[j];
-      den += w;
-      const uint4 *msrc = reinterpret_cast<const uint4 *>(hidden + (size_t)(d.row0 + d.v0 + j) * D);
-#pragma unroll
-      for (int u = 0; u < MERGE_MAX_VEC; ++u) {
-        const int v = threadIdx.x + u * MERGE_THREADS;
-        if (v < nvec) {
-          float f[8];
-          unpack8(__ldg(msrc + v), f);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) acc[u][e] += w * f[e];
-        }
-      }
-    }
-    if (den <= eps) {
-#pragma unroll
-      for (int u = 0; u < MERGE_MAX_VEC; ++u) {
-        const int v = threadIdx.x + u * MERGE_THREADS;
-        if (v < nvec) dst[v] = __ldg(src + v);
-      }
-    } else {
-      const float inv = 1.0f / den;
-#pragma unroll
-      for (int u = 0; u < MERGE_MAX_VEC; ++u) {
-        const int v = threadIdx.x + u * MERGE_THREADS;
-        if (v < nvec) {
-          uint4 o;
-          o.x = pack2_rn(acc[u][0] * inv, acc[u][1] * inv);
-          o.y = pack2_rn(acc[u][2] * inv, acc[u][3] * inv);
-          o.z = pack2_rn(acc[u][4] * inv, acc[u][5] * inv);
-          o.w = pack2_rn(acc[u][6] * inv, acc[u][7] * inv);
-          dst[v] = o;
-        }
+        uint4 o;
+        o.x = pack2_rn(acc[u][0] * inv, acc[u][1] * inv);
+        o.y = pack2_rn(acc[u][2] * inv, acc[u][3] * inv);
+        o.z = pack2_rn(acc[u][4] * inv, acc[u][5] * inv);
+        o.w = pack2_rn(acc[u][6] * inv, acc[u][7] * inv);
+        dst[v] = o;
       }
     }
   }

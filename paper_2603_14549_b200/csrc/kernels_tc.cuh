@@ -16,6 +16,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "kernels_stream.cuh"
 
 namespace asap {
 
@@ -388,6 +389,9 @@ struct SimArgs {
   const float *kept_inv;     // [B*keep_k]
   int32_t *assign;           // [B, max_vis-keep_k]
   float *best_sim;           // [B, max_vis-keep_k] or nullptr
+  int32_t *seg;              // [B, keep_k+1]       CSR of assign, built by the last block of a sample
+  int32_t *members;          // [B, max_vis-keep_k]
+  unsigned int *counters;    // [B]
   uint32_t *status;
 };
 
@@ -395,6 +399,8 @@ struct SimBook {
   uint64_t full[SIM_MAX_STAGES], empty[SIM_MAX_STAGES], acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   int abort_flag;
+  int is_last;
+  int scan[33];
 };
 
 __global__ void __launch_bounds__(SIM_THREADS, 1)
@@ -528,6 +534,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         if (a.best_sim) a.best_sim[o] = sim;
       }
     }
+    __threadfence();
   }
   tc_fence_before();
   __syncthreads();
@@ -535,6 +542,20 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     tc_fence_after();
     tmem_dealloc(tmem_base, SIM_TMEM_COLS);
   }
+  // the block that finishes last for this sample groups the dropped tokens by destination
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned int n_mt = (unsigned int)((d.nv + 127) / 128);
+    const unsigned int old = atomicAdd(a.counters + b, 1u);
+    bk->is_last = (old == n_mt - 1u);
+    if (bk->is_last) a.counters[b] = 0u;
+  }
+  __syncthreads();
+  if (!bk->is_last) return;
+  __threadfence();
+  // the tile ring is free: every copy has landed and every MMA that read it has completed
+  csr_block(d, b, a.max_vis, a.keep_k, a.assign, a.seg, a.members, reinterpret_cast<int *>(base_ptr),
+            bk->scan);
 }
 
 }  // namespace asap
