@@ -31,7 +31,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 }  // namespace
 
 struct asap_ctx {
-  int device = 0;
+  int device = 0, num_sms = 1;
   size_t cap_tokens = 0, cap_keep_rows = 0;
   int cap_B = 0, cap_H = 0, cap_D = 0;
   size_t cap_chunks = 0;      // rows of the query-sum partial buffer
@@ -200,7 +200,7 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
   mark(ctx, "mass_salience", st);
   mass_salience_kernel<<<dim3(row_blocks, B), MASS_THREADS, (size_t)D * sizeof(float), st>>>(
       static_cast<const __nv_bfloat16 *>(in->k), ctx->desc, D, in->max_vis, scale, p->lambda_max, p->eps,
-      ctx->qbar, out->mass, out->salience, out->mask_log, ctx->cnt_mass);
+      ctx->qbar, out->mass, out->salience, out->mask_log, out->rank_score, ctx->cnt_mass);
   ASAP_TRY(after_launch(ctx, "mass_salience"));
 
   CUtensorMap map_q, map_k;
@@ -208,13 +208,17 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
       !make_map(ctx, &map_k, in->k, (uint64_t)in->total_tokens, (uint64_t)D, 128))
     return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for q / k");
   ScoreArgs sa;
-  sa.desc = ctx->desc; sa.H = in->H; sa.max_vis = in->max_vis; sa.mask_enable = p->mask_enable ? 1 : 0;
+  sa.desc = ctx->desc; sa.B = B; sa.H = in->H; sa.max_vis = in->max_vis; sa.mask_enable = p->mask_enable ? 1 : 0;
   sa.scale_log2 = 1.4426950408889634f / sqrtf((float)in->head_dim);
-  sa.mask_log = out->mask_log; sa.partial = ctx->score_partial; sa.rank_score = out->rank_score;
-  sa.counters = ctx->cnt_score; sa.status = ctx->status;
+  sa.mask_log = out->mask_log; sa.partial = ctx->score_partial; sa.status = ctx->status;
   mark(ctx, "score", st);
-  score_kernel<<<dim3(in->H, B), SC_THREADS, SC_SMEM_BYTES, st>>>(map_q, map_k, sa);
-  return after_launch(ctx, "score");
+  const int items = B * in->H;
+  score_kernel<<<items < ctx->num_sms ? items : ctx->num_sms, SC_THREADS, SC_SMEM_BYTES, st>>>(map_q, map_k, sa);
+  ASAP_TRY(after_launch(ctx, "score"));
+  mark(ctx, "head_sum", st);
+  head_sum_kernel<<<dim3((in->max_vis + 255) / 256, B), 256, 0, st>>>(ctx->desc, in->H, in->max_vis,
+                                                                      ctx->score_partial, out->rank_score);
+  return after_launch(ctx, "head_sum");
 }
 
 // true when a similarity kernel will run for this call (it then writes assign / best_sim of every
@@ -311,6 +315,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   asap_ctx *ctx = new (std::nothrow) asap_ctx();
   if (!ctx) return fail(nullptr, ASAP_ERR_CUDA, "out of host memory");
   ctx->device = device;
+  ctx->num_sms = prop.multiProcessorCount;
   ctx->cap_tokens = max_total_tokens; ctx->cap_B = max_B; ctx->cap_H = max_H; ctx->cap_D = max_D;
   ctx->cap_keep_rows = max_keep_rows;
   ctx->cap_chunks = max_total_tokens / QSUM_ROWS + 2 * (size_t)max_B;

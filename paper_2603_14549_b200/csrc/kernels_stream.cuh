@@ -160,7 +160,7 @@ mass_salience_kernel(const __nv_bfloat16 *__restrict__ k, const SampleDesc *__re
                      int D, int max_vis, float scale, float lambda_max, float eps,
                      const float *__restrict__ qbar, float *__restrict__ mass,
                      float *__restrict__ salience, float *__restrict__ mask_log,
-                     unsigned int *__restrict__ counters) {
+                     float *__restrict__ rank_score, unsigned int *__restrict__ counters) {
   extern __shared__ float s_q[];   // [D]
   __shared__ float s_red[2 * (MASS_THREADS / 32)];
   __shared__ int s_last;
@@ -170,6 +170,7 @@ mass_salience_kernel(const __nv_bfloat16 *__restrict__ k, const SampleDesc *__re
   if (!d.valid) {
     for (int j = blockIdx.x * MASS_THREADS + threadIdx.x; j < max_vis; j += gridDim.x * MASS_THREADS) {
       mass_b[j] = 0.f; salience[(size_t)b * max_vis + j] = 0.f; mask_log[(size_t)b * max_vis + j] = 0.f;
+      rank_score[(size_t)b * max_vis + j] = 0.f;   // the score kernel skips the sample
     }
     return;
   }

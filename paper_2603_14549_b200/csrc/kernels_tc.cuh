@@ -23,55 +23,60 @@ namespace asap {
 constexpr long long TC_WAIT_LIMIT = 1500000000LL;   // clock cycles, roughly one second
 constexpr float LOG2E_F = 1.4426950408889634f;
 
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// named barriers of the score kernel: 2 = all eight epilogue
+// warps; 3 / 4 = one of its two epilogue groups
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
+__device__ __forceinline__ void group_bar_sync(int group) {
+  asm volatile("bar.sync %0, 128;" ::"r"(3 + group) : "memory");
+}
 
 // =======================================================================================
 // score_kernel
 //
-// One block per (head h, sample b).  For each tile of up to 128 ranking rows:
+// Persistent blocks; a work item is one (sample b, head h) and blocks take items round robin.
+// For each tile of up to 128 ranking rows of the item:
 //   pass 1  D = Q_rows K_tile^T   (M = 128 rows,  N = 128 keys): thread-per-row running
 //           max / sum over all admitted keys  ->  off_i = max_i + log2(sum_i)   (log2 units)
 //   pass 2  D = K_tile Q_rows^T   (M = 128 keys,  N = rows):     thread-per-key sum over rows
 //           of exp2(logit + mask - off_i), i.e. of the Eq. 4 probabilities A[i, j]
-// Pass 2 walks the key tiles in reverse so that the tiles still resident in the shared-memory
-// ring (a direct-mapped cache of key tiles, stage = tile mod stages) are reused without a
-// reload; tiles that were evicted come back from L2.
+// Key tiles stream through a shared-memory ring in one linear order (pass 1 ascending, pass 2
+// over the tiles that hold visual keys, coming back from L2), the query tile is double
+// buffered, and so are the accumulators in tensor memory; the producer and the MMA issuer run
+// ahead across passes, row tiles and items, so the only warps that ever wait are the four
+// epilogue warps' consumers.
 // Additive mask (Eq. 3), logits in log2 units: 0 for key j <= row position p; m_j*log2(e) for
 // j > p when both are in the image span (mask enabled); -inf otherwise.
+// The per-head sums over ranking rows go to `partial`; head_sum_kernel adds them in head order.
 // =======================================================================================
-constexpr int SC_THREADS = 192;
-constexpr int SC_STAGES = 5;
+constexpr int SC_THREADS = 320;          // producer warp, MMA warp, 2 x 4 epilogue warps
+constexpr int SC_EPI_THREADS = 256;
+constexpr int SC_STAGES = 4;
 constexpr int SC_HALF_BYTES = 128 * 128;        // 128 rows x 64 bf16
 constexpr int SC_TILE_BYTES = 2 * SC_HALF_BYTES;
-constexpr int SC_SMEM_MAIN = (1 + SC_STAGES) * SC_TILE_BYTES;
+constexpr int SC_SMEM_MAIN = (2 + SC_STAGES) * SC_TILE_BYTES;
 constexpr int SC_SMEM_BYTES = SC_SMEM_MAIN + 2048 + 1024;   // + bookkeeping + alignment slack
 constexpr uint32_t SC_TMEM_COLS = 256;
 
 struct ScoreArgs {
   const SampleDesc *desc;
-  int H, max_vis, mask_enable;
+  int B, H, max_vis, mask_enable;
   float scale_log2;           // log2(e) / sqrt(head_dim)
   const float *mask_log;      // [B, max_vis]  m_j (natural log)
   float *partial;             // [B, H, max_vis] per-head sums over ranking rows
-  float *rank_score;          // [B, max_vis]
-  unsigned int *counters;     // [B]
   uint32_t *status;
 };
 
 struct ScoreBook {             // bookkeeping block placed after the tiles in shared memory
-  uint64_t full[SC_STAGES], empty[SC_STAGES], q_full, q_empty, acc_full[2], acc_empty[2];
+  uint64_t full[SC_STAGES], empty[SC_STAGES], q_full[2], q_empty[2], acc_full[2], acc_empty[2];
   float off[128];              // per ranking row: max + log2(sum), +inf for rows past the tile
-  float soft[128];             // per key of the current tile: m_j*log2(e) or -inf
-  int sim_res[2][SC_STAGES];   // [role][stage] tile resident in the stage (producer / issuer copies)
-  int sim_fill[2][SC_STAGES];
-  int sim_use[2][SC_STAGES];
+  float soft[2][128];          // per epilogue group, per key of its current tile: m_j*log2(e) or -inf
+  float pm[128], pl[128];      // group 1's running (max, sum) per row at the end of pass 1
   uint32_t tmem_base;
   int abort_flag;
-  int is_last;
 };
 
 struct RowTile {
-  int R0, nrows, n_kt, t_lo, t_hi;
+  int R0, nrows, n_kt, t_lo, t_hi, n_p2;
   bool use_soft;
 };
 
@@ -86,6 +91,7 @@ __device__ __forceinline__ RowTile score_row_tile(const SampleDesc &d, int rt, i
   r.n_kt = jmax / 128 + 1;
   r.t_lo = d.v0 / 128;
   r.t_hi = min((d.v0 + d.nv - 1) / 128, r.n_kt - 1);
+  r.n_p2 = r.t_hi >= r.t_lo ? r.t_hi - r.t_lo + 1 : 0;
   return r;
 }
 
@@ -93,37 +99,27 @@ __global__ void __launch_bounds__(SC_THREADS, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
              ScoreArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  const int h = blockIdx.x, b = blockIdx.y;
-  const SampleDesc d = a.desc[b];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  float *rank_b = a.rank_score + (size_t)b * a.max_vis;
-  if (!d.valid) {
-    if (h == 0)
-      for (int j = threadIdx.x; j < a.max_vis; j += SC_THREADS) rank_b[j] = 0.f;
-    return;
-  }
-  if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SCORE_TIMEOUT) return;
+  const int n_items = a.B * a.H;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_smem = base;
-  const uint32_t k_smem = base + SC_TILE_BYTES;
+  const uint32_t q_smem = base;                          // two query tiles
+  const uint32_t k_smem = base + 2 * SC_TILE_BYTES;      // ring of key tiles
   ScoreBook *bk = reinterpret_cast<ScoreBook *>(base_ptr + SC_SMEM_MAIN);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < SC_STAGES; ++s) {
       mbar_init(smem_u32(&bk->full[s]), 1);
       mbar_init(smem_u32(&bk->empty[s]), 1);
-      for (int r = 0; r < 2; ++r) { bk->sim_res[r][s] = -1; bk->sim_fill[r][s] = 0; bk->sim_use[r][s] = 0; }
     }
-    mbar_init(smem_u32(&bk->q_full), 1);
-    mbar_init(smem_u32(&bk->q_empty), 1);
     for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&bk->q_full[i]), 1);
+      mbar_init(smem_u32(&bk->q_empty[i]), 1);
       mbar_init(smem_u32(&bk->acc_full[i]), 1);
       mbar_init(smem_u32(&bk->acc_empty[i]), 4);
     }
     bk->abort_flag = 0;
-    bk->is_last = 0;
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -135,202 +131,282 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = bk->tmem_base;
   WaitCtx wc{&bk->abort_flag, a.status, STATUS_SCORE_TIMEOUT, TC_WAIT_LIMIT};
-  const int n_rt = (d.nr + 127) / 128;
-  const int grow0 = d.row0;   // packed row of the sequence start
+  if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SCORE_TIMEOUT) bk->abort_flag = 1;   // benign race: same value
+  __syncthreads();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tmap_q);
       tma_prefetch_desc(&tmap_k);
-      int *res = bk->sim_res[0], *fill = bk->sim_fill[0], *use = bk->sim_use[0];
-      for (int rt = 0; rt < n_rt; ++rt) {
-        const RowTile T = score_row_tile(d, rt, a.mask_enable);
-        if (rt > 0) mbar_wait(smem_u32(&bk->q_empty), (rt - 1) & 1, wc);
-        if (!bk->abort_flag) {
-          mbar_expect_tx(smem_u32(&bk->q_full), SC_TILE_BYTES);
-          tma_load_2d(q_smem, &tmap_q, smem_u32(&bk->q_full), h * 128, grow0 + T.R0);
-          tma_load_2d(q_smem + SC_HALF_BYTES, &tmap_q, smem_u32(&bk->q_full), h * 128 + 64, grow0 + T.R0);
-        }
-        const int n_p2 = T.t_hi >= T.t_lo ? T.t_hi - T.t_lo + 1 : 0;
-        for (int u = 0; u < T.n_kt + n_p2; ++u) {
-          const int t = u < T.n_kt ? u : T.t_hi - (u - T.n_kt);
-          const int s = t % SC_STAGES;
-          // The previous use of this stage must have finished, both before a refill and
-          // before a reuse is booked: an mbarrier wait only tells phases apart by parity, so
-          // the producer may never fall two completions behind on a stage.
-          if (use[s] > 0) mbar_wait(smem_u32(&bk->empty[s]), (use[s] - 1) & 1, wc);
-          if (res[s] != t) {
+      int kc = 0, qc = 0;                       // key tiles / query tiles issued so far
+      int k_issued = 0, q_issued = 0;           // copies actually issued (an abort is sticky, so
+                                                // these are prefixes of the two sequences)
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int b = item / a.H, h = item - b * a.H;
+        const SampleDesc d = a.desc[b];
+        if (!d.valid) continue;
+        const int n_rt = (d.nr + 127) / 128;
+        for (int rt = 0; rt < n_rt; ++rt, ++qc) {
+          const RowTile T = score_row_tile(d, rt, a.mask_enable);
+          const int qb = qc & 1;
+          if (qc >= 2) mbar_wait(smem_u32(&bk->q_empty[qb]), ((qc >> 1) - 1) & 1, wc);
+          if (!bk->abort_flag) {
+            const uint32_t dst = q_smem + qb * SC_TILE_BYTES;
+            mbar_expect_tx(smem_u32(&bk->q_full[qb]), SC_TILE_BYTES);
+            tma_load_2d(dst, &tmap_q, smem_u32(&bk->q_full[qb]), h * 128, d.row0 + T.R0);
+            tma_load_2d(dst + SC_HALF_BYTES, &tmap_q, smem_u32(&bk->q_full[qb]), h * 128 + 64, d.row0 + T.R0);
+            q_issued = qc + 1;
+          }
+          for (int u = 0; u < T.n_kt + T.n_p2; ++u, ++kc) {
+            const int t = u < T.n_kt ? u : T.t_hi - (u - T.n_kt);
+            const int s = kc % SC_STAGES;
+            if (kc >= SC_STAGES) mbar_wait(smem_u32(&bk->empty[s]), ((kc / SC_STAGES) - 1) & 1, wc);
             if (!bk->abort_flag) {
               const uint32_t dst = k_smem + s * SC_TILE_BYTES;
               mbar_expect_tx(smem_u32(&bk->full[s]), SC_TILE_BYTES);
-              tma_load_2d(dst, &tmap_k, smem_u32(&bk->full[s]), h * 128, grow0 + t * 128);
-              tma_load_2d(dst + SC_HALF_BYTES, &tmap_k, smem_u32(&bk->full[s]), h * 128 + 64, grow0 + t * 128);
-              fill[s] += 1;
+              tma_load_2d(dst, &tmap_k, smem_u32(&bk->full[s]), h * 128, d.row0 + t * 128);
+              tma_load_2d(dst + SC_HALF_BYTES, &tmap_k, smem_u32(&bk->full[s]), h * 128 + 64, d.row0 + t * 128);
+              k_issued = kc + 1;
             }
-            res[s] = t;
           }
-          use[s] += 1;
         }
       }
       // every copy this thread issued must have landed before the block may leave
-      for (int s = 0; s < SC_STAGES; ++s)
-        if (fill[s] > 0) mbar_wait_drain(smem_u32(&bk->full[s]), (fill[s] - 1) & 1, TC_WAIT_LIMIT);
-      mbar_wait_drain(smem_u32(&bk->q_full), (n_rt - 1) & 1, TC_WAIT_LIMIT);
+      for (int s = 0; s < SC_STAGES; ++s) {
+        const int fills = k_issued > s ? (k_issued - s + SC_STAGES - 1) / SC_STAGES : 0;
+        if (fills > 0) mbar_wait_drain(smem_u32(&bk->full[s]), (fills - 1) & 1, TC_WAIT_LIMIT);
+      }
+      for (int i = 0; i < 2; ++i) {
+        const int fills = q_issued > i ? (q_issued - i + 1) / 2 : 0;
+        if (fills > 0) mbar_wait_drain(smem_u32(&bk->q_full[i]), (fills - 1) & 1, TC_WAIT_LIMIT);
+      }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      int *res = bk->sim_res[1], *fill = bk->sim_fill[1];
-      int g = 0;
-      for (int rt = 0; rt < n_rt; ++rt) {
-        const RowTile T = score_row_tile(d, rt, a.mask_enable);
-        const int n2 = (T.nrows + 15) & ~15;
-        const uint32_t idesc1 = umma_idesc_bf16(128, 128);
-        const uint32_t idesc2 = umma_idesc_bf16(128, n2);
-        mbar_wait(smem_u32(&bk->q_full), rt & 1, wc);
-        const int n_p2 = T.t_hi >= T.t_lo ? T.t_hi - T.t_lo + 1 : 0;
-        for (int u = 0; u < T.n_kt + n_p2; ++u, ++g) {
-          const bool pass1 = u < T.n_kt;
-          const int t = pass1 ? u : T.t_hi - (u - T.n_kt);
-          const int s = t % SC_STAGES, buf = g & 1;
-          if (g >= 2) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((g >> 1) - 1) & 1, wc);
-          if (res[s] != t) {
-            res[s] = t;
-            fill[s] += 1;
-            mbar_wait(smem_u32(&bk->full[s]), (fill[s] - 1) & 1, wc);
-          }
-          tc_fence_after();
-          if (!bk->abort_flag) {
-            const uint32_t ks = k_smem + s * SC_TILE_BYTES;
-            const uint32_t dcol = tmem_base + buf * 128;
+      int kc = 0, qc = 0, g = 0;
+      const uint32_t idesc1 = umma_idesc_bf16(128, 128);
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int b = item / a.H;
+        const SampleDesc d = a.desc[b];
+        if (!d.valid) continue;
+        const int n_rt = (d.nr + 127) / 128;
+        for (int rt = 0; rt < n_rt; ++rt, ++qc) {
+          const RowTile T = score_row_tile(d, rt, a.mask_enable);
+          const int n2 = (T.nrows + 15) & ~15;
+          const uint32_t idesc2 = umma_idesc_bf16(128, n2);
+          const int qb = qc & 1;
+          const uint32_t qs = q_smem + qb * SC_TILE_BYTES;
+          mbar_wait(smem_u32(&bk->q_full[qb]), (qc >> 1) & 1, wc);
+          for (int u = 0; u < T.n_kt + T.n_p2; ++u, ++kc, ++g) {
+            const bool pass1 = u < T.n_kt;
+            const int s = kc % SC_STAGES, buf = g & 1;
+            if (g >= 2) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((g >> 1) - 1) & 1, wc);
+            mbar_wait(smem_u32(&bk->full[s]), (kc / SC_STAGES) & 1, wc);
+            tc_fence_after();
+            if (!bk->abort_flag) {
+              const uint32_t ks = k_smem + s * SC_TILE_BYTES;
+              const uint32_t dcol = tmem_base + buf * 128;
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-              const uint32_t o = (kk >> 2) * SC_HALF_BYTES + (kk & 3) * 32;
-              const uint64_t dq = umma_desc_sw128(q_smem + o), dk = umma_desc_sw128(ks + o);
-              if (pass1) tc_mma_bf16(dcol, dq, dk, idesc1, kk > 0);
-              else       tc_mma_bf16(dcol, dk, dq, idesc2, kk > 0);
+              for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t o = (kk >> 2) * SC_HALF_BYTES + (kk & 3) * 32;
+                const uint64_t dq = umma_desc_sw128(qs + o), dk = umma_desc_sw128(ks + o);
+                if (pass1) tc_mma_bf16(dcol, dq, dk, idesc1, kk > 0);
+                else       tc_mma_bf16(dcol, dk, dq, idesc2, kk > 0);
+              }
+              tc_commit(smem_u32(&bk->empty[s]));
+              tc_commit(smem_u32(&bk->acc_full[buf]));
             }
-            tc_commit(smem_u32(&bk->empty[s]));
-            tc_commit(smem_u32(&bk->acc_full[buf]));
           }
+          if (!bk->abort_flag) tc_commit(smem_u32(&bk->q_empty[qb]));
         }
-        if (!bk->abort_flag) tc_commit(smem_u32(&bk->q_empty));
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (4 warps)
+    // ------------------------------------------------------------------ epilogue (2 groups x 4 warps)
+    // Group w owns accumulator buffer w, i.e. every second operation of the linear sequence; the
+    // two groups share the four sub-partitions, so one group's exponentials overlap the other's
+    // tensor-memory loads.  Warp q of a group reads tensor-memory lanes 32q .. 32q+31.
+    const int group = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int lrow = quarter * 32 + lane;          // tensor-memory lane owned by this thread
-    const int et = (warp - 2) * 32 + lane;         // 0..127 among the epilogue threads
-    float *part = a.partial + ((size_t)b * a.H + h) * a.max_vis;
-    for (int j = et; j < d.nv; j += 128) part[j] = 0.f;
-    epi_bar_sync();
-    const float *mlog = a.mask_log + (size_t)b * a.max_vis;
+    const int et = (warp - 2) * 32 + lane;         // 0..255 among the epilogue threads
     const float scale = a.scale_log2;
-    const int v_end = d.v0 + d.nv;
+    const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16) + group * 128;
+    float *soft = bk->soft[group];
     int g = 0;
-    for (int rt = 0; rt < n_rt; ++rt) {
-      const RowTile T = score_row_tile(d, rt, a.mask_enable);
-      const int n_p2 = T.t_hi >= T.t_lo ? T.t_hi - T.t_lo + 1 : 0;
-      // ---------------- pass 1: thread = ranking row
-      const bool row_ok = lrow < T.nrows;
-      const bool warp_rows = quarter * 32 < T.nrows;
-      const int p_i = T.R0 + lrow;
-      const bool row_vis = T.use_soft && p_i >= d.v0 && p_i < v_end;
-      float m = -INFINITY, l = 0.f;
-      for (int t = 0; t < T.n_kt; ++t, ++g) {
-        const int buf = g & 1, j0 = t * 128;
-        const bool fast = (j0 + 127 <= T.R0);
-        const bool stage_soft = T.use_soft && !fast;
-        if (stage_soft) {
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+      const int b = item / a.H, h = item - b * a.H;
+      const SampleDesc d = a.desc[b];
+      if (!d.valid) continue;
+      const int n_rt = (d.nr + 127) / 128;
+      float *part = a.partial + ((size_t)b * a.H + h) * a.max_vis;
+      const float *mlog = a.mask_log + (size_t)b * a.max_vis;
+      const int v_end = d.v0 + d.nv;
+      {
+        // visual keys beyond the tiles the first row tile visits in pass 2 (possible only when
+        // ranking rows lie before the end of the image span) start from zero; the epilogue-wide
+        // barrier that ends every pass 1 orders these stores before any later add
+        const RowTile T0 = score_row_tile(d, 0, a.mask_enable);
+        const int first = T0.n_p2 > 0 ? max((T0.t_hi + 1) * 128 - d.v0, 0) : 0;
+        for (int j = first + et; j < d.nv; j += SC_EPI_THREADS) part[j] = 0.f;
+      }
+      for (int rt = 0; rt < n_rt; ++rt) {
+        const RowTile T = score_row_tile(d, rt, a.mask_enable);
+        // ---------------- pass 1: thread = ranking row, this group's share of the key tiles
+        const bool row_ok = lrow < T.nrows;
+        const bool warp_rows = quarter * 32 < T.nrows;
+        const int p_i = T.R0 + lrow;
+        const bool row_vis = T.use_soft && p_i >= d.v0 && p_i < v_end;
+        float m = -INFINITY, l = 0.f;
+        for (int t = 0; t < T.n_kt; ++t, ++g) {
+          if ((g & 1) != group) continue;
+          const int j0 = t * 128;
+          const bool fast = (j0 + 127 <= T.R0);
+          const bool stage_soft = T.use_soft && !fast;
+          if (stage_soft) {
+            const int j = j0 + lrow;
+            soft[lrow] = (j >= d.v0 && j < v_end) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
+            group_bar_sync(group);
+          }
+          mbar_wait(smem_u32(&bk->acc_full[group]), (g >> 1) & 1, wc);
+          tc_fence_after();
+          if (warp_rows) {
+#pragma unroll 1
+            for (int c = 0; c < 128; c += 64) {
+              uint32_t r[64];
+              tmem_ld32p(tlane + c, r);
+              tmem_ld32p(tlane + c + 32, r + 32);
+              tmem_wait_ld();
+              if (fast) {
+                // every key admitted, no mask: max on the raw dot products (scale > 0), then
+                // exp2(dot * scale - max) into eight independent partial sums
+                float mx[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) mx[e] = __uint_as_float(r[e]);
+#pragma unroll
+                for (int e = 8; e < 64; ++e) mx[e & 7] = fmaxf(mx[e & 7], __uint_as_float(r[e]));
+                const float cmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                const float m_new = fmaxf(m, cmax * scale);
+                if (row_ok) {
+                  float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                  for (int e = 0; e < 64; ++e) sm[e & 7] += fast_exp2(fmaf(__uint_as_float(r[e]), scale, -m_new));
+                  l = l * fast_exp2(m - m_new) +
+                      (((sm[0] + sm[1]) + (sm[2] + sm[3])) + ((sm[4] + sm[5]) + (sm[6] + sm[7])));
+                  m = m_new;
+                }
+              } else {
+                // tile that crosses a row's own position: selects only, no branches.  `lim` =
+                // last column of this chunk the row may attend to without the soft mask
+                const int lim = p_i - (j0 + c);
+                float mx[8] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                if (!stage_soft) {
+#pragma unroll
+                  for (int e = 0; e < 64; ++e) {
+                    const float x = (e <= lim) ? __uint_as_float(r[e]) * scale : -INFINITY;
+                    r[e] = __float_as_uint(x);
+                    mx[e & 7] = fmaxf(mx[e & 7], x);
+                  }
+                } else {
+#pragma unroll
+                  for (int e = 0; e < 64; ++e) {
+                    const float sv = row_vis ? soft[c + e] : -INFINITY;
+                    const float x = fmaf(__uint_as_float(r[e]), scale, (e <= lim) ? 0.f : sv);
+                    r[e] = __float_as_uint(x);
+                    mx[e & 7] = fmaxf(mx[e & 7], x);
+                  }
+                }
+                const float cmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                const float m_new = fmaxf(m, cmax);
+                if (row_ok && m_new > -INFINITY) {
+                  float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                  for (int e = 0; e < 64; ++e) sm[e & 7] += fast_exp2(__uint_as_float(r[e]) - m_new);
+                  l = l * fast_exp2(m - m_new) +
+                      (((sm[0] + sm[1]) + (sm[2] + sm[3])) + ((sm[4] + sm[5]) + (sm[6] + sm[7])));
+                  m = m_new;
+                }
+              }
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[group]));
+          if (stage_soft) group_bar_sync(group);   // soft[] is rewritten by this group's next masked tile
+        }
+        // the two groups saw disjoint key tiles: merge their (max, sum) per row, then
+        // off_i = max_i + log2(sum_i), so that exp2(x - off_i) = exp2(x - max_i) / sum_i
+        if (group == 1) { bk->pm[lrow] = m; bk->pl[lrow] = l; }
+        epi_bar_sync();
+        if (group == 0) {
+          const float m1 = bk->pm[lrow], l1 = bk->pl[lrow];
+          const float mm = fmaxf(m, m1);
+          float ll = 0.f;
+          if (m > -INFINITY) ll += l * fast_exp2(m - mm);
+          if (m1 > -INFINITY) ll += l1 * fast_exp2(m1 - mm);
+          bk->off[lrow] = row_ok ? (mm + __log2f(ll)) : INFINITY;
+        }
+        epi_bar_sync();
+        // ---------------- pass 2: thread = key, this group's share of the visual key tiles
+        const int n2 = (T.nrows + 15) & ~15;
+        for (int u = 0; u < T.n_p2; ++u, ++g) {
+          if ((g & 1) != group) continue;
+          const int t = T.t_hi - u, j0 = t * 128;
           const int j = j0 + lrow;
-          bk->soft[lrow] = (j >= d.v0 && j < v_end) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
-          epi_bar_sync();
-        }
-        mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 1) & 1, wc);
-        tc_fence_after();
-        if (warp_rows) {
-          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 128;
+          const bool key_ok = j >= d.v0 && j < v_end;
+          const bool fast = (j0 + 127 <= T.R0);
+          const bool warp_keys = (j0 + quarter * 32 + 31 >= d.v0) && (j0 + quarter * 32 < v_end);
+          const float soft_j = (T.use_soft && key_ok) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
+          mbar_wait(smem_u32(&bk->acc_full[group]), (g >> 1) & 1, wc);
+          tc_fence_after();
+          if (warp_keys) {
+            float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            uint32_t r[32];
-            tmem_ld32(taddr + c * 32, r);
-            tmem_wait_ld();
-            float x[32];
-            float cmax = -INFINITY;
-            if (fast) {
+            for (int c = 0; c < n2; c += 32) {
+              uint32_t r[32];
+              const bool full = c + 32 <= n2;       // n2 is a multiple of 16: the last chunk may be half
+              if (full) tmem_ld32p(tlane + c, r);
+              else {
+                tmem_ld16p(tlane + c, r);
 #pragma unroll
-              for (int e = 0; e < 32; ++e) { x[e] = __uint_as_float(r[e]) * scale; cmax = fmaxf(cmax, x[e]); }
-            } else {
+                for (int e = 16; e < 32; ++e) r[e] = 0u;
+              }
+              tmem_wait_ld();
+              // rows past the tile have off = +inf, so their terms vanish
+              if (fast) {
 #pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const int j = j0 + c * 32 + e;
-                float add;
-                if (j <= p_i) add = 0.f;
-                else add = (row_vis && stage_soft) ? bk->soft[c * 32 + e] : -INFINITY;
-                x[e] = __uint_as_float(r[e]) * scale + add;
-                cmax = fmaxf(cmax, x[e]);
+                for (int e = 0; e < 32; ++e) {
+                  const float o = (full || e < 16) ? bk->off[c + e] : INFINITY;
+                  sm[e & 7] += fast_exp2(fmaf(__uint_as_float(r[e]), scale, -o));
+                }
+              } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                  const int p = T.R0 + c + e;
+                  const float o = (full || e < 16) ? bk->off[c + e] : INFINITY;
+                  const float above = (p >= d.v0 && p < v_end) ? soft_j : -INFINITY;
+                  const float add = (j <= p) ? 0.f : above;
+                  sm[e & 7] += fast_exp2(fmaf(__uint_as_float(r[e]), scale, add) - o);
+                }
               }
             }
-            const float m_new = fmaxf(m, cmax);
-            if (row_ok && m_new > -INFINITY) {
-              float sum = 0.f;
-#pragma unroll
-              for (int e = 0; e < 32; ++e) sum += fast_exp2(x[e] - m_new);
-              l = l * fast_exp2(m - m_new) + sum;
-              m = m_new;
+            if (key_ok) {
+              const float sum = ((sm[0] + sm[1]) + (sm[2] + sm[3])) + ((sm[4] + sm[5]) + (sm[6] + sm[7]));
+              // the first row tile initialises the slots it covers; later row tiles add
+              if (rt == 0) part[j - d.v0] = sum;
+              else part[j - d.v0] += sum;
             }
           }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[group]));
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
-        if (stage_soft) epi_bar_sync();
+        epi_bar_sync();   // off[] is rewritten by the next row tile
       }
-      // per-row offset: exp2(x - off) = exp2(x - max) / sum
-      bk->off[lrow] = row_ok ? (m + __log2f(l)) : INFINITY;
-      epi_bar_sync();
-      // ---------------- pass 2: thread = key
-      const int n2 = (T.nrows + 15) & ~15;
-      for (int u = 0; u < n_p2; ++u, ++g) {
-        const int t = T.t_hi - u, buf = g & 1, j0 = t * 128;
-        const int j = j0 + lrow;
-        const bool key_ok = j >= d.v0 && j < v_end;
-        const bool fast = (j0 + 127 <= T.R0);
-        const bool warp_keys = (j0 + quarter * 32 + 31 >= d.v0) && (j0 + quarter * 32 < v_end);
-        const float soft_j = (T.use_soft && key_ok) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
-        mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 1) & 1, wc);
-        tc_fence_after();
-        if (warp_keys) {
-          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 128;
-          float sum = 0.f;
-#pragma unroll 1
-          for (int c = 0; c < n2; c += 16) {
-            uint32_t r[16];
-            tmem_ld16(taddr + c, r);
-            tmem_wait_ld();
-            if (fast) {
-#pragma unroll
-              for (int e = 0; e < 16; ++e) sum += fast_exp2(__uint_as_float(r[e]) * scale - bk->off[c + e]);
-            } else {
-#pragma unroll
-              for (int e = 0; e < 16; ++e) {
-                const int p = T.R0 + c + e;
-                float add;
-                if (j <= p) add = 0.f;
-                else add = (p >= d.v0 && p < v_end) ? soft_j : -INFINITY;
-                sum += fast_exp2(__uint_as_float(r[e]) * scale + add - bk->off[c + e]);
-              }
-            }
-          }
-          if (key_ok) part[j - d.v0] += sum;
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
-      }
-      epi_bar_sync();   // off[] is rewritten by the next row tile
     }
     __threadfence();
   }
@@ -342,26 +418,32 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     tc_fence_after();
     tmem_dealloc(tmem_base, SC_TMEM_COLS);
   }
-  // the block that finishes last for this sample adds the heads in head order
-  if (threadIdx.x == 0) {
-    __threadfence();
-    const unsigned int old = atomicAdd(a.counters + b, 1u);
-    bk->is_last = (old == (unsigned int)(a.H - 1));
-    if (bk->is_last) a.counters[b] = 0u;
-  }
-  __syncthreads();
-  if (!bk->is_last) return;
-  __threadfence();
-  const float inv = 1.0f / ((float)a.H * (float)d.nr);
-  for (int j = threadIdx.x; j < a.max_vis; j += SC_THREADS) {
-    float tot = 0.f;
-    if (j < d.nv) {
-      const float *p = a.partial + (size_t)b * a.H * a.max_vis + j;
-      for (int hh = 0; hh < a.H; ++hh) tot += __ldcg(p + (size_t)hh * a.max_vis);
-      tot *= inv;
+}
+
+// r_j = (1 / (H |R|)) sum_h partial[b, h, j]: the mean over heads and ranking rows of the Eq. 4
+// probabilities, heads added in ascending order.  grid (ceil(max_vis / 256), B).
+__global__ void __launch_bounds__(256)
+head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
+                const float *__restrict__ partial, float *__restrict__ rank_score) {
+  const int b = blockIdx.y;
+  const SampleDesc d = desc[b];
+  const int j = blockIdx.x * 256 + threadIdx.x;
+  if (j >= max_vis) return;
+  float tot = 0.f;
+  if (d.valid && j < d.nv) {
+    const float *p = partial + (size_t)b * H * max_vis + j;
+    int hh = 0;
+    for (; hh + 8 <= H; hh += 8) {
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = __ldcg(p + (size_t)(hh + e) * max_vis);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) tot += v[e];
     }
-    rank_b[j] = tot;
+    for (; hh < H; ++hh) tot += __ldcg(p + (size_t)hh * max_vis);
+    tot *= 1.0f / ((float)H * (float)d.nr);
   }
+  rank_score[(size_t)b * max_vis + j] = tot;
 }
 
 // =======================================================================================
