@@ -55,7 +55,7 @@ constexpr int SC_HALF_BYTES = 128 * 128;        // 128 rows x 64 bf16
 constexpr int SC_TILE_BYTES = 2 * SC_HALF_BYTES;
 constexpr int SC_SMEM_MAIN = (2 + SC_STAGES) * SC_TILE_BYTES;
 constexpr int SC_SMEM_BYTES = SC_SMEM_MAIN + 2048 + 1024;   // + bookkeeping + alignment slack
-constexpr uint32_t SC_TMEM_COLS = 256;
+constexpr uint32_t SC_TMEM_COLS = 512;     // four accumulators of 128 columns
 
 struct ScoreArgs {
   const SampleDesc *desc;
@@ -67,7 +67,7 @@ struct ScoreArgs {
 };
 
 struct ScoreBook {             // bookkeeping block placed after the tiles in shared memory
-  uint64_t full[SC_STAGES], empty[SC_STAGES], q_full[2], q_empty[2], acc_full[2], acc_empty[2];
+  uint64_t full[SC_STAGES], empty[SC_STAGES], q_full[2], q_empty[2], acc_full[4], acc_empty[4];
   float off[128];              // per ranking row: max + log2(sum), +inf for rows past the tile
   float soft[2][128];          // per epilogue group, per key of its current tile: m_j*log2(e) or -inf
   float pm[128], pl[128];      // group 1's running (max, sum) per row at the end of pass 1
@@ -116,6 +116,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&bk->q_full[i]), 1);
       mbar_init(smem_u32(&bk->q_empty[i]), 1);
+    }
+    for (int i = 0; i < 4; ++i) {
       mbar_init(smem_u32(&bk->acc_full[i]), 1);
       mbar_init(smem_u32(&bk->acc_empty[i]), 4);
     }
@@ -201,8 +203,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           mbar_wait(smem_u32(&bk->q_full[qb]), (qc >> 1) & 1, wc);
           for (int u = 0; u < T.n_kt + T.n_p2; ++u, ++kc, ++g) {
             const bool pass1 = u < T.n_kt;
-            const int s = kc % SC_STAGES, buf = g & 1;
-            if (g >= 2) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((g >> 1) - 1) & 1, wc);
+            const int s = kc % SC_STAGES, buf = g & 3;
+            if (g >= 4) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((g >> 2) - 1) & 1, wc);
             mbar_wait(smem_u32(&bk->full[s]), (kc / SC_STAGES) & 1, wc);
             tc_fence_after();
             if (!bk->abort_flag) {
@@ -225,7 +227,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------------ epilogue (2 groups x 4 warps)
-    // Group w owns accumulator buffer w, i.e. every second operation of the linear sequence; the
+    // Group w owns accumulators w and w + 2, i.e. every second operation of the linear sequence
+    // (operation g uses accumulator g mod 4), so the MMA issuer can run two operations ahead; the
     // two groups share the four sub-partitions, so one group's exponentials overlap the other's
     // tensor-memory loads.  Warp q of a group reads tensor-memory lanes 32q .. 32q+31.
     const int group = (warp - 2) >> 2;
@@ -233,7 +236,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     const int lrow = quarter * 32 + lane;          // tensor-memory lane owned by this thread
     const int et = (warp - 2) * 32 + lane;         // 0..255 among the epilogue threads
     const float scale = a.scale_log2;
-    const uint32_t tlane = tmem_base + ((uint32_t)(quarter * 32) << 16) + group * 128;
+    const uint32_t tlane0 = tmem_base + ((uint32_t)(quarter * 32) << 16);
     float *soft = bk->soft[group];
     int g = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
@@ -270,7 +273,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             soft[lrow] = (j >= d.v0 && j < v_end) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
             group_bar_sync(group);
           }
-          mbar_wait(smem_u32(&bk->acc_full[group]), (g >> 1) & 1, wc);
+          const int buf = g & 3;
+          const uint32_t tlane = tlane0 + buf * 128;
+          mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 2) & 1, wc);
           tc_fence_after();
           if (warp_rows) {
 #pragma unroll 1
@@ -335,7 +340,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           }
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[group]));
+          if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
           if (stage_soft) group_bar_sync(group);   // soft[] is rewritten by this group's next masked tile
         }
         // the two groups saw disjoint key tiles: merge their (max, sum) per row, then
@@ -361,7 +366,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           const bool fast = (j0 + 127 <= T.R0);
           const bool warp_keys = (j0 + quarter * 32 + 31 >= d.v0) && (j0 + quarter * 32 < v_end);
           const float soft_j = (T.use_soft && key_ok) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
-          mbar_wait(smem_u32(&bk->acc_full[group]), (g >> 1) & 1, wc);
+          const int buf = g & 3;
+          const uint32_t tlane = tlane0 + buf * 128;
+          mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 2) & 1, wc);
           tc_fence_after();
           if (warp_keys) {
             float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -403,7 +410,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           }
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[group]));
+          if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
         }
         epi_bar_sync();   // off[] is rewritten by the next row tile
       }
