@@ -69,8 +69,8 @@ def algorithmic(batch, keep_k):
     every operand it consumes read once, every result written once (bf16 = 2 bytes)."""
     D = batch.D
     out = {name: {"bytes": 0, "flops": 0} for name in
-           ("qsum", "mass_salience", "score", "select", "norm_gather", "sim", "csr", "merge_compact",
-            "prepare", "fill_assign")}
+           ("qsum", "mass_salience", "score", "head_sum", "select", "kept_gather", "sim", "merge_compact",
+            "prepare", "role_map")}
     for b in range(batch.B):
         n = int(batch.cu_seqlens[b + 1] - batch.cu_seqlens[b])
         nv, tl = int(batch.vis_len[b]), int(batch.text_len[b])
@@ -84,11 +84,11 @@ def algorithmic(batch, keep_k):
         out["score"]["bytes"] += tl * row + (t0 + tl) * row + nv * 4
         out["score"]["flops"] += 2 * tl * (t0 + (tl + 1) // 2) * D
         out["select"]["bytes"] += nv * 4 + nv * 4
-        out["norm_gather"]["bytes"] += nv * row
-        out["norm_gather"]["flops"] += 2 * nv * D
+        out["head_sum"]["bytes"] += batch.H * nv * 4 + nv * 4
+        out["kept_gather"]["bytes"] += 2 * keep_k * row
+        out["kept_gather"]["flops"] += 2 * keep_k * D
         out["sim"]["bytes"] += nv * row
         out["sim"]["flops"] += 2 * (nv - keep_k) * keep_k * D
-        out["csr"]["bytes"] += (nv - keep_k) * 8
         out["merge_compact"]["bytes"] += n * row + (n - nv + keep_k) * row
         out["merge_compact"]["flops"] += 2 * nv * D
     return out

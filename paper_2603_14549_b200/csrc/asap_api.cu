@@ -39,7 +39,10 @@ struct asap_ctx {
   SampleDesc *desc = nullptr;
   float *qsum_partial = nullptr, *qbar = nullptr, *score_partial = nullptr, *inv_norm = nullptr,
         *kept_inv = nullptr;
-  unsigned int *cnt_qsum = nullptr, *cnt_mass = nullptr, *cnt_score = nullptr, *cnt_sim = nullptr;
+  unsigned int *cnt_qsum = nullptr, *cnt_mass = nullptr, *cnt_score = nullptr, *cnt_sim = nullptr,
+               *cnt_tiles = nullptr;
+  float *sim_part = nullptr;        // partial dot products / squared norms of a sliced similarity GEMM
+  size_t sim_part_bytes = 0, cap_tiles = 0;
   int32_t *role = nullptr, *seg = nullptr, *members = nullptr;
   __nv_bfloat16 *kept_rows = nullptr;
   uint32_t *status = nullptr;
@@ -240,19 +243,38 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
   const int B = in->B, D = in->D, k = p->keep_k;
   const bool do_merge = merging(in, p);
   if (do_merge) {
-    mark(ctx, "norm_gather", st);
-    norm_gather_kernel<<<dim3((in->max_vis + 7) / 8, B), NORM_THREADS, 0, st>>>(
-        static_cast<const __nv_bfloat16 *>(in->hidden), ctx->desc, D, in->max_vis, k, ctx->role,
-        ctx->inv_norm, ctx->kept_rows, ctx->kept_inv);
-    ASAP_TRY(after_launch(ctx, "norm_gather"));
+    mark(ctx, "kept_gather", st);
+    kept_gather_kernel<<<dim3((k + GATHER_THREADS / 32 - 1) / (GATHER_THREADS / 32), B), GATHER_THREADS, 0, st>>>(
+        static_cast<const __nv_bfloat16 *>(in->hidden), ctx->desc, D, k, keep_idx, ctx->kept_rows, ctx->kept_inv);
+    ASAP_TRY(after_launch(ctx, "kept_gather"));
 
     const int n_nt = (k + 255) / 256;
     const int n_tile = (((k + n_nt - 1) / n_nt) + 15) & ~15;
-    const int stage_bytes = SIM_A_BYTES + n_tile * 128;
-    int stages = (200 * 1024) / stage_bytes;
+    const int stage_bytes = 2 * (SIM_A_BYTES + n_tile * 128);   // two adjacent 64-column blocks per stage
+    // Small problems leave most SMs without a row tile: slice the hidden dimension over several
+    // blocks (at most 8, a divisor of the number of 128-column steps, scratch permitting), up to
+    // two blocks per SM.
+    const int max_mt = (in->max_vis + 127) / 128;
+    const int n_kb = D / 128;
+    int splits = 1;
+    for (int c = 2; c <= 8; ++c) {
+      if (n_kb % c != 0) continue;
+      if ((long long)max_mt * B * c > 2LL * ctx->num_sms) break;
+      if ((size_t)B * max_mt * c * ((size_t)k + 1) * 128 * sizeof(float) > ctx->sim_part_bytes) break;
+      if ((size_t)B * max_mt > ctx->cap_tiles) break;
+      splits = c;
+    }
+    // a grid between one and two blocks per SM runs as one wave if two blocks fit on an SM:
+    // give each block half of the shared memory and of the tensor memory then
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < 2 * n_tile) tmem_cols <<= 1;
+    const long long ctas = (long long)max_mt * B * splits;
+    const bool two_per_sm = ctas > ctx->num_sms && ctas <= 2LL * ctx->num_sms && tmem_cols <= 256 &&
+                            2 * stage_bytes <= 100 * 1024;
+    int stages = ((two_per_sm ? 100 : 200) * 1024) / stage_bytes;
     if (stages > SIM_MAX_STAGES) stages = SIM_MAX_STAGES;
     const size_t smem = (size_t)stages * stage_bytes + SIM_BOOK_BYTES + 1024;
-    if ((size_t)k * sizeof(int) > (size_t)stages * stage_bytes)
+    if ((size_t)(SIM_THREADS / 32 + 1) * k * sizeof(int) > (size_t)stages * stage_bytes)
       return fail(ctx, ASAP_ERR_UNSUPPORTED, "keep_k = %d is too large for the merge path", k);
     CUtensorMap map_h, map_kept;
     if (!make_map(ctx, &map_h, in->hidden, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
@@ -260,12 +282,15 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
       return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for hidden / kept rows");
     SimArgs sa;
     sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = n_tile;
-    sa.n_nt = n_nt; sa.stages = stages; sa.threshold = p->sim_threshold; sa.role = ctx->role;
-    sa.inv_norm = ctx->inv_norm; sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
+    sa.n_nt = n_nt; sa.stages = stages; sa.splits = splits; sa.max_mt = max_mt; sa.tmem_cols = tmem_cols;
+    sa.threshold = p->sim_threshold;
+    sa.role = ctx->role; sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
     sa.best_sim = out->best_sim; sa.seg = ctx->seg; sa.members = ctx->members; sa.counters = ctx->cnt_sim;
+    sa.tile_counters = ctx->cnt_tiles; sa.part = ctx->sim_part;
+    sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
     sa.status = ctx->status;
     mark(ctx, "sim", st);
-    sim_kernel<<<dim3((in->max_vis + 127) / 128, B), SIM_THREADS, smem, st>>>(map_h, map_kept, sa);
+    sim_kernel<<<dim3(max_mt, B, splits), SIM_THREADS, smem, st>>>(map_h, map_kept, sa);
     ASAP_TRY(after_launch(ctx, "sim"));
 
   }
@@ -344,6 +369,10 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   const size_t o_seg = carve((max_keep_rows + Bc) * sizeof(int32_t));
   const size_t o_mem = carve(T * sizeof(int32_t));
   const size_t o_kept = carve(max_keep_rows * Dc * sizeof(__nv_bfloat16));
+  ctx->cap_tiles = T / 128 + Bc;                       // row tiles of 128 visual rows in any batch that fits
+  ctx->sim_part_bytes = (size_t)32 << 20;
+  const size_t o_tiles = carve(ctx->cap_tiles * sizeof(unsigned int));
+  const size_t o_simpart = carve(ctx->sim_part_bytes);
   const size_t o_status = carve(sizeof(uint32_t));
   e = cudaMalloc(&ctx->arena, off);
   if (e != cudaSuccess) {
@@ -364,8 +393,11 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   ctx->seg = reinterpret_cast<int32_t *>(ctx->arena + o_seg);
   ctx->members = reinterpret_cast<int32_t *>(ctx->arena + o_mem);
   ctx->kept_rows = reinterpret_cast<__nv_bfloat16 *>(ctx->arena + o_kept);
+  ctx->cnt_tiles = reinterpret_cast<unsigned int *>(ctx->arena + o_tiles);
+  ctx->sim_part = reinterpret_cast<float *>(ctx->arena + o_simpart);
   ctx->status = reinterpret_cast<uint32_t *>(ctx->arena + o_status);
   e = cudaMemset(ctx->arena + o_cnt, 0, (Bc * col_blocks + 3 * Bc) * sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMemset(ctx->arena + o_tiles, 0, ctx->cap_tiles * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
   // kernels whose dynamic shared memory exceeds the 48 KB default
   if (e == cudaSuccess) e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_BYTES);

@@ -4,7 +4,7 @@
 //   mass_salience  s_j, then s_hat_j and m_j                          (Eq. 1, Eq. 2, Eq. 3)
 //   select         stable radix top-k of the ranking scores           (Fig. 3)
 //   role_map       kept slot / dropped position of every visual token
-//   norm_gather    inverse row norms; kept rows gathered for the similarity GEMM (Sec. 4.2)
+//   kept_gather    kept rows gathered for the similarity GEMM, with their inverse norms (Sec. 4.2)
 //   csr_block      dropped tokens grouped by destination slot (tail of the similarity kernel)
 //   merge_compact  Eq. 5 and the hand-off of Fig. 3
 #pragma once
@@ -449,57 +449,56 @@ __global__ void role_map_kernel(const SampleDesc *__restrict__ desc, int max_vis
 }
 
 // =======================================================================================
-// norm_gather: one warp per visual row.  inv_norm = 1/||h|| (0 if ||h|| < 1e-12, which makes
-// every similarity of that row 0); kept rows are also copied to their slot of the dense
-// [B*keep_k, D] operand of the similarity GEMM together with their inverse norm.
+// kept_gather: one warp per kept slot.  The kept row is copied to its slot of the dense
+// [B*keep_k, D] operand of the similarity GEMM and its inverse norm 1/||h|| is stored (0 if
+// ||h|| < 1e-12, which makes every similarity to that slot 0)   (Sec. 4.2).
 // =======================================================================================
-constexpr int NORM_THREADS = 256;
+constexpr int GATHER_THREADS = 256;
 
-__global__ void __launch_bounds__(NORM_THREADS)
-norm_gather_kernel(const __nv_bfloat16 *__restrict__ hidden, const SampleDesc *__restrict__ desc,
-                   int D, int max_vis, int keep_k, const int32_t *__restrict__ role,
-                   float *__restrict__ inv_norm /*[B, max_vis]*/,
+__global__ void __launch_bounds__(GATHER_THREADS)
+kept_gather_kernel(const __nv_bfloat16 *__restrict__ hidden, const SampleDesc *__restrict__ desc,
+                   int D, int keep_k, const int32_t *__restrict__ keep_idx,
                    __nv_bfloat16 *__restrict__ kept_rows /*[B*keep_k, D]*/,
                    float *__restrict__ kept_inv /*[B*keep_k]*/) {
   const int b = blockIdx.y;
   const SampleDesc d = desc[b];
   if (!d.valid) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int j = blockIdx.x * (NORM_THREADS / 32) + warp;
-  if (j >= d.nv) return;
-  const int slot = role[(size_t)b * max_vis + j];
+  const int slot = blockIdx.x * (GATHER_THREADS / 32) + warp;
+  if (slot >= keep_k) return;
+  const int j = min(max(keep_idx[(size_t)b * keep_k + slot], 0), d.nv - 1);
   const uint4 *src = reinterpret_cast<const uint4 *>(hidden + (size_t)(d.row0 + d.v0 + j) * D);
-  uint4 *dst = slot >= 0 ? reinterpret_cast<uint4 *>(kept_rows + ((size_t)b * keep_k + slot) * D) : nullptr;
+  uint4 *dst = reinterpret_cast<uint4 *>(kept_rows + ((size_t)b * keep_k + slot) * D);
   const int nvec = D / 8;
   float ss = 0.f;
-  for (int v = lane; v < nvec; v += 128) {
-    uint4 x[4];
+  for (int v = lane; v < nvec; v += 256) {
+    uint4 x[8];
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < 8; ++u)
       if (v + 32 * u < nvec) x[u] = __ldg(src + v + 32 * u);
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < 8; ++u)
       if (v + 32 * u < nvec) {
         float f[8];
         unpack8(x[u], f);
 #pragma unroll
         for (int e = 0; e < 8; ++e) ss += f[e] * f[e];
-        if (dst) dst[v + 32 * u] = x[u];
+        dst[v + 32 * u] = x[u];
       }
   }
   ss = warp_sum(ss);
   if (lane == 0) {
     const float nrm = sqrtf(ss);
-    const float inv = nrm >= 1e-12f ? 1.0f / nrm : 0.f;
-    inv_norm[(size_t)b * max_vis + j] = inv;
-    if (slot >= 0) kept_inv[(size_t)b * keep_k + slot] = inv;
+    kept_inv[(size_t)b * keep_k + slot] = nrm >= 1e-12f ? 1.0f / nrm : 0.f;
   }
 }
 
 // =======================================================================================
 // csr_block: group the dropped tokens of one sample by destination slot (counting sort, stable
-// in dropped order so the merge adds its members in a fixed order).  Run by one whole block
-// (any size that is a multiple of 32); s_cnt needs keep_k ints, s_scan 33 ints.
+// in dropped order so the merge adds its members in a fixed order).  Run by one whole block of
+// W <= 8 warps: warp w owns the w-th contiguous chunk of dropped positions, counts its chunk
+// into its own histogram, and after a scan over (slot, warp) writes its chunk's positions behind
+// those of the warps before it.  s_cnt needs (W + 1) * keep_k ints, s_scan 33 ints.
 // seg [B, keep_k+1], members [B, max_vis-keep_k] (dropped POSITIONS, ascending inside a slot).
 // =======================================================================================
 __device__ __forceinline__ void csr_block(const SampleDesc &d, int b, int max_vis, int keep_k,
@@ -510,46 +509,59 @@ __device__ __forceinline__ void csr_block(const SampleDesc &d, int b, int max_vi
   const int nd_max = max_vis - keep_k, nd = d.nv - keep_k;
   const int32_t *as_b = assign + (size_t)b * nd_max;
   int32_t *mem_b = members + (size_t)b * nd_max;
-  for (int i = threadIdx.x; i < keep_k; i += blockDim.x) s_cnt[i] = 0;
+  const int W = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk = (((nd + W - 1) / W) + 31) & ~31;        // positions per warp, a multiple of 32
+  int *hist = s_cnt;                                         // [W][keep_k]
+  int *tot = s_cnt + W * keep_k;                             // [keep_k] members per slot
+  for (int i = threadIdx.x; i < (W + 1) * keep_k; i += blockDim.x) s_cnt[i] = 0;
   __syncthreads();
-  for (int p = threadIdx.x; p < nd; p += blockDim.x) {
+  const int p_lo = min(nd, warp * chunk), p_hi = min(nd, p_lo + chunk);
+  for (int p = p_lo + lane; p < p_hi; p += 32) {
     const int a = __ldcg(as_b + p);
-    if (a >= 0 && a < keep_k) atomicAdd(&s_cnt[a], 1);
+    if (a >= 0 && a < keep_k) atomicAdd(&hist[warp * keep_k + a], 1);
+  }
+  __syncthreads();
+  // per slot: turn the per-warp counts into per-warp offsets inside the slot, and total them
+  for (int i = threadIdx.x; i < keep_k; i += blockDim.x) {
+    int run = 0;
+    for (int w = 0; w < W; ++w) {
+      const int c = hist[w * keep_k + i];
+      hist[w * keep_k + i] = run;
+      run += c;
+    }
+    tot[i] = run;
   }
   __syncthreads();
   // exclusive scan over slots; thread t owns a contiguous range of slots
   const int per = (keep_k + blockDim.x - 1) / blockDim.x;
   const int lo = min(keep_k, (int)threadIdx.x * per), hi = min(keep_k, lo + per);
   int mine = 0;
-  for (int i = lo; i < hi; ++i) mine += s_cnt[i];
-  int tot;
-  int run = block_exclusive_scan(mine, s_scan, tot);
+  for (int i = lo; i < hi; ++i) mine += tot[i];
+  int total;
+  int run = block_exclusive_scan(mine, s_scan, total);
   for (int i = lo; i < hi; ++i) {
-    const int c = s_cnt[i];
+    const int c = tot[i];
     seg_b[i] = run;
-    s_cnt[i] = run;      // becomes the slot's write cursor
+    tot[i] = run;        // becomes the slot's base
     run += c;
   }
-  if (threadIdx.x == 0) seg_b[keep_k] = tot;
+  if (threadIdx.x == 0) seg_b[keep_k] = total;
   __syncthreads();
-  // stable fill by one warp, 32 dropped positions at a time in ascending order
-  if (threadIdx.x < 32) {
-    const int lane = threadIdx.x;
-    for (int base = 0; base < nd; base += 32) {
-      const int p = base + lane;
-      int a = (p < nd) ? __ldcg(as_b + p) : -1;
-      if (a >= keep_k) a = -1;
-      const unsigned peers = __match_any_sync(0xffffffffu, a);
-      const int rank = __popc(peers & ((1u << lane) - 1u));
-      int cur = 0;
-      if (a >= 0) cur = s_cnt[a];
-      __syncwarp();
-      if (a >= 0) {
-        mem_b[cur + rank] = p;
-        if (rank == 0) s_cnt[a] = cur + __popc(peers);
-      }
-      __syncwarp();
+  // stable fill: every warp walks its chunk 32 positions at a time in ascending order
+  for (int base = p_lo; base < p_hi; base += 32) {
+    const int p = base + lane;
+    int a = (p < p_hi) ? __ldcg(as_b + p) : -1;
+    if (a >= keep_k) a = -1;
+    const unsigned peers = __match_any_sync(0xffffffffu, a);
+    const int rank = __popc(peers & ((1u << lane) - 1u));
+    int cur = 0;
+    if (a >= 0) cur = hist[warp * keep_k + a];
+    __syncwarp();
+    if (a >= 0) {
+      mem_b[tot[a] + cur + rank] = p;
+      if (rank == 0) hist[warp * keep_k + a] = cur + __popc(peers);
     }
+    __syncwarp();
   }
 }
 

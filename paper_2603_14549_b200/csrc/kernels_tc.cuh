@@ -456,31 +456,42 @@ head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
 // =======================================================================================
 // sim_kernel
 //
-// One block per (128 visual rows, sample).  D = V_tile Kept^T with M = 128 visual rows,
-// N = n_tile kept slots per accumulator, K = the hidden size in steps of 64.  The epilogue
-// scales column s by 1/||kept_s||, keeps the running maximum and the first slot attaining it,
-// and finally writes, for rows that were dropped, the slot (or -1 if the cosine similarity is
-// not above the threshold) and the similarity.  Rows that were kept, or lie past the image
-// span, are computed but not written.
+// One block per (128 visual rows, sample, slice of the hidden dimension).  D = V_tile Kept^T
+// with M = 128 visual rows, N = n_tile kept slots per accumulator, K = this block's slice of
+// the hidden size in steps of 64.  While the first accumulator is being built the epilogue
+// warps also read every row tile from shared memory and add up the squares (the row norms of
+// Sec. 4.2's cosine similarity), so the visual rows are read from memory once.
+//   one slice:      the epilogue scales column s by 1/||kept_s||, keeps the running maximum
+//                   and the first slot attaining it, and writes, for rows that were dropped,
+//                   the slot (or -1 if the cosine similarity is not above the threshold) and
+//                   the similarity.
+//   several slices: (small problems, to fill the machine) every block stores its partial dot
+//                   products and partial squared norms; the block that finishes last for the
+//                   row tile adds the slices in slice order and does the same epilogue.
+// Rows that were kept, or lie past the image span, are computed but not written.
+// The block that finishes a sample's last row tile groups the dropped tokens by destination.
 // =======================================================================================
 constexpr int SIM_THREADS = 192;
 constexpr int SIM_A_BYTES = 128 * 128;           // 128 rows x 64 bf16
-constexpr int SIM_BOOK_BYTES = 1024;
+constexpr int SIM_BOOK_BYTES = 2048;
 constexpr uint32_t SIM_TMEM_COLS = 512;
 constexpr int SIM_MAX_STAGES = 8;
 
 struct SimArgs {
   const SampleDesc *desc;
-  int D, max_vis, keep_k, n_tile, n_nt, stages;
+  int D, max_vis, keep_k, n_tile, n_nt, stages, splits, max_mt;
+  uint32_t tmem_cols;        // power of two >= 2 * n_tile: two accumulators
   float threshold;
   const int32_t *role;       // [B, max_vis]
-  const float *inv_norm;     // [B, max_vis]
-  const float *kept_inv;     // [B*keep_k]
+  const float *kept_inv;     // [B*keep_k]   1/||kept row||, 0 for a zero row
   int32_t *assign;           // [B, max_vis-keep_k]
   float *best_sim;           // [B, max_vis-keep_k] or nullptr
   int32_t *seg;              // [B, keep_k+1]       CSR of assign, built by the last block of a sample
   int32_t *members;          // [B, max_vis-keep_k]
-  unsigned int *counters;    // [B]
+  unsigned int *counters;    // [B]            finished row tiles per sample
+  unsigned int *tile_counters;  // [B, max_mt] finished slices per row tile
+  float *part;               // [B, max_mt, splits, keep_k, 128] partial dot products (several slices only)
+  float *ss_part;            // [B, max_mt, splits, 128]         partial squared norms
   uint32_t *status;
 };
 
@@ -492,11 +503,15 @@ struct SimBook {
   int scan[33];
 };
 
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t n) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n) : "memory");
+}
+
 __global__ void __launch_bounds__(SIM_THREADS, 1)
 sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_kept,
            SimArgs a) {
   extern __shared__ uint8_t smem_raw[];
-  const int mt = blockIdx.x, b = blockIdx.y;
+  const int mt = blockIdx.x, b = blockIdx.y, z = blockIdx.z;
   const SampleDesc d = a.desc[b];
   if (!d.valid || mt * 128 >= d.nv) return;
   if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SIM_TIMEOUT) return;
@@ -504,24 +519,27 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  // a stage holds two adjacent 64-column blocks (256 contiguous bytes of every row):
+  // [ rows, block 0 | rows, block 1 | kept, block 0 | kept, block 1 ]
   const int b_bytes = a.n_tile * 128;
-  const int stage_bytes = SIM_A_BYTES + b_bytes;
+  const int stage_bytes = 2 * (SIM_A_BYTES + b_bytes);
   SimBook *bk = reinterpret_cast<SimBook *>(base_ptr + (size_t)a.stages * stage_bytes);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.stages; ++s) {
       mbar_init(smem_u32(&bk->full[s]), 1);
-      mbar_init(smem_u32(&bk->empty[s]), 1);
+      mbar_init(smem_u32(&bk->empty[s]), 5);      // the MMAs that read the stage + four epilogue warps
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&bk->acc_full[i]), 1);
       mbar_init(smem_u32(&bk->acc_empty[i]), 4);
     }
     bk->abort_flag = 0;
+    bk->is_last = 0;
     fence_barrier_init();
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&bk->tmem_base), SIM_TMEM_COLS);
+    tmem_alloc(smem_u32(&bk->tmem_base), a.tmem_cols);
     tmem_relinquish();
     tc_fence_before();
   }
@@ -529,7 +547,8 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   tc_fence_after();
   const uint32_t tmem_base = bk->tmem_base;
   WaitCtx wc{&bk->abort_flag, a.status, STATUS_SIM_TIMEOUT, TC_WAIT_LIMIT};
-  const int n_kb = a.D / 64;
+  const int n_kb = (a.D / 128) / a.splits;         // 128-column steps of this slice
+  const int kb0 = z * n_kb;
   const int total_it = a.n_nt * n_kb;
 
   if (warp == 0) {
@@ -538,20 +557,25 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       tma_prefetch_desc(&tmap_kept);
       const int row_a = d.row0 + d.v0 + mt * 128;
       const int row_b = b * a.keep_k;
+      const int rot = (mt * 5 + b * 3) % n_kb;
       int issued = 0;
       for (int it = 0; it < total_it; ++it) {
-        const int s = it % a.stages, nt = it / n_kb, kb = it - nt * n_kb;
+        // every block walks its k-blocks from a different starting point, so that at any moment
+        // the blocks read different 128-byte columns of the rows and spread over the memory channels
+        const int s = it % a.stages, nt = it / n_kb, kb = kb0 + (it - nt * n_kb + rot) % n_kb;
         if (it >= a.stages) mbar_wait(smem_u32(&bk->empty[s]), ((it / a.stages) - 1) & 1, wc);
         if (bk->abort_flag) break;
         const uint32_t dst = base + s * stage_bytes;
         mbar_expect_tx(smem_u32(&bk->full[s]), stage_bytes);
-        tma_load_2d(dst, &tmap_h, smem_u32(&bk->full[s]), kb * 64, row_a);
-        tma_load_2d(dst + SIM_A_BYTES, &tmap_kept, smem_u32(&bk->full[s]), kb * 64, row_b + nt * a.n_tile);
+        tma_load_2d(dst, &tmap_h, smem_u32(&bk->full[s]), kb * 128, row_a);
+        tma_load_2d(dst + SIM_A_BYTES, &tmap_h, smem_u32(&bk->full[s]), kb * 128 + 64, row_a);
+        tma_load_2d(dst + 2 * SIM_A_BYTES, &tmap_kept, smem_u32(&bk->full[s]), kb * 128, row_b + nt * a.n_tile);
+        tma_load_2d(dst + 2 * SIM_A_BYTES + b_bytes, &tmap_kept, smem_u32(&bk->full[s]), kb * 128 + 64,
+                    row_b + nt * a.n_tile);
         issued = it + 1;
       }
       // drain: the last fill of every stage must have landed before the block leaves
       for (int s = 0; s < a.stages; ++s) {
-        // last iteration index < issued that maps to stage s
         if (issued > s) {
           const int last = ((issued - 1 - s) / a.stages) * a.stages + s;
           mbar_wait_drain(smem_u32(&bk->full[s]), (last / a.stages) & 1, TC_WAIT_LIMIT);
@@ -565,18 +589,21 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       for (int nt = 0; nt < a.n_nt; ++nt) {
         const int buf = nt & 1;
         if (nt >= 2) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((nt >> 1) - 1) & 1, wc);
-        const uint32_t dcol = tmem_base + buf * 256;
+        const uint32_t dcol = tmem_base + buf * (a.tmem_cols >> 1);
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const int s = it % a.stages;
           mbar_wait(smem_u32(&bk->full[s]), (it / a.stages) & 1, wc);
           tc_fence_after();
           if (!bk->abort_flag) {
-            const uint32_t sa = base + s * stage_bytes, sb = sa + SIM_A_BYTES;
+            const uint32_t sa = base + s * stage_bytes, sb = sa + 2 * SIM_A_BYTES;
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              tc_mma_bf16(dcol, umma_desc_sw128(sa + kk * 32), umma_desc_sw128(sb + kk * 32), idesc,
+            for (int kk = 0; kk < 8; ++kk)
+              tc_mma_bf16(dcol, umma_desc_sw128(sa + (kk >> 2) * SIM_A_BYTES + (kk & 3) * 32),
+                          umma_desc_sw128(sb + (kk >> 2) * b_bytes + (kk & 3) * 32), idesc,
                           (kb > 0 || kk > 0) ? 1u : 0u);
             tc_commit(smem_u32(&bk->empty[s]));
+            // after the first accumulator the epilogue warps no longer read the stages
+            if (nt > 0) mbar_arrive_n(smem_u32(&bk->empty[s]), 4);
           }
         }
         if (!bk->abort_flag) tc_commit(smem_u32(&bk->acc_full[buf]));
@@ -584,15 +611,48 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     }
   } else {
     const int quarter = warp & 3;
-    const int v = mt * 128 + quarter * 32 + lane;       // visual index of this thread's row
+    const int lrow = quarter * 32 + lane;
+    const int v = mt * 128 + lrow;                       // visual index of this thread's row
     const float *kinv = a.kept_inv + (size_t)b * a.keep_k;
+    // ---- squared norm of this thread's row, from the row tiles of the first accumulator's pass.
+    // Row r of a tile is 128 bytes; its 16-byte chunk c sits at chunk position c ^ (r & 7).
+    float ssq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int it = 0; it < n_kb; ++it) {
+      const int s = it % a.stages;
+      mbar_wait(smem_u32(&bk->full[s]), (it / a.stages) & 1, wc);
+      if (!bk->abort_flag) {
+#pragma unroll
+        for (int hb = 0; hb < 2; ++hb) {
+          const uint4 *row = reinterpret_cast<const uint4 *>(base_ptr + (size_t)s * stage_bytes +
+                                                             hb * SIM_A_BYTES + lrow * 128);
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint4 x = row[c ^ (lrow & 7)];
+            float f[8];
+            unpack8(x, f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ssq[c] = fmaf(f[e], f[e], ssq[c]);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bk->empty[s]));
+    }
+    const float ss = ((ssq[0] + ssq[1]) + (ssq[2] + ssq[3])) + ((ssq[4] + ssq[5]) + (ssq[6] + ssq[7]));
+
     float best = -INFINITY;
     int best_slot = 0;
+    float *part = nullptr;
+    if (a.splits > 1) {
+      const size_t tile = ((size_t)b * a.max_mt + mt) * a.splits + z;
+      part = a.part + tile * (size_t)a.keep_k * 128;
+      a.ss_part[tile * 128 + lrow] = ss;
+    }
     for (int nt = 0; nt < a.n_nt; ++nt) {
       const int buf = nt & 1;
       mbar_wait(smem_u32(&bk->acc_full[buf]), (nt >> 1) & 1, wc);
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 256;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (a.tmem_cols >> 1);
       const int slot0 = nt * a.n_tile;
       const int ncol = min(a.n_tile, a.keep_k - slot0);   // kept slots in this accumulator
 #pragma unroll 1
@@ -600,12 +660,18 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         uint32_t r[16];
         tmem_ld16(taddr + c, r);
         tmem_wait_ld();
+        if (part) {
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const int slot = slot0 + c + e;
-          if (c + e < ncol) {
-            const float val = __uint_as_float(r[e]) * __ldg(kinv + slot);
-            if (val > best) { best = val; best_slot = slot; }
+          for (int e = 0; e < 16; ++e)
+            if (c + e < ncol) part[(size_t)(slot0 + c + e) * 128 + lrow] = __uint_as_float(r[e]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int slot = slot0 + c + e;
+            if (c + e < ncol) {
+              const float val = __uint_as_float(r[e]) * __ldg(kinv + slot);
+              if (val > best) { best = val; best_slot = slot; }
+            }
           }
         }
       }
@@ -613,25 +679,79 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
     }
-    if (v < d.nv && !bk->abort_flag) {
+    float ss_tot = ss;
+    bool finalize = true;
+    if (a.splits > 1) {
+      // publish this slice; the last slice to arrive for the row tile reduces all of them
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (warp == 2 && lane == 0) {
+        unsigned int *cnt = a.tile_counters + (size_t)b * a.max_mt + mt;
+        const unsigned int old = atomicAdd(cnt, 1u);
+        bk->is_last = (old == (unsigned int)(a.splits - 1));
+        if (bk->is_last) *cnt = 0u;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      finalize = bk->is_last != 0;
+      if (finalize) {
+        __threadfence();
+        const size_t tile0 = ((size_t)b * a.max_mt + mt) * a.splits;
+        ss_tot = 0.f;
+        for (int zz = 0; zz < a.splits; ++zz) ss_tot += __ldcg(a.ss_part + (tile0 + zz) * 128 + lrow);
+        const float *p0 = a.part + tile0 * (size_t)a.keep_k * 128 + lrow;
+        const size_t zstride = (size_t)a.keep_k * 128;
+        for (int s0 = 0; s0 < a.keep_k; s0 += 16) {     // 16 slots x all slices in flight per thread
+          float acc[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+          for (int zz = 0; zz < a.splits; zz += 2) {
+            float x[2][16];
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+              for (int e = 0; e < 16; ++e)
+                x[t][e] = (zz + t < a.splits && s0 + e < a.keep_k)
+                              ? __ldcg(p0 + (zz + t) * zstride + (size_t)(s0 + e) * 128) : 0.f;
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+              for (int e = 0; e < 16; ++e) acc[e] += x[t][e];
+          }
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int slot = s0 + e;
+            if (slot < a.keep_k) {
+              const float val = acc[e] * __ldg(kinv + slot);
+              if (val > best) { best = val; best_slot = slot; }
+            }
+          }
+        }
+      }
+    }
+    if (finalize && v < d.nv && !bk->abort_flag) {
       const int role = a.role[(size_t)b * a.max_vis + v];
       if (role < 0) {
         const int dp = -role - 1;
-        const float sim = best * a.inv_norm[(size_t)b * a.max_vis + v];
+        const bool zero_row = !(ss_tot >= 1e-24f);      // ||h|| < 1e-12: similarity 0 to every slot
+        const float sim = zero_row ? 0.f : best * rsqrtf(ss_tot);
+        const int slot = zero_row ? 0 : best_slot;
         const size_t o = (size_t)b * (a.max_vis - a.keep_k) + dp;
-        a.assign[o] = (sim > a.threshold) ? best_slot : -1;
+        a.assign[o] = (sim > a.threshold) ? slot : -1;
         if (a.best_sim) a.best_sim[o] = sim;
       }
     }
+    if (warp == 2 && lane == 0) bk->is_last = finalize ? 1 : 0;
     __threadfence();
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, SIM_TMEM_COLS);
+    tmem_dealloc(tmem_base, a.tmem_cols);
   }
-  // the block that finishes last for this sample groups the dropped tokens by destination
+  if (!bk->is_last && a.splits > 1) return;     // a slice that did not finalize its row tile
+  __syncthreads();
+  // the block that finishes the sample's last row tile groups the dropped tokens by destination
   if (threadIdx.x == 0) {
     __threadfence();
     const unsigned int n_mt = (unsigned int)((d.nv + 127) / 128);
