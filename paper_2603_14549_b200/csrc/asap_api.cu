@@ -8,6 +8,7 @@
 #include <string.h>
 
 #include <new>
+#include <utility>
 
 #include "../../include/asap.h"
 #include "kernels_stream.cuh"
@@ -155,6 +156,24 @@ void mark(asap_ctx *ctx, const char *name, cudaStream_t st) {
   ctx->prof_name[ctx->prof_used++] = name;
 }
 
+// Every kernel is launched with programmatic stream serialization: its blocks may be scheduled
+// while the previous kernel of the stream drains, and wait (griddepcontrol.wait, first statement
+// of every kernel) until that kernel has completed and its writes are visible.
+template <typename... KArgs, typename... Args>
+void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);   // errors surface in after_launch
+}
+
 asap_status after_launch(asap_ctx *ctx, const char *what) {
   ctx->launches += 1;
   cudaError_t e = cudaGetLastError();
@@ -183,7 +202,7 @@ asap_status launch_prepare(asap_ctx *ctx, const asap_inputs *in, const asap_para
   a.text_start = in->text_start; a.text_len = in->text_len; a.rank_start = in->rank_start;
   a.rank_len = in->rank_len; a.desc = ctx->desc; a.out_cu_seqlens = out_cu; a.status = ctx->status;
   mark(ctx, "prepare", st);
-  prepare_kernel<<<1, 256, 0, st>>>(a);
+  launch_pdl(prepare_kernel, dim3(1), dim3(256), 0, st, a);
   return after_launch(ctx, "prepare");
 }
 
@@ -193,7 +212,7 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
   const int max_chunks = (in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS;
   const int col_blocks = (D + QSUM_COLS - 1) / QSUM_COLS;
   mark(ctx, "qsum", st);
-  qsum_kernel<<<dim3(max_chunks, col_blocks, B), QSUM_THREADS, 0, st>>>(
+  launch_pdl(qsum_kernel, dim3(dim3(max_chunks, col_blocks, B)), dim3(QSUM_THREADS), 0, st, 
       static_cast<const __nv_bfloat16 *>(in->q), ctx->desc, D, max_chunks, ctx->qsum_partial, ctx->qbar,
       ctx->cnt_qsum);
   ASAP_TRY(after_launch(ctx, "qsum"));
@@ -201,7 +220,7 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
   const float scale = 1.0f / ((float)in->H * sqrtf((float)in->head_dim));
   const int row_blocks = (in->max_vis + MASS_ROWS - 1) / MASS_ROWS;
   mark(ctx, "mass_salience", st);
-  mass_salience_kernel<<<dim3(row_blocks, B), MASS_THREADS, (size_t)D * sizeof(float), st>>>(
+  launch_pdl(mass_salience_kernel, dim3(dim3(row_blocks, B)), dim3(MASS_THREADS), (size_t)D * sizeof(float), st, 
       static_cast<const __nv_bfloat16 *>(in->k), ctx->desc, D, in->max_vis, scale, p->lambda_max, p->eps,
       ctx->qbar, out->mass, out->salience, out->mask_log, out->rank_score, ctx->cnt_mass);
   ASAP_TRY(after_launch(ctx, "mass_salience"));
@@ -216,10 +235,10 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
   sa.mask_log = out->mask_log; sa.partial = ctx->score_partial; sa.status = ctx->status;
   mark(ctx, "score", st);
   const int items = B * in->H;
-  score_kernel<<<items < ctx->num_sms ? items : ctx->num_sms, SC_THREADS, SC_SMEM_BYTES, st>>>(map_q, map_k, sa);
+  launch_pdl(score_kernel, dim3(items < ctx->num_sms ? items : ctx->num_sms), dim3(SC_THREADS), SC_SMEM_BYTES, st, map_q, map_k, sa);
   ASAP_TRY(after_launch(ctx, "score"));
   mark(ctx, "head_sum", st);
-  head_sum_kernel<<<dim3((in->max_vis + 255) / 256, B), 256, 0, st>>>(ctx->desc, in->H, in->max_vis,
+  launch_pdl(head_sum_kernel, dim3(dim3((in->max_vis + 255) / 256, B)), dim3(256), 0, st, ctx->desc, in->H, in->max_vis,
                                                                       ctx->score_partial, out->rank_score);
   return after_launch(ctx, "head_sum");
 }
@@ -231,7 +250,7 @@ bool merging(const asap_inputs *in, const asap_params *p) { return p->merge_enab
 asap_status launch_select(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                           const float *rank_score, const asap_outputs *out, bool with_merge, cudaStream_t st) {
   mark(ctx, "select", st);
-  select_kernel<<<in->B, SELECT_THREADS, (size_t)in->max_vis * sizeof(uint32_t), st>>>(
+  launch_pdl(select_kernel, dim3(in->B), dim3(SELECT_THREADS), (size_t)in->max_vis * sizeof(uint32_t), st, 
       rank_score, ctx->desc, in->max_vis, p->keep_k, out->keep_idx, out->drop_idx, ctx->role,
       with_merge ? out->assign : nullptr, with_merge ? out->best_sim : nullptr, merging(in, p) ? 1 : 0);
   return after_launch(ctx, "select");
@@ -244,7 +263,7 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
   const bool do_merge = merging(in, p);
   if (do_merge) {
     mark(ctx, "kept_gather", st);
-    kept_gather_kernel<<<dim3((k + GATHER_THREADS / 32 - 1) / (GATHER_THREADS / 32), B), GATHER_THREADS, 0, st>>>(
+    launch_pdl(kept_gather_kernel, dim3(dim3((k + GATHER_THREADS / 32 - 1) / (GATHER_THREADS / 32), B)), dim3(GATHER_THREADS), 0, st, 
         static_cast<const __nv_bfloat16 *>(in->hidden), ctx->desc, D, k, keep_idx, ctx->kept_rows, ctx->kept_inv);
     ASAP_TRY(after_launch(ctx, "kept_gather"));
 
@@ -290,7 +309,7 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
     sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
     sa.status = ctx->status;
     mark(ctx, "sim", st);
-    sim_kernel<<<dim3(max_mt, B, splits), SIM_THREADS, smem, st>>>(map_h, map_kept, sa);
+    launch_pdl(sim_kernel, dim3(dim3(max_mt, B, splits)), dim3(SIM_THREADS), smem, st, map_h, map_kept, sa);
     ASAP_TRY(after_launch(ctx, "sim"));
 
   }
@@ -305,10 +324,10 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
   const int nv = (D / 8 + MERGE_THREADS - 1) / MERGE_THREADS;
   mark(ctx, "merge_compact", st);
   switch (nv) {
-    case 1: merge_compact_kernel<1><<<grid, MERGE_THREADS, 0, st>>>(ma); break;
-    case 2: merge_compact_kernel<2><<<grid, MERGE_THREADS, 0, st>>>(ma); break;
-    case 3: merge_compact_kernel<3><<<grid, MERGE_THREADS, 0, st>>>(ma); break;
-    default: merge_compact_kernel<4><<<grid, MERGE_THREADS, 0, st>>>(ma); break;
+    case 1: launch_pdl(merge_compact_kernel<1>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
+    case 2: launch_pdl(merge_compact_kernel<2>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
+    case 3: launch_pdl(merge_compact_kernel<3>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
+    default: launch_pdl(merge_compact_kernel<4>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
   }
   return after_launch(ctx, "merge_compact");
 }
@@ -439,7 +458,7 @@ asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
   mark(ctx, "role_map", st);
-  role_map_kernel<<<dim3((in->max_vis + 255) / 256, in->B), 256, 0, st>>>(ctx->desc, in->max_vis, p->keep_k,
+  launch_pdl(role_map_kernel, dim3(dim3((in->max_vis + 255) / 256, in->B)), dim3(256), 0, st, ctx->desc, in->max_vis, p->keep_k,
                                                                          keep_idx, drop_idx, ctx->role, out->assign,
                                                                          out->best_sim, merging(in, p) ? 1 : 0);
   ASAP_TRY(after_launch(ctx, "role_map"));

@@ -32,6 +32,12 @@ enum : uint32_t {
   STATUS_SIM_TIMEOUT = 8u,     // a bounded wait ran out in the similarity kernel
 };
 
+// Programmatic dependent launch: wait until the previous kernel of the stream has completed and
+// its writes are visible; then allow the next kernel's blocks to be scheduled behind this one.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() { pdl_wait(); pdl_trigger(); }
+
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 

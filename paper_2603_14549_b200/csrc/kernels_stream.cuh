@@ -25,6 +25,7 @@ struct PrepareArgs {
 };
 
 __global__ void prepare_kernel(PrepareArgs a) {
+  pdl_enter();
   __shared__ int s_bad;
   if (threadIdx.x == 0) s_bad = 0;
   __syncthreads();
@@ -80,6 +81,7 @@ __global__ void __launch_bounds__(QSUM_THREADS)
 qsum_kernel(const __nv_bfloat16 *__restrict__ q, const SampleDesc *__restrict__ desc, int D,
             int max_chunks, float *__restrict__ partial /*[B, max_chunks, D]*/,
             float *__restrict__ qbar /*[B, D]*/, unsigned int *__restrict__ counters) {
+  pdl_enter();
   const int b = blockIdx.z, cb = blockIdx.y, chunk = blockIdx.x;
   const SampleDesc d = desc[b];
   if (!d.valid) return;
@@ -161,6 +163,7 @@ mass_salience_kernel(const __nv_bfloat16 *__restrict__ k, const SampleDesc *__re
                      const float *__restrict__ qbar, float *__restrict__ mass,
                      float *__restrict__ salience, float *__restrict__ mask_log,
                      float *__restrict__ rank_score, unsigned int *__restrict__ counters) {
+  pdl_enter();
   extern __shared__ float s_q[];   // [D]
   __shared__ float s_red[2 * (MASS_THREADS / 32)];
   __shared__ int s_last;
@@ -306,6 +309,7 @@ select_kernel(const float *__restrict__ rank_score, const SampleDesc *__restrict
               int max_vis, int keep_k, int32_t *__restrict__ keep_idx, int32_t *__restrict__ drop_idx,
               int32_t *__restrict__ role /*[B, max_vis]*/, int32_t *__restrict__ assign /*nullable*/,
               float *__restrict__ best_sim /*nullable*/, int sim_follows) {
+  pdl_enter();
   extern __shared__ uint32_t s_key[];   // [max_vis]
   __shared__ int s_hist[256];
   __shared__ int s_scan[33];
@@ -425,6 +429,7 @@ __global__ void role_map_kernel(const SampleDesc *__restrict__ desc, int max_vis
                                 const int32_t *__restrict__ drop_idx, int32_t *__restrict__ role,
                                 int32_t *__restrict__ assign, float *__restrict__ best_sim,
                                 int sim_follows) {
+  pdl_enter();
   const int b = blockIdx.y;
   const SampleDesc d = desc[b];
   const int nd_max = max_vis - keep_k;
@@ -460,6 +465,7 @@ kept_gather_kernel(const __nv_bfloat16 *__restrict__ hidden, const SampleDesc *_
                    int D, int keep_k, const int32_t *__restrict__ keep_idx,
                    __nv_bfloat16 *__restrict__ kept_rows /*[B*keep_k, D]*/,
                    float *__restrict__ kept_inv /*[B*keep_k]*/) {
+  pdl_enter();
   const int b = blockIdx.y;
   const SampleDesc d = desc[b];
   if (!d.valid) return;
@@ -596,6 +602,7 @@ struct MergeArgs {
 template <int NV>   // 16-byte vectors per thread: D <= NV * 256 * 8
 __global__ void __launch_bounds__(MERGE_THREADS)
 merge_compact_kernel(MergeArgs a) {
+  pdl_enter();
   __shared__ int s_j[MERGE_LIST];
   __shared__ float s_w[MERGE_LIST];
   const int b = blockIdx.y;

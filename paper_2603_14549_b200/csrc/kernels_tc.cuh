@@ -98,6 +98,7 @@ __device__ __forceinline__ RowTile score_row_tile(const SampleDesc &d, int rt, i
 __global__ void __launch_bounds__(SC_THREADS, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
              ScoreArgs a) {
+  pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_items = a.B * a.H;
@@ -432,6 +433,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
 __global__ void __launch_bounds__(256)
 head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
                 const float *__restrict__ partial, float *__restrict__ rank_score) {
+  pdl_enter();
   const int b = blockIdx.y;
   const SampleDesc d = desc[b];
   const int j = blockIdx.x * 256 + threadIdx.x;
@@ -510,6 +512,7 @@ __device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t n) {
 __global__ void __launch_bounds__(SIM_THREADS, 1)
 sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_kept,
            SimArgs a) {
+  pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   const int mt = blockIdx.x, b = blockIdx.y, z = blockIdx.z;
   const SampleDesc d = a.desc[b];
