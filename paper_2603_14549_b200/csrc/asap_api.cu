@@ -193,27 +193,35 @@ asap_status finish(asap_ctx *ctx, asap_status result, cudaStream_t st) {
   } while (0)
 
 // ---- stage launchers -------------------------------------------------------------------------
-asap_status launch_prepare(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
-                           int32_t *out_cu, int out_capacity, cudaStream_t st) {
+PrepareArgs prepare_args(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, int32_t *out_cu,
+                         int out_capacity) {
   PrepareArgs a;
   a.B = in->B; a.total_tokens = in->total_tokens; a.min_vis = in->min_vis; a.max_vis = in->max_vis;
   a.max_seq = in->max_seq; a.max_rank = in->max_rank; a.keep_k = p->keep_k; a.out_capacity = out_capacity;
   a.cu_seqlens = in->cu_seqlens; a.vis_start = in->vis_start; a.vis_len = in->vis_len;
   a.text_start = in->text_start; a.text_len = in->text_len; a.rank_start = in->rank_start;
   a.rank_len = in->rank_len; a.desc = ctx->desc; a.out_cu_seqlens = out_cu; a.status = ctx->status;
+  return a;
+}
+
+asap_status launch_prepare(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                           int32_t *out_cu, int out_capacity, cudaStream_t st) {
   mark(ctx, "prepare", st);
-  launch_pdl(prepare_kernel, dim3(1), dim3(256), 0, st, a);
+  launch_pdl(prepare_kernel, dim3(1), dim3(256), 0, st, prepare_args(ctx, in, p, out_cu, out_capacity));
   return after_launch(ctx, "prepare");
 }
 
+// The query-sum kernel opens the step: it also carries the device-side validation (prepare).
 asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
-                         const asap_outputs *out, cudaStream_t st) {
+                         const asap_outputs *out, int32_t *out_cu, int out_capacity, bool with_head_sum,
+                         cudaStream_t st) {
   const int D = in->D, B = in->B;
   const int max_chunks = (in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS;
   const int col_blocks = (D + QSUM_COLS - 1) / QSUM_COLS;
   mark(ctx, "qsum", st);
   launch_pdl(qsum_kernel, dim3(dim3(max_chunks, col_blocks, B)), dim3(QSUM_THREADS), 0, st, 
-      static_cast<const __nv_bfloat16 *>(in->q), ctx->desc, D, max_chunks, ctx->qsum_partial, ctx->qbar,
+      static_cast<const __nv_bfloat16 *>(in->q), prepare_args(ctx, in, p, out_cu, out_capacity), D, max_chunks,
+      ctx->qsum_partial, ctx->qbar,
       ctx->cnt_qsum);
   ASAP_TRY(after_launch(ctx, "qsum"));
 
@@ -237,6 +245,7 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
   const int items = B * in->H;
   launch_pdl(score_kernel, dim3(items < ctx->num_sms ? items : ctx->num_sms), dim3(SC_THREADS), SC_SMEM_BYTES, st, map_q, map_k, sa);
   ASAP_TRY(after_launch(ctx, "score"));
+  if (!with_head_sum) return ASAP_OK;
   mark(ctx, "head_sum", st);
   launch_pdl(head_sum_kernel, dim3(dim3((in->max_vis + 255) / 256, B)), dim3(256), 0, st, ctx->desc, in->H, in->max_vis,
                                                                       ctx->score_partial, out->rank_score);
@@ -247,12 +256,16 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
 // dropped token itself)
 bool merging(const asap_inputs *in, const asap_params *p) { return p->merge_enable && in->max_vis > p->keep_k; }
 
+// `fused_head_sum`: the ranking scores are still per-head sums in scratch (the score kernel ran
+// without its head-sum kernel); the selection adds the heads itself and writes out->rank_score.
 asap_status launch_select(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
-                          const float *rank_score, const asap_outputs *out, bool with_merge, cudaStream_t st) {
+                          const float *rank_score, const asap_outputs *out, bool with_merge,
+                          bool fused_head_sum, cudaStream_t st) {
   mark(ctx, "select", st);
-  launch_pdl(select_kernel, dim3(in->B), dim3(SELECT_THREADS), (size_t)in->max_vis * sizeof(uint32_t), st, 
-      rank_score, ctx->desc, in->max_vis, p->keep_k, out->keep_idx, out->drop_idx, ctx->role,
-      with_merge ? out->assign : nullptr, with_merge ? out->best_sim : nullptr, merging(in, p) ? 1 : 0);
+  launch_pdl(select_kernel, dim3(in->B), dim3(SELECT_THREADS), (size_t)in->max_vis * sizeof(uint32_t), st,
+             rank_score, ctx->desc, in->max_vis, p->keep_k, out->keep_idx, out->drop_idx, ctx->role,
+             with_merge ? out->assign : nullptr, with_merge ? out->best_sim : nullptr, merging(in, p) ? 1 : 0,
+             fused_head_sum ? ctx->score_partial : nullptr, in->H, fused_head_sum ? out->rank_score : nullptr);
   return after_launch(ctx, "select");
 }
 
@@ -436,8 +449,7 @@ asap_status asap_score(asap_ctx *ctx, const asap_inputs *in, const asap_params *
                        void *stream) {
   ASAP_TRY(validate(ctx, in, p, out, NEED_QK | NEED_SCORE_OUT));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  ASAP_TRY(launch_prepare(ctx, in, p, nullptr, 0x7fffffff, st));
-  return finish(ctx, launch_score(ctx, in, p, out, st), st);
+  return finish(ctx, launch_score(ctx, in, p, out, nullptr, 0x7fffffff, true, st), st);
 }
 
 asap_status asap_select(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *rank_score,
@@ -446,7 +458,7 @@ asap_status asap_select(asap_ctx *ctx, const asap_inputs *in, const asap_params 
   if (!rank_score) return fail(ctx, ASAP_ERR_INVALID, "null rank_score");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   ASAP_TRY(launch_prepare(ctx, in, p, nullptr, 0x7fffffff, st));
-  return finish(ctx, launch_select(ctx, in, p, rank_score, out, false, st), st);
+  return finish(ctx, launch_select(ctx, in, p, rank_score, out, false, false, st), st);
 }
 
 asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *salience,
@@ -469,9 +481,8 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
                             void *stream) {
   ASAP_TRY(validate(ctx, in, p, out, NEED_QK | NEED_HIDDEN | NEED_SCORE_OUT | NEED_SELECT_OUT | NEED_MERGE_OUT));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
-  ASAP_TRY(launch_score(ctx, in, p, out, st));
-  ASAP_TRY(launch_select(ctx, in, p, out->rank_score, out, true, st));
+  ASAP_TRY(launch_score(ctx, in, p, out, out->out_cu_seqlens, out->out_rows_capacity, false, st));
+  ASAP_TRY(launch_select(ctx, in, p, out->rank_score, out, true, true, st));
   return finish(ctx, launch_merge(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st), st);
 }
 
@@ -628,7 +639,7 @@ asap_status asap_select_static(const asap_inputs *in, const asap_params *p, cons
   out.keep_idx = keep_idx;
   out.drop_idx = drop_idx;
   asap_status r = launch_prepare(&view, in, p, nullptr, 0x7fffffff, st);
-  if (r == ASAP_OK) r = launch_select(&view, in, p, rank_score, &out, false, st);
+  if (r == ASAP_OK) r = launch_select(&view, in, p, rank_score, &out, false, false, st);
   if (r != ASAP_OK) snprintf(g_init_error, sizeof(g_init_error), "asap_select_static: %s", view.err);
   return r;
 }

@@ -24,30 +24,37 @@ struct PrepareArgs {
   uint32_t *status;
 };
 
-__global__ void prepare_kernel(PrepareArgs a) {
-  pdl_enter();
+// Descriptor of sequence b with its validity (out_row0 is filled in by prepare_block).
+__device__ __forceinline__ SampleDesc make_desc(const PrepareArgs &a, int b) {
+  const int lo = a.cu_seqlens[b], hi = a.cu_seqlens[b + 1];
+  const int n = hi - lo;
+  const int v0 = a.vis_start[b], nv = a.vis_len[b];
+  const int t0 = a.text_start[b], tl = a.text_len[b];
+  const int r0 = a.rank_start ? a.rank_start[b] : t0;
+  const int nr = a.rank_len ? a.rank_len[b] : tl;
+  bool ok = lo >= 0 && n > 0 && n <= a.max_seq && hi <= a.total_tokens;
+  ok = ok && v0 >= 0 && nv >= a.min_vis && nv <= a.max_vis && v0 + nv <= n;
+  ok = ok && tl >= 0 && t0 >= v0 + nv && t0 + tl <= n;
+  ok = ok && r0 >= 0 && nr >= 1 && nr <= a.max_rank && r0 + nr <= n;
+  ok = ok && a.keep_k <= nv;
+  if (b == 0) ok = ok && lo == 0;
+  if (b == a.B - 1) ok = ok && hi == a.total_tokens;
+  SampleDesc d;
+  d.row0 = lo; d.n = n; d.v0 = v0; d.nv = nv; d.r0 = r0; d.nr = nr; d.out_row0 = 0;
+  d.valid = ok ? 1 : 0;
+  return d;
+}
+
+// Run by one whole block: validates every sequence, writes the descriptors, the output row
+// offsets and the status bits.
+__device__ __forceinline__ void prepare_block(const PrepareArgs &a) {
   __shared__ int s_bad;
   if (threadIdx.x == 0) s_bad = 0;
   __syncthreads();
   for (int b = threadIdx.x; b < a.B; b += blockDim.x) {
-    const int lo = a.cu_seqlens[b], hi = a.cu_seqlens[b + 1];
-    const int n = hi - lo;
-    const int v0 = a.vis_start[b], nv = a.vis_len[b];
-    const int t0 = a.text_start[b], tl = a.text_len[b];
-    const int r0 = a.rank_start ? a.rank_start[b] : t0;
-    const int nr = a.rank_len ? a.rank_len[b] : tl;
-    bool ok = lo >= 0 && n > 0 && n <= a.max_seq && hi <= a.total_tokens;
-    ok = ok && v0 >= 0 && nv >= a.min_vis && nv <= a.max_vis && v0 + nv <= n;
-    ok = ok && tl >= 0 && t0 >= v0 + nv && t0 + tl <= n;
-    ok = ok && r0 >= 0 && nr >= 1 && nr <= a.max_rank && r0 + nr <= n;
-    ok = ok && a.keep_k <= nv;
-    if (b == 0) ok = ok && lo == 0;
-    if (b == a.B - 1) ok = ok && hi == a.total_tokens;
-    SampleDesc d;
-    d.row0 = lo; d.n = n; d.v0 = v0; d.nv = nv; d.r0 = r0; d.nr = nr; d.out_row0 = 0;
-    d.valid = ok ? 1 : 0;
+    const SampleDesc d = make_desc(a, b);
     a.desc[b] = d;
-    if (!ok) s_bad = 1;
+    if (!d.valid) s_bad = 1;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -66,6 +73,12 @@ __global__ void prepare_kernel(PrepareArgs a) {
     }
     if (bits) atomicOr(a.status, bits);
   }
+  __syncthreads();
+}
+
+__global__ void prepare_kernel(PrepareArgs a) {
+  pdl_enter();
+  prepare_block(a);
 }
 
 // =======================================================================================
@@ -78,12 +91,15 @@ constexpr int QSUM_THREADS = 256;
 constexpr int QSUM_COLS = QSUM_THREADS * 8;
 
 __global__ void __launch_bounds__(QSUM_THREADS)
-qsum_kernel(const __nv_bfloat16 *__restrict__ q, const SampleDesc *__restrict__ desc, int D,
+qsum_kernel(const __nv_bfloat16 *__restrict__ q, PrepareArgs pa, int D,
             int max_chunks, float *__restrict__ partial /*[B, max_chunks, D]*/,
             float *__restrict__ qbar /*[B, D]*/, unsigned int *__restrict__ counters) {
   pdl_enter();
   const int b = blockIdx.z, cb = blockIdx.y, chunk = blockIdx.x;
-  const SampleDesc d = desc[b];
+  // This is the first kernel of the step: block (0,0,0) also does the device-side validation
+  // and writes the descriptors every later kernel reads; each block derives its own copy.
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) prepare_block(pa);
+  const SampleDesc d = make_desc(pa, b);
   if (!d.valid) return;
   const int nchunks = (d.nv + QSUM_ROWS - 1) / QSUM_ROWS;
   if (chunk >= nchunks) return;
@@ -308,7 +324,9 @@ __global__ void __launch_bounds__(SELECT_THREADS)
 select_kernel(const float *__restrict__ rank_score, const SampleDesc *__restrict__ desc,
               int max_vis, int keep_k, int32_t *__restrict__ keep_idx, int32_t *__restrict__ drop_idx,
               int32_t *__restrict__ role /*[B, max_vis]*/, int32_t *__restrict__ assign /*nullable*/,
-              float *__restrict__ best_sim /*nullable*/, int sim_follows) {
+              float *__restrict__ best_sim /*nullable*/, int sim_follows,
+              const float *__restrict__ head_partial /*nullable: [B, H, max_vis]*/, int H,
+              float *__restrict__ rank_out /*[B, max_vis], written when head_partial is given*/) {
   pdl_enter();
   extern __shared__ uint32_t s_key[];   // [max_vis]
   __shared__ int s_hist[256];
@@ -337,8 +355,32 @@ select_kernel(const float *__restrict__ rank_score, const SampleDesc *__restrict
     return;
   }
   const int nv = d.nv;
-  for (int j = threadIdx.x; j < nv; j += blockDim.x)
-    s_key[j] = score_key(rank_score[(size_t)b * max_vis + j]);
+  if (head_partial) {
+    // r_j = mean over heads and ranking rows of the Eq. 4 probabilities: the per-head sums
+    // over ranking rows are added here in head order, and r is also written out
+    const float inv = 1.0f / ((float)H * (float)d.nr);
+    for (int j = threadIdx.x; j < max_vis; j += blockDim.x) {
+      float tot = 0.f;
+      if (j < nv) {
+        const float *p = head_partial + (size_t)b * H * max_vis + j;
+        int hh = 0;
+        for (; hh + 8 <= H; hh += 8) {
+          float v[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) v[e] = __ldcg(p + (size_t)(hh + e) * max_vis);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) tot += v[e];
+        }
+        for (; hh < H; ++hh) tot += __ldcg(p + (size_t)hh * max_vis);
+        tot *= inv;
+        s_key[j] = score_key(tot);
+      }
+      rank_out[(size_t)b * max_vis + j] = tot;
+    }
+  } else {
+    for (int j = threadIdx.x; j < nv; j += blockDim.x)
+      s_key[j] = score_key(rank_score[(size_t)b * max_vis + j]);
+  }
   if (threadIdx.x == 0) { s_prefix = 0u; s_remaining = keep_k; }
   __syncthreads();
 
