@@ -48,6 +48,8 @@ struct asap_ctx {
   __nv_bfloat16 *kept_rows = nullptr;
   uint32_t *status = nullptr;
   EncodeTiledFn encode = nullptr;
+  cudaStream_t side = nullptr;            // second stream for the mass kernels of asap_prune_step
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   uint64_t launches = 0;
   char err[512] = "";
   // per-kernel timing (asap_profile): one event before every launch, one at the end of a call
@@ -211,28 +213,34 @@ asap_status launch_prepare(asap_ctx *ctx, const asap_inputs *in, const asap_para
   return after_launch(ctx, "prepare");
 }
 
-// The query-sum kernel opens the step: it also carries the device-side validation (prepare).
-asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
-                         const asap_outputs *out, int32_t *out_cu, int out_capacity, bool with_head_sum,
-                         cudaStream_t st) {
+// Steps 1a-1b: query sum, attention mass, salience, mask vector.  With `fold_prepare` the query-sum
+// kernel also carries the device-side validation and writes the descriptors.
+asap_status launch_mass(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const asap_outputs *out,
+                        bool fold_prepare, int32_t *out_cu, int out_capacity, cudaStream_t st) {
   const int D = in->D, B = in->B;
   const int max_chunks = (in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS;
   const int col_blocks = (D + QSUM_COLS - 1) / QSUM_COLS;
+  PrepareArgs pa = prepare_args(ctx, in, p, out_cu, out_capacity);
+  pa.write_desc = fold_prepare ? 1 : 0;
   mark(ctx, "qsum", st);
-  launch_pdl(qsum_kernel, dim3(dim3(max_chunks, col_blocks, B)), dim3(QSUM_THREADS), 0, st, 
-      static_cast<const __nv_bfloat16 *>(in->q), prepare_args(ctx, in, p, out_cu, out_capacity), D, max_chunks,
-      ctx->qsum_partial, ctx->qbar,
-      ctx->cnt_qsum);
+  launch_pdl(qsum_kernel, dim3(max_chunks, col_blocks, B), dim3(QSUM_THREADS), 0, st,
+             static_cast<const __nv_bfloat16 *>(in->q), pa, D, max_chunks, ctx->qsum_partial, ctx->qbar,
+             ctx->cnt_qsum);
   ASAP_TRY(after_launch(ctx, "qsum"));
 
   const float scale = 1.0f / ((float)in->H * sqrtf((float)in->head_dim));
   const int row_blocks = (in->max_vis + MASS_ROWS - 1) / MASS_ROWS;
   mark(ctx, "mass_salience", st);
-  launch_pdl(mass_salience_kernel, dim3(dim3(row_blocks, B)), dim3(MASS_THREADS), (size_t)D * sizeof(float), st, 
-      static_cast<const __nv_bfloat16 *>(in->k), ctx->desc, D, in->max_vis, scale, p->lambda_max, p->eps,
-      ctx->qbar, out->mass, out->salience, out->mask_log, out->rank_score, ctx->cnt_mass);
-  ASAP_TRY(after_launch(ctx, "mass_salience"));
+  launch_pdl(mass_salience_kernel, dim3(row_blocks, B), dim3(MASS_THREADS), (size_t)D * sizeof(float), st,
+             static_cast<const __nv_bfloat16 *>(in->k), ctx->desc, D, in->max_vis, scale, p->lambda_max, p->eps,
+             ctx->qbar, out->mass, out->salience, out->mask_log, out->rank_score, ctx->cnt_mass);
+  return after_launch(ctx, "mass_salience");
+}
 
+// Steps 1c-2: Eq. 4 probabilities of the ranking rows, summed per head; optionally the head sum.
+asap_status launch_rank(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const asap_outputs *out,
+                        bool with_head_sum, cudaStream_t st) {
+  const int D = in->D, B = in->B;
   CUtensorMap map_q, map_k;
   if (!make_map(ctx, &map_q, in->q, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
       !make_map(ctx, &map_k, in->k, (uint64_t)in->total_tokens, (uint64_t)D, 128))
@@ -243,12 +251,13 @@ asap_status launch_score(asap_ctx *ctx, const asap_inputs *in, const asap_params
   sa.mask_log = out->mask_log; sa.partial = ctx->score_partial; sa.status = ctx->status;
   mark(ctx, "score", st);
   const int items = B * in->H;
-  launch_pdl(score_kernel, dim3(items < ctx->num_sms ? items : ctx->num_sms), dim3(SC_THREADS), SC_SMEM_BYTES, st, map_q, map_k, sa);
+  launch_pdl(score_kernel, dim3(items < ctx->num_sms ? items : ctx->num_sms), dim3(SC_THREADS), SC_SMEM_BYTES, st,
+             map_q, map_k, sa);
   ASAP_TRY(after_launch(ctx, "score"));
   if (!with_head_sum) return ASAP_OK;
   mark(ctx, "head_sum", st);
-  launch_pdl(head_sum_kernel, dim3(dim3((in->max_vis + 255) / 256, B)), dim3(256), 0, st, ctx->desc, in->H, in->max_vis,
-                                                                      ctx->score_partial, out->rank_score);
+  launch_pdl(head_sum_kernel, dim3((in->max_vis + 255) / 256, B), dim3(256), 0, st, ctx->desc, in->H, in->max_vis,
+             ctx->score_partial, out->rank_score);
   return after_launch(ctx, "head_sum");
 }
 
@@ -269,12 +278,11 @@ asap_status launch_select(asap_ctx *ctx, const asap_inputs *in, const asap_param
   return after_launch(ctx, "select");
 }
 
-asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
-                         const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
-                         const asap_outputs *out, cudaStream_t st) {
+// Step 4a: kept rows gathered, cosine similarity and assignment, CSR of the assignment.
+asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                               const int32_t *keep_idx, const asap_outputs *out, cudaStream_t st) {
   const int B = in->B, D = in->D, k = p->keep_k;
-  const bool do_merge = merging(in, p);
-  if (do_merge) {
+  if (merging(in, p)) {
     mark(ctx, "kept_gather", st);
     launch_pdl(kept_gather_kernel, dim3(dim3((k + GATHER_THREADS / 32 - 1) / (GATHER_THREADS / 32), B)), dim3(GATHER_THREADS), 0, st, 
         static_cast<const __nv_bfloat16 *>(in->hidden), ctx->desc, D, k, keep_idx, ctx->kept_rows, ctx->kept_inv);
@@ -324,8 +332,16 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
     mark(ctx, "sim", st);
     launch_pdl(sim_kernel, dim3(dim3(max_mt, B, splits)), dim3(SIM_THREADS), smem, st, map_h, map_kept, sa);
     ASAP_TRY(after_launch(ctx, "sim"));
-
   }
+  return ASAP_OK;
+}
+
+// Steps 4b-5: weighted merge and compaction (the first consumer of the salience).
+asap_status launch_merge_back(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                              const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
+                              const asap_outputs *out, cudaStream_t st) {
+  const int B = in->B, D = in->D, k = p->keep_k;
+  const bool do_merge = merging(in, p);
   MergeArgs ma;
   ma.hidden = static_cast<const __nv_bfloat16 *>(in->hidden); ma.pos_ids = in->pos_ids; ma.desc = ctx->desc;
   ma.D = D; ma.max_vis = in->max_vis; ma.keep_k = k; ma.merge_enable = do_merge ? 1 : 0; ma.eps = p->eps;
@@ -343,6 +359,13 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
     default: launch_pdl(merge_compact_kernel<4>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
   }
   return after_launch(ctx, "merge_compact");
+}
+
+asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                         const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
+                         const asap_outputs *out, cudaStream_t st) {
+  ASAP_TRY(launch_merge_front(ctx, in, p, keep_idx, out, st));
+  return launch_merge_back(ctx, in, p, salience, keep_idx, drop_idx, out, st);
 }
 
 }  // namespace
@@ -435,8 +458,14 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   if (e == cudaSuccess) e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    if (ctx->side) cudaStreamDestroy(ctx->side);
     cudaFree(ctx->arena);
     delete ctx;
     return fail(nullptr, ASAP_ERR_CUDA, "asap_init set-up: %s", cudaGetErrorString(e));
@@ -449,7 +478,8 @@ asap_status asap_score(asap_ctx *ctx, const asap_inputs *in, const asap_params *
                        void *stream) {
   ASAP_TRY(validate(ctx, in, p, out, NEED_QK | NEED_SCORE_OUT));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return finish(ctx, launch_score(ctx, in, p, out, nullptr, 0x7fffffff, true, st), st);
+  ASAP_TRY(launch_mass(ctx, in, p, out, true, nullptr, 0x7fffffff, st));
+  return finish(ctx, launch_rank(ctx, in, p, out, true, st), st);
 }
 
 asap_status asap_select(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *rank_score,
@@ -481,9 +511,34 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
                             void *stream) {
   ASAP_TRY(validate(ctx, in, p, out, NEED_QK | NEED_HIDDEN | NEED_SCORE_OUT | NEED_SELECT_OUT | NEED_MERGE_OUT));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  ASAP_TRY(launch_score(ctx, in, p, out, out->out_cu_seqlens, out->out_rows_capacity, false, st));
-  ASAP_TRY(launch_select(ctx, in, p, out->rank_score, out, true, true, st));
-  return finish(ctx, launch_merge(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st), st);
+  // With the text span as ranking rows the Eq. 3 mask never touches a ranked row (a text query lies
+  // after every visual key), so the score kernel does not need the attention mass: the memory-bound
+  // mass kernels then run on the context's side stream next to the score kernel, and rejoin before
+  // the merge, which is the first consumer of the salience.  With caller-given ranking rows (which may
+  // be visual) and while per-kernel timing is on, everything runs in order on `stream`.
+  const bool overlap = in->rank_start == nullptr && !ctx->prof_on && ctx->side != nullptr;
+  if (!overlap) {
+    ASAP_TRY(launch_mass(ctx, in, p, out, true, out->out_cu_seqlens, out->out_rows_capacity, st));
+    ASAP_TRY(launch_rank(ctx, in, p, out, false, st));
+    ASAP_TRY(launch_select(ctx, in, p, out->rank_score, out, true, true, st));
+    return finish(ctx, launch_merge(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st), st);
+  }
+  ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
+  cudaError_t e = cudaEventRecord(ctx->ev_fork, st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0);
+  if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "fork to the side stream: %s", cudaGetErrorString(e));
+  asap_status side_status = launch_mass(ctx, in, p, out, false, nullptr, 0x7fffffff, ctx->side);
+  e = cudaEventRecord(ctx->ev_join, ctx->side);
+  if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "join event: %s", cudaGetErrorString(e));
+  asap_status main_status = side_status;
+  if (main_status == ASAP_OK) main_status = launch_rank(ctx, in, p, out, false, st);
+  if (main_status == ASAP_OK) main_status = launch_select(ctx, in, p, out->rank_score, out, true, true, st);
+  if (main_status == ASAP_OK) main_status = launch_merge_front(ctx, in, p, out->keep_idx, out, st);
+  // the side stream always rejoins, also after an error, so that `stream` stays ordered behind it
+  e = cudaStreamWaitEvent(st, ctx->ev_join, 0);
+  if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "join with the side stream: %s", cudaGetErrorString(e));
+  if (main_status != ASAP_OK) return main_status;
+  return finish(ctx, launch_merge_back(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st), st);
 }
 
 asap_status asap_check(asap_ctx *ctx, void *stream) {
@@ -656,6 +711,9 @@ void asap_free(asap_ctx *ctx) {
     delete[] ctx->prof_ev;
     delete[] ctx->prof_name;
   }
+  if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
   cudaFree(ctx->arena);
   delete ctx;
 }

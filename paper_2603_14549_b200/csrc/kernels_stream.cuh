@@ -18,6 +18,7 @@ namespace asap {
 // =======================================================================================
 struct PrepareArgs {
   int32_t B, total_tokens, min_vis, max_vis, max_seq, max_rank, keep_k, out_capacity;
+  int32_t write_desc;        // query-sum kernel only: its first block also runs prepare_block
   const int32_t *cu_seqlens, *vis_start, *vis_len, *text_start, *text_len, *rank_start, *rank_len;
   SampleDesc *desc;          // [B]
   int32_t *out_cu_seqlens;   // [B+1] or nullptr
@@ -96,9 +97,9 @@ qsum_kernel(const __nv_bfloat16 *__restrict__ q, PrepareArgs pa, int D,
             float *__restrict__ qbar /*[B, D]*/, unsigned int *__restrict__ counters) {
   pdl_enter();
   const int b = blockIdx.z, cb = blockIdx.y, chunk = blockIdx.x;
-  // This is the first kernel of the step: block (0,0,0) also does the device-side validation
+  // When this is the first kernel of the step, block (0,0,0) also does the device-side validation
   // and writes the descriptors every later kernel reads; each block derives its own copy.
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) prepare_block(pa);
+  if (pa.write_desc && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) prepare_block(pa);
   const SampleDesc d = make_desc(pa, b);
   if (!d.valid) return;
   const int nchunks = (d.nv + QSUM_ROWS - 1) / QSUM_ROWS;
