@@ -242,7 +242,7 @@ asap_status launch_rank(asap_ctx *ctx, const asap_inputs *in, const asap_params 
                         bool with_head_sum, cudaStream_t st) {
   const int D = in->D, B = in->B;
   CUtensorMap map_q, map_k;
-  if (!make_map(ctx, &map_q, in->q, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
+  if (!make_map(ctx, &map_q, in->q, (uint64_t)in->total_tokens, (uint64_t)D, 32) ||
       !make_map(ctx, &map_k, in->k, (uint64_t)in->total_tokens, (uint64_t)D, 128))
     return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for q / k");
   ScoreArgs sa;
