@@ -242,7 +242,7 @@ asap_status launch_rank(asap_ctx *ctx, const asap_inputs *in, const asap_params 
                         bool with_head_sum, cudaStream_t st) {
   const int D = in->D, B = in->B;
   CUtensorMap map_q, map_k;
-  if (!make_map(ctx, &map_q, in->q, (uint64_t)in->total_tokens, (uint64_t)D, 32) ||
+  if (!make_map(ctx, &map_q, in->q, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
       !make_map(ctx, &map_k, in->k, (uint64_t)in->total_tokens, (uint64_t)D, 128))
     return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for q / k");
   ScoreArgs sa;
@@ -310,8 +310,10 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     while ((int)tmem_cols < 2 * n_tile) tmem_cols <<= 1;
     const long long ctas = (long long)max_mt * B * splits;
     const bool two_per_sm = ctas > ctx->num_sms && ctas <= 2LL * ctx->num_sms && tmem_cols <= 256 &&
-                            2 * stage_bytes <= 100 * 1024;
-    int stages = ((two_per_sm ? 100 : 200) * 1024) / stage_bytes;
+                            2 * stage_bytes <= 96 * 1024;
+    // at most 192 KB of tiles: the block then fits the 196 KB shared-memory carve-out, which leaves
+    // the SM its 32 KB of L1
+    int stages = ((two_per_sm ? 96 : 192) * 1024) / stage_bytes;
     if (stages > SIM_MAX_STAGES) stages = SIM_MAX_STAGES;
     const size_t smem = (size_t)stages * stage_bytes + SIM_BOOK_BYTES + 1024;
     if ((size_t)(SIM_THREADS / 32 + 1) * k * sizeof(int) > (size_t)stages * stage_bytes)

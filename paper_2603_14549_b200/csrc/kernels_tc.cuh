@@ -54,8 +54,11 @@ constexpr int SC_STAGES = 4;
 constexpr int SC_HALF_BYTES = 128 * 128;        // 128 rows x 64 bf16
 constexpr int SC_TILE_BYTES = 2 * SC_HALF_BYTES;
 constexpr int SC_SMEM_MAIN = (2 + SC_STAGES) * SC_TILE_BYTES;
-constexpr int SC_BOOK_BYTES = 4096;
-constexpr int SC_SMEM_BYTES = SC_SMEM_MAIN + SC_BOOK_BYTES + 1024;   // + bookkeeping + alignment slack
+// Total dynamic shared memory stays at 195 KB: with the 1 KB the system reserves per block that
+// is the 196 KB carve-out, which leaves the SM 32 KB of L1 for the memory-bound kernels that run
+// beside this one; one byte more selects the 228 KB carve-out and costs them about 10 us.
+constexpr int SC_BOOK_BYTES = 3072;
+constexpr int SC_SMEM_BYTES = SC_SMEM_MAIN + SC_BOOK_BYTES;
 constexpr uint32_t SC_TMEM_COLS = 512;     // four accumulators of 128 columns
 
 struct ScoreArgs {
@@ -71,7 +74,7 @@ struct ScoreBook {             // bookkeeping block placed after the tiles in sh
   uint64_t full[SC_STAGES], empty[SC_STAGES], q_full[2], q_empty[2], acc_full[4], acc_empty[4];
   float off[128];              // per ranking row: max + log2(sum), +inf for rows past the tile
   float soft[2][128];          // per epilogue group, per key of its current tile: m_j*log2(e) or -inf
-  float pm[2][128], pl[2][128];   // per epilogue group and lane: running (max, sum) at the end of pass 1
+  float pm[128], pl[128];      // group 1's running (max, sum) per row at the end of pass 1
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -80,7 +83,6 @@ static_assert(sizeof(ScoreBook) <= SC_BOOK_BYTES, "score kernel bookkeeping exce
 
 struct RowTile {
   int R0, nrows, n_kt, t_lo, t_hi, n_p2;
-  int tpad;        // rows rounded up to 32, 64 or 128: the query tile holds 128 / tpad copies of them
   bool use_soft;
 };
 
@@ -88,7 +90,6 @@ __device__ __forceinline__ RowTile score_row_tile(const SampleDesc &d, int rt, i
   RowTile r;
   r.R0 = d.r0 + rt * 128;
   r.nrows = min(128, d.nr - rt * 128);
-  r.tpad = r.nrows <= 32 ? 32 : (r.nrows <= 64 ? 64 : 128);
   const int p_max = r.R0 + r.nrows - 1;
   r.use_soft = mask_enable && (r.R0 < d.v0 + d.nv) && (p_max >= d.v0);
   int jmax = p_max;
@@ -104,12 +105,17 @@ __global__ void __launch_bounds__(SC_THREADS, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
              ScoreArgs a) {
   pdl_enter();
-  extern __shared__ uint8_t smem_raw[];
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_items = a.B * a.H;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  if ((base - smem_u32(smem_raw)) + SC_SMEM_MAIN + sizeof(ScoreBook) > (uint32_t)SC_SMEM_BYTES) {
+    // the tiles need a 1024-byte aligned start; the window is expected to provide it
+    if (threadIdx.x == 0) atomicOr(a.status, STATUS_SCORE_TIMEOUT);
+    return;
+  }
   const uint32_t q_smem = base;                          // two query tiles
   const uint32_t k_smem = base + 2 * SC_TILE_BYTES;      // ring of key tiles
   ScoreBook *bk = reinterpret_cast<ScoreBook *>(base_ptr + SC_SMEM_MAIN);
@@ -162,14 +168,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           if (!bk->abort_flag) {
             const uint32_t dst = q_smem + qb * SC_TILE_BYTES;
             mbar_expect_tx(smem_u32(&bk->q_full[qb]), SC_TILE_BYTES);
-            // four groups of 32 tile rows; with few ranking rows the groups repeat them, so that
-            // every 32-lane quarter of the accumulator (one per sub-partition) holds live rows
-#pragma unroll
-            for (int grp = 0; grp < 4; ++grp) {
-              const int src = d.row0 + T.R0 + (grp * 32) % T.tpad;
-              tma_load_2d(dst + grp * 4096, &tmap_q, smem_u32(&bk->q_full[qb]), h * 128, src);
-              tma_load_2d(dst + SC_HALF_BYTES + grp * 4096, &tmap_q, smem_u32(&bk->q_full[qb]), h * 128 + 64, src);
-            }
+            tma_load_2d(dst, &tmap_q, smem_u32(&bk->q_full[qb]), h * 128, d.row0 + T.R0);
+            tma_load_2d(dst + SC_HALF_BYTES, &tmap_q, smem_u32(&bk->q_full[qb]), h * 128 + 64, d.row0 + T.R0);
             q_issued = qc + 1;
           }
           for (int u = 0; u < T.n_kt + T.n_p2; ++u, ++kc) {
@@ -269,16 +269,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       }
       for (int rt = 0; rt < n_rt; ++rt) {
         const RowTile T = score_row_tile(d, rt, a.mask_enable);
-        // ---------------- pass 1: thread = ranking row, this group's share of the key tiles.
-        // Lane lrow holds copy (lrow / tpad) of row (lrow % tpad) and reduces that copy's share
-        // of each tile's 128 columns.
-        const int ncopy = 128 / T.tpad;
-        const int srow = lrow % T.tpad;                 // row of the tile this lane works for
-        const int ncols = 128 / ncopy;                  // columns of a tile this lane reduces
-        const int c_lo = (lrow / T.tpad) * ncols;
-        const bool row_ok = srow < T.nrows;
-        const bool warp_rows = ((quarter * 32) % T.tpad) < T.nrows;
-        const int p_i = T.R0 + srow;
+        // ---------------- pass 1: thread = ranking row, this group's share of the key tiles
+        const bool row_ok = lrow < T.nrows;
+        const bool warp_rows = quarter * 32 < T.nrows;
+        const int p_i = T.R0 + lrow;
         const bool row_vis = T.use_soft && p_i >= d.v0 && p_i < v_end;
         float m = -INFINITY, l = 0.f;
         for (int t = 0; t < T.n_kt; ++t, ++g) {
@@ -296,70 +290,62 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 2) & 1, wc);
           tc_fence_after();
           if (warp_rows) {
-            uint32_t ra[32], rb[32];
-            tmem_ld32(tlane + c_lo, ra);
 #pragma unroll 1
-            for (int c = c_lo; c < c_lo + ncols; c += 64) {
+            for (int c = 0; c < 128; c += 64) {
+              uint32_t r[64];
+              tmem_ld32p(tlane + c, r);
+              tmem_ld32p(tlane + c + 32, r + 32);
+              tmem_wait_ld();
+              if (fast) {
+                // every key admitted, no mask: max on the raw dot products (scale > 0), then
+                // exp2(dot * scale - max) into eight independent partial sums
+                float mx[8];
 #pragma unroll
-              for (int half = 0; half < 2; ++half) {
-                const int cc = c + half * 32;
-                if (cc < c_lo + ncols) {
-                  uint32_t (&r)[32] = half ? rb : ra;
-                  uint32_t (&rn)[32] = half ? ra : rb;
-                  tmem_wait_ld();
-                  if (cc + 32 < c_lo + ncols) tmem_ld32(tlane + cc + 32, rn);   // next chunk travels meanwhile
-                  if (fast) {
-                    // every key admitted, no mask: max on the raw dot products (scale > 0), then
-                    // exp2(dot * scale - max) into eight independent partial sums
-                    float mx[8];
+                for (int e = 0; e < 8; ++e) mx[e] = __uint_as_float(r[e]);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) mx[e] = __uint_as_float(r[e]);
+                for (int e = 8; e < 64; ++e) mx[e & 7] = fmaxf(mx[e & 7], __uint_as_float(r[e]));
+                const float cmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                const float m_new = fmaxf(m, cmax * scale);
+                if (row_ok) {
+                  float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int e = 8; e < 32; ++e) mx[e & 7] = fmaxf(mx[e & 7], __uint_as_float(r[e]));
-                    const float cmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                                             fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-                    const float m_new = fmaxf(m, cmax * scale);
-                    if (row_ok) {
-                      float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                  for (int e = 0; e < 64; ++e) sm[e & 7] += fast_exp2(fmaf(__uint_as_float(r[e]), scale, -m_new));
+                  l = l * fast_exp2(m - m_new) +
+                      (((sm[0] + sm[1]) + (sm[2] + sm[3])) + ((sm[4] + sm[5]) + (sm[6] + sm[7])));
+                  m = m_new;
+                }
+              } else {
+                // tile that crosses a row's own position: selects only, no branches.  `lim` =
+                // last column of this chunk the row may attend to without the soft mask
+                const int lim = p_i - (j0 + c);
+                float mx[8] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                if (!stage_soft) {
 #pragma unroll
-                      for (int e = 0; e < 32; ++e) sm[e & 7] += fast_exp2(fmaf(__uint_as_float(r[e]), scale, -m_new));
-                      l = l * fast_exp2(m - m_new) +
-                          (((sm[0] + sm[1]) + (sm[2] + sm[3])) + ((sm[4] + sm[5]) + (sm[6] + sm[7])));
-                      m = m_new;
-                    }
-                  } else {
-                    // tile that crosses a row's own position: selects only, no branches.  `lim` =
-                    // last column of this chunk the row may attend to without the soft mask
-                    const int lim = p_i - (j0 + cc);
-                    float mx[8] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                    if (!stage_soft) {
-#pragma unroll
-                      for (int e = 0; e < 32; ++e) {
-                        const float x = (e <= lim) ? __uint_as_float(r[e]) * scale : -INFINITY;
-                        r[e] = __float_as_uint(x);
-                        mx[e & 7] = fmaxf(mx[e & 7], x);
-                      }
-                    } else {
-#pragma unroll
-                      for (int e = 0; e < 32; ++e) {
-                        const float sv = row_vis ? soft[cc + e] : -INFINITY;
-                        const float x = fmaf(__uint_as_float(r[e]), scale, (e <= lim) ? 0.f : sv);
-                        r[e] = __float_as_uint(x);
-                        mx[e & 7] = fmaxf(mx[e & 7], x);
-                      }
-                    }
-                    const float cmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                                             fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-                    const float m_new = fmaxf(m, cmax);
-                    if (row_ok && m_new > -INFINITY) {
-                      float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                      for (int e = 0; e < 32; ++e) sm[e & 7] += fast_exp2(__uint_as_float(r[e]) - m_new);
-                      l = l * fast_exp2(m - m_new) +
-                          (((sm[0] + sm[1]) + (sm[2] + sm[3])) + ((sm[4] + sm[5]) + (sm[6] + sm[7])));
-                      m = m_new;
-                    }
+                  for (int e = 0; e < 64; ++e) {
+                    const float x = (e <= lim) ? __uint_as_float(r[e]) * scale : -INFINITY;
+                    r[e] = __float_as_uint(x);
+                    mx[e & 7] = fmaxf(mx[e & 7], x);
                   }
+                } else {
+#pragma unroll
+                  for (int e = 0; e < 64; ++e) {
+                    const float sv = row_vis ? soft[c + e] : -INFINITY;
+                    const float x = fmaf(__uint_as_float(r[e]), scale, (e <= lim) ? 0.f : sv);
+                    r[e] = __float_as_uint(x);
+                    mx[e & 7] = fmaxf(mx[e & 7], x);
+                  }
+                }
+                const float cmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                const float m_new = fmaxf(m, cmax);
+                if (row_ok && m_new > -INFINITY) {
+                  float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                  for (int e = 0; e < 64; ++e) sm[e & 7] += fast_exp2(__uint_as_float(r[e]) - m_new);
+                  l = l * fast_exp2(m - m_new) +
+                      (((sm[0] + sm[1]) + (sm[2] + sm[3])) + ((sm[4] + sm[5]) + (sm[6] + sm[7])));
+                  m = m_new;
                 }
               }
             }
@@ -369,26 +355,17 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
           if (stage_soft) group_bar_sync(group);   // soft[] is rewritten by this group's next masked tile
         }
-        // every (group, copy) saw a disjoint part of the keys: merge their (max, sum) per row, then
+        // the two groups saw disjoint key tiles: merge their (max, sum) per row, then
         // off_i = max_i + log2(sum_i), so that exp2(x - off_i) = exp2(x - max_i) / sum_i
-        bk->pm[group][lrow] = m;
-        bk->pl[group][lrow] = l;
+        if (group == 1) { bk->pm[lrow] = m; bk->pl[lrow] = l; }
         epi_bar_sync();
         if (group == 0) {
-          float off = INFINITY;
-          if (lrow < T.tpad && lrow < T.nrows) {
-            float mm = -INFINITY;
-            for (int gq = 0; gq < 2; ++gq)
-              for (int cp = 0; cp < ncopy; ++cp) mm = fmaxf(mm, bk->pm[gq][lrow + cp * T.tpad]);
-            float ll = 0.f;
-            for (int gq = 0; gq < 2; ++gq)
-              for (int cp = 0; cp < ncopy; ++cp) {
-                const float mi = bk->pm[gq][lrow + cp * T.tpad];
-                if (mi > -INFINITY) ll += bk->pl[gq][lrow + cp * T.tpad] * fast_exp2(mi - mm);
-              }
-            off = mm + __log2f(ll);
-          }
-          bk->off[lrow] = off;
+          const float m1 = bk->pm[lrow], l1 = bk->pl[lrow];
+          const float mm = fmaxf(m, m1);
+          float ll = 0.f;
+          if (m > -INFINITY) ll += l * fast_exp2(m - mm);
+          if (m1 > -INFINITY) ll += l1 * fast_exp2(m1 - mm);
+          bk->off[lrow] = row_ok ? (mm + __log2f(ll)) : INFINITY;
         }
         epi_bar_sync();
         // ---------------- pass 2: thread = key, this group's share of the visual key tiles
