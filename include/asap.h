@@ -36,6 +36,10 @@
  *   - bf16 tensors are row-major with the stated shapes and no padding.
  *   - A context serves one stream at a time: two calls on the same context that overlap on
  *     the GPU race on its scratch memory.
+ *   - asap_prune_step may enqueue two of its kernels (attention mass, salience) on a second
+ *     stream that belongs to the context, forked from and joined back into `stream` with
+ *     events inside the call: everything the call enqueues is ordered after the work already
+ *     in `stream`, and work enqueued in `stream` after the call is ordered after all of it.
  */
 #ifndef ASAP_H
 #define ASAP_H
