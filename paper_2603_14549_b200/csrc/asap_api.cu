@@ -49,7 +49,7 @@ struct asap_ctx {
   uint32_t *status = nullptr;
   EncodeTiledFn encode = nullptr;
   cudaStream_t side = nullptr;            // second stream for the mass kernels of asap_prune_step
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_desc = nullptr, ev_join = nullptr;
   uint64_t launches = 0;
   char err[512] = "";
   // per-kernel timing (asap_profile): one event before every launch, one at the end of a call
@@ -216,7 +216,8 @@ asap_status launch_prepare(asap_ctx *ctx, const asap_inputs *in, const asap_para
 // Steps 1a-1b: query sum, attention mass, salience, mask vector.  With `fold_prepare` the query-sum
 // kernel also carries the device-side validation and writes the descriptors.
 asap_status launch_mass(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const asap_outputs *out,
-                        bool fold_prepare, int32_t *out_cu, int out_capacity, cudaStream_t st) {
+                        bool fold_prepare, int32_t *out_cu, int out_capacity, cudaStream_t st,
+                        cudaEvent_t after_qsum = nullptr) {
   const int D = in->D, B = in->B;
   const int max_chunks = (in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS;
   const int col_blocks = (D + QSUM_COLS - 1) / QSUM_COLS;
@@ -227,6 +228,8 @@ asap_status launch_mass(asap_ctx *ctx, const asap_inputs *in, const asap_params 
              static_cast<const __nv_bfloat16 *>(in->q), pa, D, max_chunks, ctx->qsum_partial, ctx->qbar,
              ctx->cnt_qsum);
   ASAP_TRY(after_launch(ctx, "qsum"));
+  if (after_qsum && cudaEventRecord(after_qsum, st) != cudaSuccess)
+    return fail(ctx, ASAP_ERR_CUDA, "event after the query-sum kernel");
 
   const float scale = 1.0f / ((float)in->H * sqrtf((float)in->head_dim));
   const int row_blocks = (in->max_vis + MASS_ROWS - 1) / MASS_ROWS;
@@ -246,7 +249,7 @@ asap_status launch_rank(asap_ctx *ctx, const asap_inputs *in, const asap_params 
       !make_map(ctx, &map_k, in->k, (uint64_t)in->total_tokens, (uint64_t)D, 128))
     return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for q / k");
   ScoreArgs sa;
-  sa.desc = ctx->desc; sa.B = B; sa.H = in->H; sa.max_vis = in->max_vis; sa.mask_enable = p->mask_enable ? 1 : 0;
+  sa.pa = prepare_args(ctx, in, p, nullptr, 0x7fffffff); sa.pa.write_desc = 0; sa.B = B; sa.H = in->H; sa.max_vis = in->max_vis; sa.mask_enable = p->mask_enable ? 1 : 0;
   sa.scale_log2 = 1.4426950408889634f / sqrtf((float)in->head_dim);
   sa.mask_log = out->mask_log; sa.partial = ctx->score_partial; sa.status = ctx->status;
   mark(ctx, "score", st);
@@ -460,13 +463,19 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   if (e == cudaSuccess) e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
-  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
+  // lowest priority: when both streams have blocks to place, the score kernel's go first and the
+  // mass kernels fill what is left of each SM
+  int prio_least = 0, prio_greatest = 0;
+  if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest);
+  if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&ctx->side, cudaStreamNonBlocking, prio_least);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_desc, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    if (ctx->ev_desc) cudaEventDestroy(ctx->ev_desc);
     if (ctx->side) cudaStreamDestroy(ctx->side);
     cudaFree(ctx->arena);
     delete ctx;
@@ -525,15 +534,22 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
     ASAP_TRY(launch_select(ctx, in, p, out->rank_score, out, true, true, st));
     return finish(ctx, launch_merge(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st), st);
   }
-  ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
+  // stream:      [fork] score (derives its own descriptors) -> wait descriptors -> select -> gather -> sim
+  // side stream: qsum (carrying the validation) -> [descriptors ready] -> mass -> [join]
+  // The score kernel is enqueued first, so its one block per SM is placed before the mass kernels'
+  // many small blocks, which then fill what is left of each SM.
   cudaError_t e = cudaEventRecord(ctx->ev_fork, st);
-  if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0);
+  if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "fork event: %s", cudaGetErrorString(e));
+  asap_status main_status = launch_rank(ctx, in, p, out, false, st);
+  e = cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0);
   if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "fork to the side stream: %s", cudaGetErrorString(e));
-  asap_status side_status = launch_mass(ctx, in, p, out, false, nullptr, 0x7fffffff, ctx->side);
+  asap_status side_status = launch_mass(ctx, in, p, out, true, out->out_cu_seqlens, out->out_rows_capacity, ctx->side,
+                                        ctx->ev_desc);
   e = cudaEventRecord(ctx->ev_join, ctx->side);
   if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "join event: %s", cudaGetErrorString(e));
-  asap_status main_status = side_status;
-  if (main_status == ASAP_OK) main_status = launch_rank(ctx, in, p, out, false, st);
+  if (main_status == ASAP_OK) main_status = side_status;
+  if (main_status == ASAP_OK && cudaStreamWaitEvent(st, ctx->ev_desc, 0) != cudaSuccess)
+    main_status = fail(ctx, ASAP_ERR_CUDA, "wait for the descriptors");
   if (main_status == ASAP_OK) main_status = launch_select(ctx, in, p, out->rank_score, out, true, true, st);
   if (main_status == ASAP_OK) main_status = launch_merge_front(ctx, in, p, out->keep_idx, out, st);
   // the side stream always rejoins, also after an error, so that `stream` stays ordered behind it
@@ -716,6 +732,7 @@ void asap_free(asap_ctx *ctx) {
   if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
   if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+  if (ctx->ev_desc) cudaEventDestroy(ctx->ev_desc);
   cudaFree(ctx->arena);
   delete ctx;
 }

@@ -62,7 +62,8 @@ constexpr int SC_SMEM_BYTES = SC_SMEM_MAIN + SC_BOOK_BYTES;
 constexpr uint32_t SC_TMEM_COLS = 512;     // four accumulators of 128 columns
 
 struct ScoreArgs {
-  const SampleDesc *desc;
+  PrepareArgs pa;             // every block derives its descriptors itself: the kernel does not wait
+                              // for the validation kernel (it writes nothing but scratch)
   int B, H, max_vis, mask_enable;
   float scale_log2;           // log2(e) / sqrt(head_dim)
   const float *mask_log;      // [B, max_vis]  m_j (natural log)
@@ -158,7 +159,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                                                 // these are prefixes of the two sequences)
       for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
         const int b = item / a.H, h = item - b * a.H;
-        const SampleDesc d = a.desc[b];
+        const SampleDesc d = make_desc(a.pa, b);
         if (!d.valid) continue;
         const int n_rt = (d.nr + 127) / 128;
         for (int rt = 0; rt < n_rt; ++rt, ++qc) {
@@ -203,7 +204,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       const uint32_t idesc1 = umma_idesc_bf16(128, 128);
       for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
         const int b = item / a.H;
-        const SampleDesc d = a.desc[b];
+        const SampleDesc d = make_desc(a.pa, b);
         if (!d.valid) continue;
         const int n_rt = (d.nr + 127) / 128;
         for (int rt = 0; rt < n_rt; ++rt, ++qc) {
@@ -253,7 +254,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     int g = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
       const int b = item / a.H, h = item - b * a.H;
-      const SampleDesc d = a.desc[b];
+      const SampleDesc d = make_desc(a.pa, b);
       if (!d.valid) continue;
       const int n_rt = (d.nr + 127) / 128;
       float *part = a.partial + ((size_t)b * a.H + h) * a.max_vis;
