@@ -59,9 +59,7 @@ constexpr int SC_SMEM_MAIN = (2 + SC_STAGES) * SC_TILE_BYTES;
 // beside this one; one byte more selects the 228 KB carve-out and costs them about 10 us.
 constexpr int SC_BOOK_BYTES = 3072;
 constexpr int SC_SMEM_BYTES = SC_SMEM_MAIN + SC_BOOK_BYTES;
-constexpr uint32_t SC_TMEM_COLS = 512;     // three accumulators of 128 columns + two query tiles of 64
-constexpr int SC_ACC = 3;
-constexpr uint32_t SC_TMEM_Q = SC_ACC * 128;   // first column of the query tiles in tensor memory
+constexpr uint32_t SC_TMEM_COLS = 512;     // four accumulators of 128 columns
 
 struct ScoreArgs {
   PrepareArgs pa;             // every block derives its descriptors itself: the kernel does not wait
@@ -74,7 +72,7 @@ struct ScoreArgs {
 };
 
 struct ScoreBook {             // bookkeeping block placed after the tiles in shared memory
-  uint64_t full[SC_STAGES], empty[SC_STAGES], q_full[2], q_empty[2], acc_full[SC_ACC], acc_empty[SC_ACC];
+  uint64_t full[SC_STAGES], empty[SC_STAGES], q_full[2], q_empty[2], acc_full[4], acc_empty[4];
   float off[128];              // per ranking row: max + log2(sum), +inf for rows past the tile
   float soft[2][128];          // per epilogue group, per key of its current tile: m_j*log2(e) or -inf
   float pm[128], pl[128];      // group 1's running (max, sum) per row at the end of pass 1
@@ -132,7 +130,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       mbar_init(smem_u32(&bk->q_full[i]), 1);
       mbar_init(smem_u32(&bk->q_empty[i]), 1);
     }
-    for (int i = 0; i < SC_ACC; ++i) {
+    for (int i = 0; i < 4; ++i) {
       mbar_init(smem_u32(&bk->acc_full[i]), 1);
       mbar_init(smem_u32(&bk->acc_empty[i]), 4);
     }
@@ -216,20 +214,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           const int qb = qc & 1;
           const uint32_t qs = q_smem + qb * SC_TILE_BYTES;
           mbar_wait(smem_u32(&bk->q_full[qb]), (qc >> 1) & 1, wc);
-          // the query tile also goes to tensor memory (8 slices of 16 dims): pass 1 then fetches
-          // only the key tile from shared memory, which the incoming TMA copies compete for.
-          // Copies and MMAs of this thread run in order, and the two query regions alternate.
-          const uint32_t qt = tmem_base + SC_TMEM_Q + qb * 64;
-          tc_fence_after();
-          if (!bk->abort_flag) {
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-              tc_cp_128x256b(qt + kk * 8, umma_desc_sw128(qs + (kk >> 2) * SC_HALF_BYTES + (kk & 3) * 32));
-          }
           for (int u = 0; u < T.n_kt + T.n_p2; ++u, ++kc, ++g) {
             const bool pass1 = u < T.n_kt;
-            const int s = kc % SC_STAGES, buf = g % SC_ACC;
-            if (g >= SC_ACC) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((g / SC_ACC) - 1) & 1, wc);
+            const int s = kc % SC_STAGES, buf = g & 3;
+            if (g >= 4) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((g >> 2) - 1) & 1, wc);
             mbar_wait(smem_u32(&bk->full[s]), (kc / SC_STAGES) & 1, wc);
             tc_fence_after();
             if (!bk->abort_flag) {
@@ -239,7 +227,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
               for (int kk = 0; kk < 8; ++kk) {
                 const uint32_t o = (kk >> 2) * SC_HALF_BYTES + (kk & 3) * 32;
                 const uint64_t dq = umma_desc_sw128(qs + o), dk = umma_desc_sw128(ks + o);
-                if (pass1) tc_mma_bf16_ta(dcol, qt + kk * 8, dk, idesc1, kk > 0);
+                if (pass1) tc_mma_bf16(dcol, dq, dk, idesc1, kk > 0);
                 else       tc_mma_bf16(dcol, dk, dq, idesc2, kk > 0);
               }
               tc_commit(smem_u32(&bk->empty[s]));
@@ -252,8 +240,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------------ epilogue (2 groups x 4 warps)
-    // Group w takes every second operation of the linear sequence (operation g uses accumulator
-    // g mod 3, so the MMA issuer can run up to three operations ahead of the epilogue); the
+    // Group w owns accumulators w and w + 2, i.e. every second operation of the linear sequence
+    // (operation g uses accumulator g mod 4), so the MMA issuer can run two operations ahead; the
     // two groups share the four sub-partitions, so one group's exponentials overlap the other's
     // tensor-memory loads.  Warp q of a group reads tensor-memory lanes 32q .. 32q+31.
     const int group = (warp - 2) >> 2;
@@ -298,9 +286,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             soft[lrow] = (j >= d.v0 && j < v_end) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
             group_bar_sync(group);
           }
-          const int buf = g % SC_ACC;
+          const int buf = g & 3;
           const uint32_t tlane = tlane0 + buf * 128;
-          mbar_wait(smem_u32(&bk->acc_full[buf]), (g / SC_ACC) & 1, wc);
+          mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 2) & 1, wc);
           tc_fence_after();
           if (warp_rows) {
 #pragma unroll 1
@@ -391,9 +379,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           const bool fast = (j0 + 127 <= T.R0);
           const bool warp_keys = (j0 + quarter * 32 + 31 >= d.v0) && (j0 + quarter * 32 < v_end);
           const float soft_j = (T.use_soft && key_ok) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
-          const int buf = g % SC_ACC;
+          const int buf = g & 3;
           const uint32_t tlane = tlane0 + buf * 128;
-          mbar_wait(smem_u32(&bk->acc_full[buf]), (g / SC_ACC) & 1, wc);
+          mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 2) & 1, wc);
           tc_fence_after();
           if (warp_keys) {
             float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
