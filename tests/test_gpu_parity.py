@@ -141,6 +141,41 @@ def test_c4_prefix_sampled(ctx):
     print("c4 parity maxima", stats)
 
 
+@pytest.fixture(scope="module")
+def big_ctx():
+    """Capacity of the largest benchmark shape (64 sequences of 35 + 2880 + up to 256 tokens)."""
+    c = A.asap_init(0, max_total_tokens=64 * (35 + 2880 + 256), max_B=64, max_H=40, max_D=5120,
+                    max_keep_rows=64 * 1152)
+    yield c
+    A.asap_free(c)
+
+
+@pytest.mark.parametrize("k", [320, 160])
+def test_c3_full_size_sampled(big_ctx, k):
+    """The whole LLaVA-NeXT batch of 8 as bench.py runs it; the oracle checks two sequences."""
+    stats = {}
+    batch = W.config("c3", keep_k=k)
+    run_step(big_ctx, batch, A.Params(keep_k=k), samples=[0, 7], stats=stats)
+    print("c3 full parity maxima", stats)
+
+
+def test_c4_full_size_sampled(big_ctx):
+    """The AnyRes throughput shape at full size (64 sequences, 2880 visual tokens, ragged text up
+    to 256 rows = two ranking-row tiles); the oracle checks the first and the last sequence."""
+    stats = {}
+    batch = W.config("c4")
+    run_step(big_ctx, batch, A.Params(keep_k=batch.keep_k), samples=[0, 63], stats=stats)
+    print("c4 full parity maxima", stats)
+
+
+def test_c5_full_size_first_step_sampled(big_ctx):
+    """13B-shaped batch of 32 (D = 5120, 40 heads), first step 2304 -> 1152, at full size."""
+    stats = {}
+    batch = W.config("c5")
+    run_step(big_ctx, batch, A.Params(keep_k=batch.keep_k), samples=[31], stats=stats)
+    print("c5 full parity maxima", stats)
+
+
 def test_c5_progressive_three_steps(ctx):
     """13B-shaped schedule 2304 -> 1152 -> 576 -> 288: every step consumes the previous step's
     hidden states and gathered position ids, with Q/K re-drawn at those positions."""
