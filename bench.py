@@ -98,7 +98,7 @@ def algorithmic(batch, keep_k):
 # clocks
 # ------------------------------------------------------------------------------------------
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -111,40 +111,47 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Samples taken between the wall-clock times t_begin and t_end (the timed region); if
+        the region was too short to catch one, all samples of the run."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        time.sleep(0.15)
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, pw, reasons = [], [], [], set()
+        import datetime
+        rows = []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         try:
             with open(self.path) as f:
                 for line in f:
                     parts = [p.strip() for p in line.split(",")]
-                    if len(parts) < 7:
+                    if len(parts) < 8:
                         continue
                     try:
-                        sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+                        ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                        rows.append((ts, float(parts[1]), float(parts[2]), float(parts[3]),
+                                     [nm for nm, v in zip(names, parts[4:8]) if v.lower().startswith("active")]))
                     except ValueError:
                         continue
-                    for nm, v in zip(names, parts[3:7]):
-                        if v.lower().startswith("active"):
-                            reasons.add(nm)
             os.unlink(self.path)
         except OSError:
             pass
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons), "samples": len(sm)}
+        inside = [r for r in rows if t_begin is not None and t_begin <= r[0] <= t_end]
+        use = inside if inside else rows
+        reasons = sorted({nm for r in use for nm in r[4]})
+        return {"sm_mhz": statistics.median(r[1] for r in use) if use else None,
+                "sm_max_mhz": max(r[2] for r in use) if use else None,
+                "power_w_max": max(r[3] for r in use) if use else None, "reasons": reasons,
+                "samples": len(use), "samples_in_timed_region": len(inside)}
 
 
 # ------------------------------------------------------------------------------------------
@@ -246,21 +253,24 @@ def run_cuda(args):
         A.asap_prune_step(ctx, copies[i % n_copies], params, out, stream)
 
     # ---- device-resident timing
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     for i in range(args.warmup):
         step(i)
     torch.cuda.synchronize()
     A.asap_check(ctx)
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     launches0 = A.asap_launch_count(ctx)
     R.barrier(); torch.cuda.synchronize()
+    wall_begin = time.time()
     marks[0].record(stream)
     for i in range(args.steps):
         step(args.warmup + i)
         marks[i + 1].record(stream)
     torch.cuda.synchronize(); R.barrier()
+    wall_end = time.time()
+    clocks = sampler.stop(wall_begin, wall_end) if rank == 0 else None
     launches = A.asap_launch_count(ctx) - launches0
     total_ms = marks[0].elapsed_time(marks[-1])
     per_step = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
@@ -270,12 +280,11 @@ def run_cuda(args):
 
     # ---- per-kernel device times: the same steps again with the library's own events on
     A.asap_profile(ctx, True)
-    for i in range(args.steps):
+    for i in range(min(args.steps, 1000)):        # the library times at most 16384 events between reads
         step(args.warmup + i)
     torch.cuda.synchronize()
     ktimes = A.asap_profile_read(ctx)
     A.asap_profile(ctx, False)
-    clocks = sampler.stop() if rank == 0 else None
 
     # ---- end to end from pinned host memory
     e2e = None
@@ -300,7 +309,7 @@ def run_cuda(args):
             host_out["keep_idx"].copy_(out.keep_idx, non_blocking=True)
             stream.synchronize()            # the caller consumes the shortened batch every step
 
-        e_steps = max(3, min(args.steps, 20))
+        e_steps = max(3, min(args.steps, 30))
         for _ in range(3):
             e2e_step()
         R.barrier(); torch.cuda.synchronize()
@@ -380,7 +389,8 @@ def run_cuda(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps (default 2000 for the CUDA arm, 20 for --impl reference)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
@@ -391,6 +401,10 @@ def main():
                     help="--impl reference: sequences of the workload the oracle prunes per step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    if args.steps is None:
+        args.steps = 2000 if args.impl == "cuda" else 20
+    if args.impl == "reference" and args.steps > 100:
+        args.ref_sequences = 1          # many steps: the smallest sample, one sequence per step
     if args.impl == "reference":
         run_reference(args)
     else:
