@@ -286,6 +286,30 @@ def run_cuda(args):
     ktimes = A.asap_profile_read(ctx)
     A.asap_profile(ctx, False)
 
+    # ---- KV-cache compaction of the layers up to the pruning layer (next-row feature, timed apart
+    # from the step: keys and values of `kv_layers` layers gathered with the step's row map)
+    kv = None
+    if args.kv_layers > 0:
+        n_out = batch.total - units + batch.B * keep_k
+        n_t = 2 * args.kv_layers
+        kv_src = [torch.randn(batch.total, batch.D, device=device).to(torch.bfloat16) for _ in range(n_t)]
+        kv_dst = [torch.empty(out.out_hidden.shape[0], batch.D, dtype=torch.bfloat16, device=device) for _ in range(n_t)]
+        n_rows = out.out_cu_seqlens[batch.B:]
+        for _ in range(3):
+            A.asap_compact_kv(ctx, out.src_row, n_rows, kv_src, kv_dst, stream)
+        k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        k0.record(stream)
+        for _ in range(20):
+            A.asap_compact_kv(ctx, out.src_row, n_rows, kv_src, kv_dst, stream)
+        k1.record(stream)
+        torch.cuda.synchronize()
+        kv_us = k0.elapsed_time(k1) / 20 * 1e3
+        kv_bytes = 2 * n_out * batch.D * 2 * n_t
+        kv = {"layers": args.kv_layers, "tensors": n_t, "rows_out": n_out, "bytes": kv_bytes, "us": kv_us,
+              "GBs": kv_bytes / kv_us / 1e3, "frac_of_hbm_peak": kv_bytes / kv_us / 1e3 / peaks["hbm_gbs"]}
+        del kv_src, kv_dst
+
     # ---- end to end from pinned host memory
     e2e = None
     if not args.no_e2e:
@@ -380,7 +404,7 @@ def run_cuda(args):
         "latency_us": {"p10": per_step[len(per_step) // 10] * 1e3, "p50": per_step[len(per_step) // 2] * 1e3,
                        "p90": per_step[(len(per_step) * 9) // 10] * 1e3},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "kernels": kernels,
-        "cpu_baseline": cpu,
+        "cpu_baseline": cpu, "kv_compaction": kv,
     }
     print(json.dumps(line))
     R.shutdown()
@@ -395,6 +419,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--kv-layers", type=int, default=3,
+                    help="also time KV-cache compaction of this many layers (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--ref-sequences", type=int, default=2,

@@ -144,6 +144,22 @@ asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *
 asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                             const asap_outputs *out, void *stream);
 
+/* KV-cache compaction (the paper presents the method as KV-cache compatible, Sec. 1, and reports
+ * the key/value storage it saves, Sec. 5.5 / Table 4).  The decoder layers up to the pruning layer
+ * have already cached keys and values for every token of the prompt; after the prune step only
+ * the rows of the shortened sequence are needed.  For each of `n_tensors` (<= 64) row-major
+ * tensors of `src_rows` rows of `row_bytes` bytes (a multiple of 16; e.g. one layer's K or V,
+ * [total_tokens, kv_heads * head_dim]) this writes dst[t][r] = src[t][src_row[r]] for
+ * r < *n_rows, r < rows_capacity.  `src_row` and `n_rows` are DEVICE pointers: the row map
+ * written by asap_merge / asap_prune_step and the number of rows of the shortened batch
+ * (out_cu_seqlens + B); `src` and `dst` are HOST arrays of device pointers, 16-byte aligned,
+ * that must not overlap.  A map entry outside [0, src_rows) leaves its output row untouched.
+ * Position ids of the kept rows are the gathered ones of asap_outputs::out_pos, so rotary
+ * phases already baked into cached keys stay valid. */
+asap_status asap_compact_kv(asap_ctx *ctx, const int32_t *src_row, const int32_t *n_rows,
+                            int32_t rows_capacity, int32_t src_rows, size_t row_bytes, int32_t n_tensors,
+                            const void *const *src, void *const *dst, void *stream);
+
 /* Reads the device status word (one 4-byte copy after synchronising `stream`).  ASAP_OK, or
  * ASAP_ERR_DEVICE with the reason in asap_last_error; the word is cleared. */
 asap_status asap_check(asap_ctx *ctx, void *stream);

@@ -18,6 +18,7 @@ Parity status of each function (what pins it, see tests/test_oracle_pins.py):
   select_topk           pinned  (hand-enumerated ties; library stable sort)
   cosine_assign         pinned  (library cosine similarity; hand-worked vectors)
   weighted_merge        pinned  (hand-worked fixture; convexity; weight conservation)
+  compact_rows          pinned  (library fancy indexing; identity and reversal maps)
   compact / prune_step  pinned  (invariants: k kept ascending; identity at k = N_v;
                                  plain attention top-k with mask and merge off; twins)
   Not pinned by anything the paper prints: that the ranking rule (mean of the Eq. 4
@@ -262,6 +263,15 @@ def prune_sample(q_bits, k_bits, hidden_bits, pos_ids, v0: int, nv: int, r0: int
                 assign=assign, best_sim=best, margin=margin, merged=merged,
                 out_hidden=out_hidden, out_hidden_bits=out_bits,
                 out_pos=np.asarray(pos_ids)[src_row].astype(np.int32), src_row=src_row)
+
+
+def compact_rows(cache: np.ndarray, src_row: np.ndarray) -> np.ndarray:
+    """KV-cache compaction after the hand-off: the cached key / value row of every surviving token,
+    in the order of the shortened sequence (row r of the result is row src_row[r] of the cache)."""
+    out = np.empty((len(src_row),) + cache.shape[1:], dtype=cache.dtype)
+    for r, sr in enumerate(src_row):
+        out[r] = cache[int(sr)]
+    return out
 
 
 def prune_batch(q_bits, k_bits, hidden_bits, pos_ids, cu_seqlens, vis_start, vis_len,

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "ASAP_OK", -1: "ASAP_ERR_INVALID", -2: "ASAP_ERR_ALIGN", -3: 
                 -4: "ASAP_ERR_CUDA", -5: "ASAP_ERR_UNSUPPORTED", -6: "ASAP_ERR_DEVICE"}
 
 EXPORTS = ("asap_init", "asap_score", "asap_select", "asap_merge", "asap_prune_step", "asap_check",
-           "asap_last_error", "asap_launch_count", "asap_free", "asap_profile", "asap_profile_read", "asap_select_static")
+           "asap_last_error", "asap_launch_count", "asap_free", "asap_profile", "asap_profile_read", "asap_select_static", "asap_compact_kv")
 
 
 class AsapError(RuntimeError):
@@ -87,6 +87,9 @@ def load_library() -> C.CDLL:
     lib.asap_select_static.restype = C.c_int
     lib.asap_select_static.argtypes = [C.POINTER(CInputs), C.POINTER(CParams), C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.asap_compact_kv.restype = C.c_int
+    lib.asap_compact_kv.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_size_t, C.c_int32,
+                                    C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.c_void_p]
     lib.asap_check.restype = C.c_int
     lib.asap_check.argtypes = [C.c_void_p, C.c_void_p]
     lib.asap_last_error.restype = C.c_char_p
@@ -261,6 +264,18 @@ def asap_merge(ctx, inp: Inputs, params: Params, salience: torch.Tensor, keep_id
 def asap_prune_step(ctx, inp: Inputs, params: Params, out: Outputs, stream=None) -> None:
     ci, cp, co = inp.c_struct(), params.c_struct(), out.c_struct()
     _raise(ctx, load_library().asap_prune_step(ctx, C.byref(ci), C.byref(cp), C.byref(co), _stream(stream)))
+
+
+def asap_compact_kv(ctx, src_row: torch.Tensor, n_rows: torch.Tensor, src, dst, stream=None) -> None:
+    """dst[t][r] = src[t][src_row[r]] for r < n_rows[0]: `src` / `dst` are equally long lists of 2-D device
+    tensors (rows x anything, contiguous); `n_rows` is a one-element int32 device tensor (or a view
+    such as out_cu_seqlens[B:])."""
+    assert len(src) == len(dst) and len(src) > 0
+    row_bytes = src[0][0].numel() * src[0].element_size()
+    ps = (C.c_void_p * len(src))(*[t.data_ptr() for t in src])
+    pd = (C.c_void_p * len(dst))(*[t.data_ptr() for t in dst])
+    _raise(ctx, load_library().asap_compact_kv(ctx, _ptr(src_row), _ptr(n_rows), int(min(dst[0].shape[0], src_row.numel())),
+                                               int(src[0].shape[0]), int(row_bytes), len(src), ps, pd, _stream(stream)))
 
 
 def asap_check(ctx, stream=None) -> None:

@@ -559,6 +559,34 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
   return finish(ctx, launch_merge_back(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st), st);
 }
 
+asap_status asap_compact_kv(asap_ctx *ctx, const int32_t *src_row, const int32_t *n_rows, int32_t rows_capacity,
+                            int32_t src_rows, size_t row_bytes, int32_t n_tensors, const void *const *src,
+                            void *const *dst, void *stream) {
+  if (!ctx) return fail(nullptr, ASAP_ERR_INVALID, "null context");
+  ctx->err[0] = 0;
+  if (!src_row || !n_rows || !src || !dst) return fail(ctx, ASAP_ERR_INVALID, "asap_compact_kv: null argument");
+  if (rows_capacity <= 0 || src_rows <= 0) return fail(ctx, ASAP_ERR_INVALID, "asap_compact_kv: row counts must be positive");
+  if (n_tensors <= 0 || n_tensors > KV_MAX_TENSORS)
+    return fail(ctx, ASAP_ERR_UNSUPPORTED, "asap_compact_kv: 1 .. %d tensors per call", KV_MAX_TENSORS);
+  if (row_bytes == 0 || row_bytes % 16 != 0 || row_bytes / 16 > 0x7fffffff)
+    return fail(ctx, ASAP_ERR_ALIGN, "asap_compact_kv: row_bytes must be a positive multiple of 16");
+  GatherArgs ga;
+  for (int i = 0; i < n_tensors; ++i) {
+    if (!src[i] || !dst[i]) return fail(ctx, ASAP_ERR_INVALID, "asap_compact_kv: null tensor %d", i);
+    if (!aligned16(src[i]) || !aligned16(dst[i]))
+      return fail(ctx, ASAP_ERR_ALIGN, "asap_compact_kv: tensor %d is not 16-byte aligned", i);
+    ga.src[i] = src[i];
+    ga.dst[i] = dst[i];
+  }
+  ga.src_row = src_row; ga.n_rows = n_rows; ga.rows_capacity = rows_capacity; ga.src_rows = src_rows;
+  ga.row_vecs = (int32_t)(row_bytes / 16);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  mark(ctx, "gather_rows", st);
+  launch_pdl(gather_rows_kernel, dim3((rows_capacity + KV_THREADS / 32 - 1) / (KV_THREADS / 32), n_tensors),
+             dim3(KV_THREADS), 0, st, ga);
+  return finish(ctx, after_launch(ctx, "gather_rows"), st);
+}
+
 asap_status asap_check(asap_ctx *ctx, void *stream) {
   if (!ctx) return fail(nullptr, ASAP_ERR_INVALID, "null context");
   cudaStream_t st = static_cast<cudaStream_t>(stream);

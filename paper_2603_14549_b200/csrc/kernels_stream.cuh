@@ -7,6 +7,7 @@
 //   kept_gather    kept rows gathered for the similarity GEMM, with their inverse norms (Sec. 4.2)
 //   csr_block      dropped tokens grouped by destination slot (tail of the similarity kernel)
 //   merge_compact  Eq. 5 and the hand-off of Fig. 3
+//   gather_rows    KV-cache compaction with the row map of the hand-off
 #pragma once
 
 #include "common.cuh"
@@ -781,6 +782,43 @@ merge_compact_kernel(MergeArgs a) {
         dst[v] = o;
       }
     }
+  }
+}
+
+// =======================================================================================
+// gather_rows: KV-cache compaction.  Output row r of every tensor is input row src_row[r] (the
+// row map the prune step wrote); one warp per (row, tensor), 16-byte vectors, eight in flight.
+// Rows at or past *n_rows (a device-side count, e.g. out_cu_seqlens[B]) are left untouched.
+// =======================================================================================
+constexpr int KV_MAX_TENSORS = 64;
+constexpr int KV_THREADS = 256;
+
+struct GatherArgs {
+  const void *src[KV_MAX_TENSORS];
+  void *dst[KV_MAX_TENSORS];
+  const int32_t *src_row;
+  const int32_t *n_rows;      // device scalar
+  int32_t rows_capacity, src_rows, row_vecs;   // row_vecs = row bytes / 16
+};
+
+__global__ void __launch_bounds__(KV_THREADS)
+gather_rows_kernel(GatherArgs a) {
+  pdl_enter();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (KV_THREADS / 32) + warp;
+  if (r >= a.rows_capacity || r >= *a.n_rows) return;
+  const int sr = a.src_row[r];
+  if (sr < 0 || sr >= a.src_rows) return;                 // not a valid source row: leave the output row alone
+  const uint4 *src = reinterpret_cast<const uint4 *>(a.src[blockIdx.y]) + (size_t)sr * a.row_vecs;
+  uint4 *dst = reinterpret_cast<uint4 *>(a.dst[blockIdx.y]) + (size_t)r * a.row_vecs;
+  for (int v = lane; v < a.row_vecs; v += 32 * 8) {
+    uint4 x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (v + 32 * u < a.row_vecs) x[u] = __ldg(src + v + 32 * u);
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (v + 32 * u < a.row_vecs) dst[v + 32 * u] = x[u];
   }
 }
 

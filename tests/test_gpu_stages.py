@@ -199,3 +199,30 @@ def test_repeated_calls_are_deterministic(ctx):
         for name in ("mass", "salience", "rank_score", "keep_idx", "assign", "out_pos"):
             assert torch.equal(getattr(o, name), getattr(outs[0], name)), name
         assert torch.equal(o.out_hidden.view(torch.int16), outs[0].out_hidden.view(torch.int16))
+
+
+def test_kv_cache_compaction_follows_the_row_map(ctx):
+    """asap_compact_kv gathers cached K / V rows with the step's own row map: bit-exact against the
+    oracle's row gather, rows past the shortened batch untouched, several tensors per call."""
+    batch = W.tiny(B=3, n_vis=[90, 140, 64], text_lens=[5, 9, 2], H=2, keep_k=20, seed=308)
+    inp = A.make_inputs(batch, DEV)
+    p = A.Params(keep_k=20)
+    out = A.alloc_outputs(inp, 20, fill=True)
+    A.asap_prune_step(ctx, inp, p, out)
+    g = torch.Generator().manual_seed(9)
+    kv_dim = 2 * 128
+    caches = [torch.randint(-30000, 30000, (batch.total, kv_dim), generator=g, dtype=torch.int16).view(torch.bfloat16)
+              for _ in range(6)]                                   # K and V of three layers
+    src = [c.to(DEV) for c in caches]
+    rows_cap = out.out_hidden.shape[0]
+    dst = [torch.full((rows_cap, kv_dim), 7.0, dtype=torch.bfloat16, device=DEV) for _ in range(6)]
+    A.asap_compact_kv(ctx, out.src_row, out.out_cu_seqlens[batch.B:], src, dst)
+    torch.cuda.synchronize(); A.asap_check(ctx)
+    n_out = int(out.out_cu_seqlens[-1])
+    rowmap = out.src_row[:n_out].cpu().numpy()
+    for c, d in zip(caches, dst):
+        want = O.compact_rows(bits(c), rowmap)
+        assert np.array_equal(bits(d[:n_out].cpu()), want)
+        assert torch.all(d[n_out:] == 7.0)                          # capacity tail untouched
+    with pytest.raises(A.AsapError):                                # 65 tensors: refused before any launch
+        A.asap_compact_kv(ctx, out.src_row, out.out_cu_seqlens[batch.B:], src * 11, dst * 11)

@@ -459,3 +459,15 @@ def test_planted_slip_is_caught(label, patch, checks):
         except AssertionError:
             caught += 1
     assert caught >= 1, f"no pin noticed: {label}"
+
+
+# ----------------------------------------------------------------------------- KV-cache compaction
+def test_compact_rows_is_a_row_gather():
+    rng = np.random.default_rng(11)
+    cache = rng.integers(0, 65535, size=(23, 6)).astype(np.uint16)
+    src = np.array([0, 1, 2, 7, 9, 15, 21, 22], dtype=np.int32)
+    got = O.compact_rows(cache, src)
+    assert np.array_equal(got, cache[src])                          # library fancy indexing
+    assert np.array_equal(O.compact_rows(cache, np.arange(23)), cache)            # identity map
+    assert np.array_equal(O.compact_rows(cache, np.arange(23)[::-1]), cache[::-1])  # reversal
+    assert got.dtype == cache.dtype and got.shape == (8, 6)
