@@ -299,13 +299,18 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     // two blocks per SM.
     const int max_mt = (in->max_vis + 127) / 128;
     const int n_kb = D / 128;
+    // The slice count minimises a simple cost: streaming a row tile takes about 1 us per 128-column
+    // step of the slice, and the last slice adds up keep_k * slices partial values per row at about
+    // 0.5 us per 64 of them.
     int splits = 1;
+    float best_cost = (float)n_kb;
     for (int c = 2; c <= 8; ++c) {
       if (n_kb % c != 0) continue;
       if ((long long)max_mt * B * c > 2LL * ctx->num_sms) break;
       if ((size_t)B * max_mt * c * ((size_t)k + 1) * 128 * sizeof(float) > ctx->sim_part_bytes) break;
       if ((size_t)B * max_mt > ctx->cap_tiles) break;
-      splits = c;
+      const float cost = (float)n_kb / c + 0.5f * (float)k * c / 64.f;
+      if (cost < best_cost) { best_cost = cost; splits = c; }
     }
     // a grid between one and two blocks per SM runs as one wave if two blocks fit on an SM:
     // give each block half of the shared memory and of the tensor memory then

@@ -721,16 +721,16 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
           float acc[16];
 #pragma unroll
           for (int e = 0; e < 16; ++e) acc[e] = 0.f;
-          for (int zz = 0; zz < a.splits; zz += 2) {
-            float x[2][16];
+          for (int zz = 0; zz < a.splits; zz += 4) {    // 64 loads in flight per thread
+            float x[4][16];
 #pragma unroll
-            for (int t = 0; t < 2; ++t)
+            for (int t = 0; t < 4; ++t)
 #pragma unroll
               for (int e = 0; e < 16; ++e)
                 x[t][e] = (zz + t < a.splits && s0 + e < a.keep_k)
                               ? __ldcg(p0 + (zz + t) * zstride + (size_t)(s0 + e) * 128) : 0.f;
 #pragma unroll
-            for (int t = 0; t < 2; ++t)
+            for (int t = 0; t < 4; ++t)
 #pragma unroll
               for (int e = 0; e < 16; ++e) acc[e] += x[t][e];
           }
