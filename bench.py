@@ -64,7 +64,7 @@ def load_peaks():
 # ------------------------------------------------------------------------------------------
 # algorithmic traffic / work of each kernel for one launch over the whole batch
 # ------------------------------------------------------------------------------------------
-def algorithmic(batch, keep_k):
+def algorithmic(batch, keep_k, rank_visual=False):
     """Bytes each kernel must move and flops it must do, from the problem sizes alone:
     every operand it consumes read once, every result written once (bf16 = 2 bytes)."""
     D = batch.D
@@ -83,6 +83,10 @@ def algorithmic(batch, keep_k):
         # ranking rows = text span: queries once, every key they may attend to once
         out["score"]["bytes"] += tl * row + (t0 + tl) * row + nv * 4
         out["score"]["flops"] += 2 * tl * (t0 + (tl + 1) // 2) * D
+        if rank_visual:     # image span ranked too: its rows see the prefix and, through Eq. 3, every visual key
+            v0 = int(batch.vis_start[b])
+            out["score"]["bytes"] += nv * row
+            out["score"]["flops"] += 2 * nv * (v0 + nv) * D
         out["select"]["bytes"] += nv * 4 + nv * 4
         out["head_sum"]["bytes"] += batch.H * nv * 4 + nv * 4
         out["kept_gather"]["bytes"] += 2 * keep_k * row
@@ -249,6 +253,14 @@ def run_cuda(args):
     out = A.alloc_outputs(copies[0], keep_k)
     stream = torch.cuda.current_stream()
 
+    rank_visual = args.rank_rows == "visual+text"
+    if rank_visual:       # Eq. 3 acts on these rows; the score kernel becomes a dense, tensor-pipe-heavy pass
+        import dataclasses
+        rs = batch.vis_start.to(device)
+        rl = (batch.vis_len + batch.text_len).to(device)
+        copies = [dataclasses.replace(c, rank_start=rs, rank_len=rl, max_rank=int((batch.vis_len + batch.text_len).max()))
+                  for c in copies]
+
     def step(i):
         A.asap_prune_step(ctx, copies[i % n_copies], params, out, stream)
 
@@ -354,7 +366,7 @@ def run_cuda(args):
         return
 
     # ---- roofline of the dominant kernel
-    alg = algorithmic(batch, keep_k)
+    alg = algorithmic(batch, keep_k, rank_visual)
     ksum = sum(ms for _, ms in ktimes.values()) or 1.0
     kernels = {}
     for name, (n, ms) in sorted(ktimes.items(), key=lambda kv: -kv[1][1]):
@@ -369,7 +381,7 @@ def run_cuda(args):
         a, kt = alg[top], kernels[top]
         hbm_frac = kt["alg_GBs"] / peaks["hbm_gbs"]
         tc_frac = kt["alg_TFLOPs"] / peaks["bf16_tflops"]
-        if top == "sim" and tc_frac > hbm_frac:
+        if top in ("sim", "score") and tc_frac > hbm_frac:
             roofline = {"kernel": top, "bound": "tensor", "achieved": kt["alg_TFLOPs"], "peak": peaks["bf16_tflops"],
                         "unit": "TFLOP/s", "frac": tc_frac, "traffic": None, "peak_kind": peak_kind + " (burst)"}
         else:
@@ -379,7 +391,7 @@ def run_cuda(args):
         roofline["algorithmic_flops_per_launch"] = a["flops"]
         roofline["avg_launch_us"] = kt["avg_us"]
         traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-        if os.path.exists(traffic_path):       # DRAM bytes per launch from the committed ncu capture
+        if os.path.exists(traffic_path) and not rank_visual:   # DRAM bytes per launch from the committed ncu capture
             with open(traffic_path) as f:
                 tr = json.load(f).get(args.workload, {}).get(top)
             roofline["traffic"] = tr
@@ -397,7 +409,7 @@ def run_cuda(args):
         "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}", "sequences_per_gpu": batch.B,
-                   "visual_tokens_per_gpu": units, "keep_k": keep_k, "ranking_rows": "text span",
+                   "visual_tokens_per_gpu": units, "keep_k": keep_k, "ranking_rows": "image span + text span" if rank_visual else "text span",
                    "l2": f"inputs rotate over {n_copies} device copies ({n_copies * in_bytes / 2**20:.0f} MiB) "
                          f"so no step finds its inputs in the {L2_BYTES // 2**20} MiB L2",
                    "parallelism": "replicas only (one batch per GPU, no collective)"},
@@ -418,6 +430,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--rank-rows", default="text", choices=["text", "visual+text"],
+                    help="query rows whose Eq. 4 probabilities rank the visual keys (default: the text span)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--kv-layers", type=int, default=3,
                     help="also time KV-cache compaction of this many layers (0 = skip)")
