@@ -19,6 +19,12 @@ Parity status of each function (what pins it, see tests/test_oracle_pins.py):
   cosine_assign         pinned  (library cosine similarity; hand-worked vectors)
   weighted_merge        pinned  (hand-worked fixture; convexity; weight conservation)
   compact_rows          pinned  (library fancy indexing; identity and reversal maps)
+  route_within_kept /
+  refill_from_pruned /
+  consolidate_sample    pinned  (hand-worked fixture; t >= 1 -> nothing merges and the output is the
+                                 plain top-k gather; twins; anchors are never absorbed; set sizes;
+                                 Eq. 5 weight conservation; library sort for the refill).  Not pinned
+                                 by the paper: the reading of which anchor absorbs a token.
   compact / prune_step  pinned  (invariants: k kept ascending; identity at k = N_v;
                                  plain attention top-k with mask and merge off; twins)
   Not pinned by anything the paper prints: that the ranking rule (mean of the Eq. 4
@@ -262,6 +268,102 @@ def prune_sample(q_bits, k_bits, hidden_bits, pos_ids, v0: int, nv: int, r0: int
     return dict(mass=s, salience=s_hat, mask_log=m, rank_score=r, keep_idx=keep, drop_idx=drop,
                 assign=assign, best_sim=best, margin=margin, merged=merged,
                 out_hidden=out_hidden, out_hidden_bits=out_bits,
+                out_pos=np.asarray(pos_ids)[src_row].astype(np.int32), src_row=src_row)
+
+
+# ----------------------------------------------------------------------------------
+# Stage 2 as Sec. 4.2 states it: consolidation INSIDE the kept set, then budget reallocation
+# ----------------------------------------------------------------------------------
+def route_within_kept(hv: np.ndarray, s_hat: np.ndarray, keep: np.ndarray, threshold: float):
+    """Salience-anchored routing of Sec. 4.2 among the kept tokens.
+
+    A token j may be absorbed by a token i only if S_ij > t and i comes before j in the order
+    (s_hat descending, sequence index ascending) -- the paper's "s_hat_i >= s_hat_j, ties by
+    sequence index".  Reading taken for what the paper leaves open (which i, and whether an
+    absorbed token can absorb): the kept tokens are visited in that order; a token joins the
+    most similar token among those that were NOT absorbed before it (the anchors), lowest
+    sequence index among equally similar ones, provided that similarity exceeds t; otherwise it
+    becomes an anchor itself.  Source sets are therefore disjoint and end at anchors.
+
+    Returns (dest [k]: slot of the absorbing anchor, -1 for anchors; margin [k]: how far the
+    decision of each token was from flipping: distance of its best similarity from t, and from
+    the runner-up anchor's)."""
+    k = len(keep)
+    S = cosine_matrix(hv[keep], hv[keep])
+    order = sorted(range(k), key=lambda p: (-s_hat[keep[p]], int(keep[p])))
+    dest = np.full(k, -1, dtype=np.int32)
+    margin = np.full(k, np.inf)
+    anchors = []
+    for p in order:
+        best, best_a, second = -np.inf, -1, -np.inf
+        for a in sorted(anchors):                 # ascending slot = ascending sequence index
+            v = S[a, p]
+            if v > best:
+                second, best, best_a = best, v, a
+            elif v > second:
+                second = v
+        if best_a >= 0:
+            margin[p] = min(abs(best - threshold), best - second)
+        if best_a >= 0 and best > threshold:
+            dest[p] = best_a
+        else:
+            anchors.append(p)
+    return dest, margin
+
+
+def refill_from_pruned(mass: np.ndarray, drop: np.ndarray, n: int) -> np.ndarray:
+    """Budget reallocation of Sec. 4.2: the n pruned tokens of largest attention mass s_j (Eq. 1),
+    lower index first among equals; returned in ascending index order."""
+    if n == 0:
+        return np.zeros(0, dtype=np.int32)
+    order = np.lexsort((drop, -mass[drop]))
+    return np.sort(drop[order[:n]]).astype(np.int32)
+
+
+def consolidate_sample(hidden_bits, pos_ids, v0: int, nv: int, mass, s_hat, keep, drop, threshold: float,
+                       eps: float = EPS_DEFAULT, dest_override=None, refill_override=None):
+    """Sec. 4.2 on one sequence, given stage 1's outputs (mass s, salience s_hat, kept / pruned
+    lists): routing inside the kept set, Eq. 5 at every anchor (sources added in ascending
+    sequence index), refill of the vacated slots from the pruned pool by s_j, hand-off."""
+    hid = bf16_bits_to_f64(hidden_bits)
+    hv = hid[v0:v0 + nv]
+    n = hid.shape[0]
+    dest, margin = route_within_kept(hv, s_hat, keep, threshold)
+    if dest_override is not None:
+        dest = np.asarray(dest_override, dtype=np.int32)
+    absorbed = np.nonzero(dest >= 0)[0]
+    anchors = np.nonzero(dest < 0)[0]
+    refill = refill_from_pruned(mass, drop, len(absorbed))
+    if refill_override is not None:
+        refill = np.asarray(refill_override, dtype=np.int32)
+    final = np.sort(np.concatenate([keep[anchors], refill])).astype(np.int32)
+    rows = np.empty((len(final), hv.shape[1]))
+    merged_mask = np.zeros(len(final), dtype=bool)
+    slot_of = {int(v): i for i, v in enumerate(final)}
+    for i, v in enumerate(final):
+        rows[i] = hv[v]
+    for a in anchors:
+        src = [int(keep[p]) for p in absorbed if dest[p] == a]          # ascending: keep is ascending
+        if not src:
+            continue
+        i = int(keep[a])
+        num = s_hat[i] * hv[i]
+        den = s_hat[i]
+        for j in src:
+            num = num + s_hat[j] * hv[j]
+            den = den + s_hat[j]
+        if den > eps:
+            rows[slot_of[i]] = num / den
+            merged_mask[slot_of[i]] = True
+    src_row = np.concatenate([np.arange(0, v0), v0 + final, np.arange(v0 + nv, n)]).astype(np.int32)
+    out_hidden = np.concatenate([hid[:v0], rows, hid[v0 + nv:]], axis=0)
+    out_bits = f64_to_bf16_bits(out_hidden)
+    out_bits[:v0] = hidden_bits[:v0]
+    out_bits[v0 + len(final):] = hidden_bits[v0 + nv:]
+    unmerged = np.nonzero(~merged_mask)[0]
+    out_bits[v0 + unmerged] = hidden_bits[v0 + final[unmerged]]        # pure copies keep their bits
+    return dict(dest=dest, margin=margin, n_absorbed=len(absorbed), refill=refill, final_keep=final,
+                merged=rows, merged_mask=merged_mask, out_hidden=out_hidden, out_hidden_bits=out_bits,
                 out_pos=np.asarray(pos_ids)[src_row].astype(np.int32), src_row=src_row)
 
 

@@ -471,3 +471,129 @@ def test_compact_rows_is_a_row_gather():
     assert np.array_equal(O.compact_rows(cache, np.arange(23)), cache)            # identity map
     assert np.array_equal(O.compact_rows(cache, np.arange(23)[::-1]), cache[::-1])  # reversal
     assert got.dtype == cache.dtype and got.shape == (8, 6)
+
+
+# ----------------------------------------------------------------------------- Sec. 4.2 inside the kept set
+def check_hand_consolidation(o):
+    g = GOLD["consolidate_within_kept"]
+    h = np.array(g["h"], float)
+    s_hat, mass = np.array(g["s_hat"]), np.array(g["mass"], float)
+    keep, drop = np.array(g["keep"]), np.array(g["drop"])
+    dest, _ = o.route_within_kept(h, s_hat, keep, g["t"])
+    assert dest.tolist() == g["dest"]
+    assert o.refill_from_pruned(mass, drop, 3).tolist() == g["refill"]
+    hb = bits(torch.tensor(h, dtype=torch.float32).to(torch.bfloat16))
+    r = o.consolidate_sample(hb, np.arange(10), 0, 10, mass, s_hat, keep, drop, g["t"])
+    assert r["final_keep"].tolist() == g["final_keep"] and r["n_absorbed"] == 3
+    for slot, row in g["merged_rows"].items():
+        assert np.allclose(r["merged"][int(slot)], row, rtol=1e-15)
+    assert r["merged_mask"].tolist() == [True, True, False, False, False]
+    assert np.array_equal(r["out_hidden_bits"][2:], hb[[4, 6, 7]])          # refilled rows are copies
+
+
+def test_hand_consolidation_within_kept():
+    check_hand_consolidation(O)
+
+
+def _clustered(n, D, centres, seed, spread=0.25):
+    rng = np.random.default_rng(seed)
+    c = rng.standard_normal((centres, D))
+    h = c[rng.integers(0, centres, n)] + spread * rng.standard_normal((n, D))
+    hb = bits(torch.tensor(h, dtype=torch.float32).to(torch.bfloat16))
+    return O.bf16_bits_to_f64(hb), hb, rng
+
+
+def test_refill_matches_library_sort():
+    rng = np.random.default_rng(21)
+    mass = np.round(rng.uniform(0, 1, 200), 1)                         # many exact ties
+    drop = np.sort(rng.choice(200, 120, replace=False))
+    for n in (0, 1, 37, 120):
+        want = np.sort(drop[np.argsort(-mass[drop], kind="stable")[:n]])
+        assert np.array_equal(O.refill_from_pruned(mass, drop, n), want)
+
+
+def test_routing_invariants_against_library_cosine():
+    """What the rules of Sec. 4.2 force, checked with torch's cosine similarity: an absorbed token's
+    anchor is itself not absorbed, precedes it in (s_hat desc, index asc), is more similar than t
+    and at least as similar as any other anchor that precedes it; two anchors are never more
+    similar than t in the direction the order allows."""
+    h, hb, rng = _clustered(160, 24, 9, 22)
+    s_hat = np.round(rng.uniform(0, 1, 160), 2)                        # ties exercise the index rule
+    keep = np.sort(rng.choice(160, 70, replace=False))
+    t = 0.8
+    dest, _ = O.route_within_kept(h, s_hat, keep, t)
+    S = torch.nn.functional.cosine_similarity(torch.from_numpy(h[keep])[:, None], torch.from_numpy(h[keep])[None], dim=-1).numpy()
+    before = lambda a, p: (s_hat[keep[a]], -keep[a]) > (s_hat[keep[p]], -keep[p])
+    anchors = [p for p in range(70) if dest[p] < 0]
+    assert 0 < len(anchors) < 70
+    for p in range(70):
+        cands = [a for a in anchors if before(a, p)]
+        if dest[p] >= 0:
+            a = dest[p]
+            assert dest[a] < 0 and before(a, p) and S[a, p] > t
+            assert all(S[a, p] >= S[c, p] - 1e-12 for c in cands)
+        else:
+            assert all(S[c, p] <= t + 1e-12 for c in cands)
+
+
+def test_consolidation_special_cases():
+    h, hb, rng = _clustered(120, 16, 5, 23)
+    s_hat, mass = rng.uniform(0, 1, 120), rng.uniform(0, 5, 120)
+    keep = np.sort(rng.choice(120, 40, replace=False)); drop = np.setdiff1d(np.arange(120), keep)
+    pos = np.arange(1000, 1120)
+    # t >= 1: nothing can be absorbed; the step is the plain gather of the kept rows
+    r = O.consolidate_sample(hb, pos, 0, 120, mass, s_hat, keep, drop, 1.0)
+    assert r["n_absorbed"] == 0 and np.array_equal(r["final_keep"], keep)
+    assert np.array_equal(r["out_hidden_bits"], hb[keep]) and np.array_equal(r["out_pos"], pos[keep])
+    # general t: sizes, disjointness, the refill is the heaviest part of the pool, weights conserved
+    r = O.consolidate_sample(hb, pos, 0, 120, mass, s_hat, keep, drop, 0.7)
+    a = r["n_absorbed"]
+    assert 0 < a < 40 and len(r["final_keep"]) == 40 and np.all(np.diff(r["final_keep"]) > 0)
+    assert set(r["refill"]) <= set(drop) and len(r["refill"]) == a
+    rest = np.setdiff1d(drop, r["refill"])
+    assert mass[r["refill"]].min() >= mass[rest].max()
+    anchors = keep[r["dest"] < 0]
+    assert set(r["final_keep"]) == set(anchors) | set(r["refill"])
+    for slot in np.nonzero(r["merged_mask"])[0]:                      # Eq. 5 is a convex combination
+        i = r["final_keep"][slot]
+        src = keep[(r["dest"] >= 0) & (keep[np.maximum(r["dest"], 0)] == i)]
+        grp = np.concatenate([[i], src])
+        lo, hi = h[grp].min(axis=0), h[grp].max(axis=0)
+        assert np.all(r["merged"][slot] >= lo - 1e-12) and np.all(r["merged"][slot] <= hi + 1e-12)
+        w = s_hat[grp] / s_hat[grp].sum()
+        assert np.allclose(r["merged"][slot], w @ h[grp], rtol=1e-12, atol=1e-14)
+    # a twin of a kept token (same row, lower salience) is absorbed and leaves its anchor's row unchanged
+    h2 = h.copy(); j, i = keep[7], keep[3]
+    h2[j] = h2[i]
+    hb2 = O.f64_to_bf16_bits(h2)
+    s2 = s_hat.copy(); s2[i], s2[j] = 0.99, 0.01
+    r2 = O.consolidate_sample(hb2, pos, 0, 120, mass, s2, keep, drop, 0.999)
+    assert r2["dest"][7] == 3 or r2["dest"][r2["dest"][7]] < 0
+    if r2["dest"][7] == 3 and (r2["dest"] == 3).sum() == 1:
+        slot = int(np.nonzero(r2["final_keep"] == i)[0][0])
+        assert np.allclose(r2["merged"][slot], h2[i], rtol=1e-12)
+
+
+PLANTED_42 = [
+    ("absorbed tokens may absorb in turn",
+     lambda mod: dict(route_within_kept=lambda hv, sh, keep, t: (lambda S, order: (
+         np.array([max([(S[a, p], -a) for a in order[:order.index(p)] if S[a, p] > t] or [(0, 1)])[1] * -1
+                   for p in range(len(keep))], dtype=np.int32), None))(
+         mod.cosine_matrix(hv[keep], hv[keep]), sorted(range(len(keep)), key=lambda p: (-sh[keep[p]], keep[p]))))),
+    ("low salience absorbs high salience",
+     lambda mod: dict(route_within_kept=lambda hv, sh, keep, t: O.route_within_kept(hv, -sh, keep, t))),
+    ("refill ranked by salience instead of attention mass",
+     lambda mod: dict(refill_from_pruned=lambda mass, drop, n: np.sort(drop[::-1][:n]).astype(np.int32))),
+    ("refill ties go to the higher index",
+     lambda mod: dict(refill_from_pruned=lambda mass, drop, n: np.sort(
+         drop[np.lexsort((-drop, -mass[drop]))[:n]]).astype(np.int32))),
+]
+
+
+@pytest.mark.parametrize("label,patch", PLANTED_42, ids=[p[0] for p in PLANTED_42])
+def test_planted_slip_in_consolidation_is_caught(label, patch):
+    mod = _mutant()
+    for name, fn in patch(mod).items():
+        setattr(mod, name, fn)
+    with pytest.raises(AssertionError):
+        check_hand_consolidation(mod)
