@@ -323,6 +323,38 @@ def run_cuda(args):
               "GBs": kv_bytes / kv_us / 1e3, "frac_of_hbm_peak": kv_bytes / kv_us / 1e3 / peaks["hbm_gbs"]}
         del kv_src, kv_dst
 
+    # ---- stage 2 as Sec. 4.2 words it (routing inside the kept set, refill by attention mass), timed
+    # apart from the step on the step's own stage-1 results
+    cons = None
+    if args.consolidate_threshold is not None and keep_k < int(batch.vis_len.max()):
+        import dataclasses
+        p2 = dataclasses.replace(params, sim_threshold=args.consolidate_threshold)
+        st1 = [t.clone() for t in (out.mass, out.salience, out.keep_idx, out.drop_idx)]
+        out2 = A.alloc_outputs(copies[0], keep_k)
+        scratch = torch.empty(A.asap_consolidate_scratch_bytes(batch.B, keep_k), dtype=torch.uint8, device=device)
+        n_abs = torch.zeros(batch.B, dtype=torch.int32, device=device)
+        call = lambda i: A.asap_consolidate(ctx, copies[i % n_copies], p2, st1[0], st1[1], st1[2], st1[3], scratch,
+                                            out2, n_abs, stream)
+        for i in range(3):
+            call(i)
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        c0.record(stream)
+        for i in range(50):
+            call(i)
+        c1.record(stream)
+        torch.cuda.synchronize()
+        A.asap_check(ctx)
+        A.asap_profile(ctx, True)
+        for i in range(50):
+            call(i)
+        torch.cuda.synchronize()
+        ck = {name: ms / max(n, 1) * 1e3 for name, (n, ms) in A.asap_profile_read(ctx).items()}
+        A.asap_profile(ctx, False)
+        cons = {"threshold": args.consolidate_threshold, "us": c0.elapsed_time(c1) / 50 * 1e3,
+                "absorbed_per_sequence": float(n_abs.float().mean()), "kernel_us": ck}
+        del scratch, out2
+
     # ---- end to end from pinned host memory
     e2e = None
     if not args.no_e2e:
@@ -418,7 +450,7 @@ def run_cuda(args):
         "latency_us": {"p10": per_step[len(per_step) // 10] * 1e3, "p50": per_step[len(per_step) // 2] * 1e3,
                        "p90": per_step[(len(per_step) * 9) // 10] * 1e3},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "kernels": kernels,
-        "cpu_baseline": cpu, "kv_compaction": kv,
+        "cpu_baseline": cpu, "kv_compaction": kv, "consolidate_within_kept": cons,
     }
     print(json.dumps(line))
     R.shutdown()
@@ -437,6 +469,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--kv-layers", type=int, default=3,
                     help="also time KV-cache compaction of this many layers (0 = skip)")
+    ap.add_argument("--consolidate-threshold", type=float, default=0.8,
+                    help="also time asap_consolidate (Sec. 4.2 inside the kept set) with this threshold t")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--ref-sequences", type=int, default=2,

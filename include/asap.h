@@ -140,6 +140,36 @@ asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *
                        const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
                        const asap_outputs *out, void *stream);
 
+/* Stage 2 in the wording of Sec. 4.2: redundancy is removed INSIDE the kept set and the freed
+ * budget goes back to the pruned pool.  Given stage 1's results (`mass` s_j of Eq. 1, `salience`
+ * s_hat_j of Eq. 2, the kept and pruned lists of asap_select, all device arrays laid out as in
+ * asap_outputs) the call
+ *   - forms the cosine similarity S of every pair of kept tokens;
+ *   - visits the kept tokens by salience (descending, lower sequence index first among equals):
+ *     a token whose similarity to an earlier, not absorbed token (an anchor) exceeds
+ *     p->sim_threshold is absorbed by the most similar such anchor (lowest index among equals),
+ *     any other token becomes an anchor; at most vis_len[b] - keep_k tokens are absorbed, so that
+ *     every vacated slot can be refilled;
+ *   - replaces every anchor by the salience-weighted mean of itself and its sources (Eq. 5);
+ *   - refills the vacated slots with the pruned tokens of largest s_j (lower index first among
+ *     equals), so that exactly keep_k visual tokens leave;
+ *   - compacts hidden states and position ids as asap_merge does.
+ * Outputs: out->keep_idx = the final kept list (anchors and refilled tokens, ascending);
+ * out->drop_idx = the absorbed tokens, ascending, padded with -1; out->assign = the slot in
+ * out->keep_idx each of them was merged into; out->best_sim (if non-NULL) = its similarity to that
+ * anchor; out_hidden, out_pos, src_row, out_cu_seqlens as in asap_merge.  `n_absorbed` ([B],
+ * device, may be NULL) receives the number of absorbed tokens per sequence.
+ * `keep_idx` / `drop_idx` must not be the arrays `out` points to.  `scratch` is caller-owned
+ * device memory of at least asap_consolidate_scratch_bytes(B, keep_k) bytes, 16-byte aligned
+ * (the similarity matrix, keep_k * keep_k floats per sequence, and a bit matrix); nothing is
+ * kept in it between calls.  Requires p->merge_enable and keep_k < max_vis (ASAP_ERR_INVALID
+ * otherwise: asap_merge covers those cases) and keep_k <= 4096 (ASAP_ERR_UNSUPPORTED). */
+size_t asap_consolidate_scratch_bytes(int32_t B, int32_t keep_k);
+asap_status asap_consolidate(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                             const float *mass, const float *salience, const int32_t *keep_idx,
+                             const int32_t *drop_idx, void *scratch, size_t scratch_bytes,
+                             const asap_outputs *out, int32_t *n_absorbed, void *stream);
+
 /* Steps 1a-5 back to back on `stream`; fills every field of `out`. */
 asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                             const asap_outputs *out, void *stream);

@@ -274,7 +274,8 @@ def prune_sample(q_bits, k_bits, hidden_bits, pos_ids, v0: int, nv: int, r0: int
 # ----------------------------------------------------------------------------------
 # Stage 2 as Sec. 4.2 states it: consolidation INSIDE the kept set, then budget reallocation
 # ----------------------------------------------------------------------------------
-def route_within_kept(hv: np.ndarray, s_hat: np.ndarray, keep: np.ndarray, threshold: float):
+def route_within_kept(hv: np.ndarray, s_hat: np.ndarray, keep: np.ndarray, threshold: float,
+                      max_absorb=None):
     """Salience-anchored routing of Sec. 4.2 among the kept tokens.
 
     A token j may be absorbed by a token i only if S_ij > t and i comes before j in the order
@@ -284,6 +285,9 @@ def route_within_kept(hv: np.ndarray, s_hat: np.ndarray, keep: np.ndarray, thres
     most similar token among those that were NOT absorbed before it (the anchors), lowest
     sequence index among equally similar ones, provided that similarity exceeds t; otherwise it
     becomes an anchor itself.  Source sets are therefore disjoint and end at anchors.
+    A vacated slot must be refilled from the pruned pool (the budget is fixed), so at most
+    `max_absorb` tokens (the size of that pool) are absorbed: once that many have been, every
+    later token stays an anchor.
 
     Returns (dest [k]: slot of the absorbing anchor, -1 for anchors; margin [k]: how far the
     decision of each token was from flipping: distance of its best similarity from t, and from
@@ -294,6 +298,7 @@ def route_within_kept(hv: np.ndarray, s_hat: np.ndarray, keep: np.ndarray, thres
     dest = np.full(k, -1, dtype=np.int32)
     margin = np.full(k, np.inf)
     anchors = []
+    n_absorbed = 0
     for p in order:
         best, best_a, second = -np.inf, -1, -np.inf
         for a in sorted(anchors):                 # ascending slot = ascending sequence index
@@ -304,8 +309,9 @@ def route_within_kept(hv: np.ndarray, s_hat: np.ndarray, keep: np.ndarray, thres
                 second = v
         if best_a >= 0:
             margin[p] = min(abs(best - threshold), best - second)
-        if best_a >= 0 and best > threshold:
+        if best_a >= 0 and best > threshold and (max_absorb is None or n_absorbed < max_absorb):
             dest[p] = best_a
+            n_absorbed += 1
         else:
             anchors.append(p)
     return dest, margin
@@ -328,7 +334,7 @@ def consolidate_sample(hidden_bits, pos_ids, v0: int, nv: int, mass, s_hat, keep
     hid = bf16_bits_to_f64(hidden_bits)
     hv = hid[v0:v0 + nv]
     n = hid.shape[0]
-    dest, margin = route_within_kept(hv, s_hat, keep, threshold)
+    dest, margin = route_within_kept(hv, s_hat, keep, threshold, max_absorb=len(drop))
     if dest_override is not None:
         dest = np.asarray(dest_override, dtype=np.int32)
     absorbed = np.nonzero(dest >= 0)[0]

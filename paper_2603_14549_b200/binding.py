@@ -23,7 +23,8 @@ STATUS_NAMES = {0: "ASAP_OK", -1: "ASAP_ERR_INVALID", -2: "ASAP_ERR_ALIGN", -3: 
                 -4: "ASAP_ERR_CUDA", -5: "ASAP_ERR_UNSUPPORTED", -6: "ASAP_ERR_DEVICE"}
 
 EXPORTS = ("asap_init", "asap_score", "asap_select", "asap_merge", "asap_prune_step", "asap_check",
-           "asap_last_error", "asap_launch_count", "asap_free", "asap_profile", "asap_profile_read", "asap_select_static", "asap_compact_kv")
+           "asap_last_error", "asap_launch_count", "asap_free", "asap_profile", "asap_profile_read", "asap_select_static", "asap_compact_kv",
+           "asap_consolidate", "asap_consolidate_scratch_bytes")
 
 
 class AsapError(RuntimeError):
@@ -90,6 +91,12 @@ def load_library() -> C.CDLL:
     lib.asap_compact_kv.restype = C.c_int
     lib.asap_compact_kv.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_size_t, C.c_int32,
                                     C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.c_void_p]
+    lib.asap_consolidate_scratch_bytes.restype = C.c_size_t
+    lib.asap_consolidate_scratch_bytes.argtypes = [C.c_int32, C.c_int32]
+    lib.asap_consolidate.restype = C.c_int
+    lib.asap_consolidate.argtypes = [C.c_void_p, C.POINTER(CInputs), C.POINTER(CParams), C.c_void_p, C.c_void_p,
+                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(COutputs),
+                                     C.c_void_p, C.c_void_p]
     lib.asap_check.restype = C.c_int
     lib.asap_check.argtypes = [C.c_void_p, C.c_void_p]
     lib.asap_last_error.restype = C.c_char_p
@@ -259,6 +266,20 @@ def asap_merge(ctx, inp: Inputs, params: Params, salience: torch.Tensor, keep_id
     ci, cp, co = inp.c_struct(), params.c_struct(), out.c_struct()
     _raise(ctx, load_library().asap_merge(ctx, C.byref(ci), C.byref(cp), _ptr(salience), _ptr(keep_idx),
                                           _ptr(drop_idx), C.byref(co), _stream(stream)))
+
+
+def asap_consolidate_scratch_bytes(B: int, keep_k: int) -> int:
+    return int(load_library().asap_consolidate_scratch_bytes(int(B), int(keep_k)))
+
+
+def asap_consolidate(ctx, inp: Inputs, params: Params, mass: torch.Tensor, salience: torch.Tensor,
+                     keep_idx: torch.Tensor, drop_idx: torch.Tensor, scratch: torch.Tensor, out: Outputs,
+                     n_absorbed: Optional[torch.Tensor] = None, stream=None) -> None:
+    """`scratch`: a contiguous device tensor of at least asap_consolidate_scratch_bytes(B, keep_k) bytes."""
+    ci, cp, co = inp.c_struct(), params.c_struct(), out.c_struct()
+    _raise(ctx, load_library().asap_consolidate(
+        ctx, C.byref(ci), C.byref(cp), _ptr(mass), _ptr(salience), _ptr(keep_idx), _ptr(drop_idx), _ptr(scratch),
+        int(scratch.numel() * scratch.element_size()), C.byref(co), _ptr(n_absorbed), _stream(stream)))
 
 
 def asap_prune_step(ctx, inp: Inputs, params: Params, out: Outputs, stream=None) -> None:

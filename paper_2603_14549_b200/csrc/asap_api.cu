@@ -338,6 +338,7 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     sa.best_sim = out->best_sim; sa.seg = ctx->seg; sa.members = ctx->members; sa.counters = ctx->cnt_sim;
     sa.tile_counters = ctx->cnt_tiles; sa.part = ctx->sim_part;
     sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
+    sa.smat = nullptr;
     sa.status = ctx->status;
     mark(ctx, "sim", st);
     launch_pdl(sim_kernel, dim3(dim3(max_mt, B, splits)), dim3(SIM_THREADS), smem, st, map_h, map_kept, sa);
@@ -376,6 +377,64 @@ asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params
                          const asap_outputs *out, cudaStream_t st) {
   ASAP_TRY(launch_merge_front(ctx, in, p, keep_idx, out, st));
   return launch_merge_back(ctx, in, p, salience, keep_idx, drop_idx, out, st);
+}
+
+// Sec. 4.2 inside the kept set: kept rows gathered, their keep_k x keep_k cosine matrix, routing.
+size_t route_smat_bytes(int B, int k) { return align_up((size_t)B * k * k * sizeof(float), 256); }
+size_t route_mask_bytes(int B, int k) { return (size_t)B * k * ((k + 31) / 32) * sizeof(uint32_t); }
+
+asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                                     const float *mass, const float *salience, const int32_t *keep_idx,
+                                     const int32_t *drop_idx, void *scratch, const asap_outputs *out,
+                                     int32_t *n_absorbed, cudaStream_t st) {
+  const int B = in->B, D = in->D, k = p->keep_k;
+  mark(ctx, "kept_gather", st);
+  launch_pdl(kept_gather_kernel, dim3((k + GATHER_THREADS / 32 - 1) / (GATHER_THREADS / 32), B), dim3(GATHER_THREADS), 0, st,
+             static_cast<const __nv_bfloat16 *>(in->hidden), ctx->desc, D, k, keep_idx, ctx->kept_rows, ctx->kept_inv);
+  ASAP_TRY(after_launch(ctx, "kept_gather"));
+
+  const int n_nt = (k + 255) / 256;
+  const int n_tile = (((k + n_nt - 1) / n_nt) + 15) & ~15;
+  const int stage_bytes = 2 * (SIM_A_BYTES + n_tile * 128);
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < 2 * n_tile) tmem_cols <<= 1;
+  int stages = (192 * 1024) / stage_bytes;
+  if (stages > SIM_MAX_STAGES) stages = SIM_MAX_STAGES;
+  const size_t smem = (size_t)stages * stage_bytes + SIM_BOOK_BYTES + 1024;
+  CUtensorMap map_a, map_b;
+  if (!make_map(ctx, &map_a, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, 128) ||
+      !make_map(ctx, &map_b, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, (uint32_t)n_tile))
+    return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for the kept rows");
+  float *smat = static_cast<float *>(scratch);
+  SimArgs sa;
+  sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = n_tile;
+  sa.n_nt = n_nt; sa.stages = stages; sa.splits = 1; sa.max_mt = (k + 127) / 128; sa.tmem_cols = tmem_cols;
+  sa.threshold = p->sim_threshold;
+  sa.role = ctx->role; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
+  sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr; sa.tile_counters = nullptr;
+  sa.part = nullptr; sa.ss_part = nullptr; sa.smat = smat; sa.status = ctx->status;
+  mark(ctx, "sim_kept", st);
+  launch_pdl(sim_kernel, dim3((k + 127) / 128, B, 1), dim3(SIM_THREADS), smem, st, map_a, map_b, sa);
+  ASAP_TRY(after_launch(ctx, "sim_kept"));
+
+  RouteArgs ra;
+  ra.desc = ctx->desc; ra.max_vis = in->max_vis; ra.keep_k = k; ra.kw = (k + 31) / 32;
+  ra.threshold = p->sim_threshold; ra.smat = smat;
+  const size_t fixed_words = 5 * (size_t)k;
+  const size_t tail_words = (size_t)(in->max_vis - k) + (size_t)in->max_vis;
+  const size_t mask_words = (size_t)k * ra.kw;
+  const bool mask_in_smem = (fixed_words + (mask_words > tail_words ? mask_words : tail_words)) * 4 <= 200 * 1024;
+  ra.mask_g = mask_in_smem ? nullptr
+                           : reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(scratch) + route_smat_bytes(B, k));
+  const size_t route_smem = (fixed_words + (mask_in_smem && mask_words > tail_words ? mask_words : tail_words)) * 4;
+  if (route_smem > 224 * 1024)
+    return fail(ctx, ASAP_ERR_UNSUPPORTED, "max_vis = %d is too large for the routing kernel", in->max_vis);
+  ra.salience = salience; ra.mass = mass; ra.keep_idx = keep_idx; ra.drop_idx = drop_idx;
+  ra.final_keep = out->keep_idx; ra.src_idx = out->drop_idx; ra.src_assign = out->assign;
+  ra.seg = ctx->seg; ra.members = ctx->members; ra.n_absorbed = n_absorbed; ra.src_sim = out->best_sim;
+  mark(ctx, "route", st);
+  launch_pdl(route_kernel, dim3(B), dim3(ROUTE_THREADS), route_smem, st, ra);
+  return after_launch(ctx, "route");
 }
 
 }  // namespace
@@ -468,6 +527,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   if (e == cudaSuccess) e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
   // lowest priority: when both streams have blocks to place, the score kernel's go first and the
   // mass kernels fill what is left of each SM
   int prio_least = 0, prio_greatest = 0;
@@ -521,6 +581,31 @@ asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *
                                                                          out->best_sim, merging(in, p) ? 1 : 0);
   ASAP_TRY(after_launch(ctx, "role_map"));
   return finish(ctx, launch_merge(ctx, in, p, salience, keep_idx, drop_idx, out, st), st);
+}
+
+size_t asap_consolidate_scratch_bytes(int32_t B, int32_t keep_k) {
+  if (B <= 0 || keep_k <= 0) return 0;
+  return route_smat_bytes(B, keep_k) + route_mask_bytes(B, keep_k);
+}
+
+asap_status asap_consolidate(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *mass,
+                             const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
+                             void *scratch, size_t scratch_bytes, const asap_outputs *out,
+                             int32_t *n_absorbed, void *stream) {
+  ASAP_TRY(validate(ctx, in, p, out, NEED_HIDDEN | NEED_SELECT_OUT | NEED_MERGE_OUT));
+  if (!mass || !salience || !keep_idx || !drop_idx) return fail(ctx, ASAP_ERR_INVALID, "null mass / salience / keep_idx / drop_idx");
+  if (!p->merge_enable || in->max_vis <= p->keep_k)
+    return fail(ctx, ASAP_ERR_INVALID, "asap_consolidate needs merge_enable and keep_k < max_vis; asap_merge covers the rest");
+  if (keep_idx == out->keep_idx || drop_idx == out->drop_idx)
+    return fail(ctx, ASAP_ERR_INVALID, "asap_consolidate: the stage-1 lists must not be the output lists");
+  if (p->keep_k > 32 * 32 * ROUTE_LANE_WORDS)
+    return fail(ctx, ASAP_ERR_UNSUPPORTED, "asap_consolidate: keep_k above %d", 32 * 32 * ROUTE_LANE_WORDS);
+  if (!scratch || !aligned16(scratch) || scratch_bytes < asap_consolidate_scratch_bytes(in->B, p->keep_k))
+    return fail(ctx, ASAP_ERR_WORKSPACE, "asap_consolidate: scratch is null, unaligned or smaller than asap_consolidate_scratch_bytes");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ASAP_TRY(launch_prepare(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity, st));
+  ASAP_TRY(launch_consolidate_front(ctx, in, p, mass, salience, keep_idx, drop_idx, scratch, out, n_absorbed, st));
+  return finish(ctx, launch_merge_back(ctx, in, p, salience, out->keep_idx, out->drop_idx, out, st), st);
 }
 
 asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const asap_outputs *out,

@@ -616,6 +616,303 @@ __device__ __forceinline__ void csr_block(const SampleDesc &d, int b, int max_vi
 }
 
 // =======================================================================================
+// route: Sec. 4.2 inside the kept set, one block per sample.  Input: the keep_k x keep_k cosine
+// matrix S of the kept rows, the salience, the attention mass, stage 1's kept / pruned lists.
+//   A  visiting order of the kept slots: salience descending, sequence index ascending.
+//   B  bit matrix  M[p] = { q : S[p][q] > t }.
+//   C  one warp walks the slots in visiting order.  A slot whose bit is set in the running union
+//      of the anchors' rows is absorbed (while the pruned pool can still refill a slot, i.e. at
+//      most nv - keep_k times); any other slot becomes an anchor and adds its row to the union.
+//      This is the greedy rule "join the most similar earlier anchor if that similarity exceeds t,
+//      else become an anchor" with the question WHICH anchor left to step D.
+//   D  every absorbed slot finds the most similar anchor that was visited before it (lowest slot
+//      among equals).
+//   E  the vacated slots are refilled with the pruned tokens of largest attention mass (radix
+//      select, lower index first among equals).
+//   F  anchors and refilled tokens, in sequence order, form the final kept list; the absorbed
+//      tokens, ascending, form the source list with their anchor's FINAL slot; CSR of that list.
+// Outputs use the layouts of the merge kernel: final_keep [B, keep_k], src_idx / src_assign /
+// src_sim [B, max_vis - keep_k] (padding -1 / 0), seg [B, keep_k + 1], members [B, max_vis - keep_k].
+// =======================================================================================
+constexpr int ROUTE_THREADS = 1024;
+constexpr int ROUTE_LANE_WORDS = 4;                     // keep_k <= 32 * 32 * 4
+
+struct RouteArgs {
+  const SampleDesc *desc;
+  int max_vis, keep_k, kw;        // kw = ceil(keep_k / 32)
+  float threshold;
+  const float *smat;              // [B, keep_k, keep_k]
+  uint32_t *mask_g;               // [B, keep_k, kw] or nullptr: the bit matrix lives in shared memory
+  const float *salience, *mass;   // [B, max_vis]
+  const int32_t *keep_idx;        // [B, keep_k]            stage 1
+  const int32_t *drop_idx;        // [B, max_vis - keep_k]  stage 1
+  int32_t *final_keep, *src_idx, *src_assign, *seg, *members, *n_absorbed;
+  float *src_sim;                 // nullable
+};
+
+__global__ void __launch_bounds__(ROUTE_THREADS)
+route_kernel(RouteArgs a) {
+  pdl_enter();
+  extern __shared__ uint32_t r_smem[];
+  __shared__ int s_hist[256];
+  __shared__ int s_scan[33];
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_remaining, s_nabs;
+  const int b = blockIdx.x;
+  const SampleDesc d = a.desc[b];
+  const int k = a.keep_k, kw = a.kw, nd_max = a.max_vis - k;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nthr = blockDim.x;
+  int32_t *fk_b = a.final_keep + (size_t)b * k;
+  int32_t *si_b = a.src_idx + (size_t)b * nd_max;
+  int32_t *sa_b = a.src_assign + (size_t)b * nd_max;
+  float *ss_b = a.src_sim ? a.src_sim + (size_t)b * nd_max : nullptr;
+  int32_t *seg_b = a.seg + (size_t)b * (k + 1);
+  int32_t *mem_b = a.members + (size_t)b * nd_max;
+  if (!d.valid) {
+    for (int j = tid; j < k; j += nthr) fk_b[j] = -1;
+    for (int j = tid; j < nd_max; j += nthr) { si_b[j] = -1; sa_b[j] = -1; if (ss_b) ss_b[j] = 0.f; }
+    for (int j = tid; j <= k; j += nthr) seg_b[j] = 0;
+    if (tid == 0 && a.n_absorbed) a.n_absorbed[b] = 0;
+    return;
+  }
+  const int nv = d.nv, nd = nv - k;
+  // shared memory: [order k][rank k][flag k][dest k][tmp k] [union: bit matrix k*kw | key nd_max + pos max_vis]
+  int *s_order = reinterpret_cast<int *>(r_smem);
+  int *s_rank = s_order + k;
+  int *s_flag = s_rank + k;
+  int *s_dest = s_flag + k;
+  uint32_t *s_tmp = r_smem + 4 * (size_t)k;
+  uint32_t *s_union = s_tmp + k;
+  uint32_t *mask = a.mask_g ? a.mask_g + (size_t)b * k * kw : s_union;
+  const int32_t *keep_b = a.keep_idx + (size_t)b * k;
+  const int32_t *drop_b = a.drop_idx + (size_t)b * nd_max;
+  const float *sal_b = a.salience + (size_t)b * a.max_vis;
+  const float *S = a.smat + (size_t)b * k * k;
+
+  // ---- A: visiting order.  Keys are order-preserving integers, so NaN cannot break the permutation.
+  for (int p = tid; p < k; p += nthr) {
+    const int j = min(max(keep_b[p], 0), nv - 1);
+    s_tmp[p] = score_key(sal_b[j]);
+  }
+  __syncthreads();
+  for (int p = tid; p < k; p += nthr) {
+    const uint32_t mine = s_tmp[p];
+    int r = 0;
+    for (int q = 0; q < k; ++q) {
+      const uint32_t o = s_tmp[q];
+      r += (o > mine) || (o == mine && q < p);       // the kept list is ascending: q < p is the lower index
+    }
+    s_rank[p] = r;
+    s_order[r] = p;
+  }
+  // ---- B: bit matrix, one warp per row, coalesced
+  for (int p = warp; p < k; p += (nthr >> 5)) {
+    const float *row = S + (size_t)p * k;
+    for (int w = 0; w < kw; ++w) {
+      const int q = w * 32 + lane;
+      const bool hit = q < k && q != p && __ldcg(row + q) > a.threshold;
+      const unsigned bits = __ballot_sync(0xffffffffu, hit);
+      if (lane == 0) mask[(size_t)p * kw + w] = bits;
+    }
+  }
+  __syncthreads();
+  // ---- C: greedy walk by one warp; the union lives in registers, word w in lane w % 32
+  if (warp == 0) {
+    uint32_t supp[ROUTE_LANE_WORDS];
+#pragma unroll
+    for (int i = 0; i < ROUTE_LANE_WORDS; ++i) supp[i] = 0u;
+    int n_abs = 0;
+    for (int r = 0; r < k; ++r) {
+      const int p = s_order[r];
+      const int w = p >> 5;
+      uint32_t word = 0u;
+#pragma unroll
+      for (int i = 0; i < ROUTE_LANE_WORDS; ++i)
+        if ((w >> 5) == i) word = supp[i];
+      word = __shfl_sync(0xffffffffu, word, w & 31);
+      const bool absorbed = ((word >> (p & 31)) & 1u) && n_abs < nd;
+      if (absorbed) {
+        ++n_abs;
+      } else {
+#pragma unroll
+        for (int i = 0; i < ROUTE_LANE_WORDS; ++i) {
+          const int ww = i * 32 + lane;
+          if (ww < kw) supp[i] |= mask[(size_t)p * kw + ww];
+        }
+      }
+      if (lane == 0) s_flag[p] = absorbed ? 0 : 1;
+    }
+    if (lane == 0) s_nabs = n_abs;
+  }
+  __syncthreads();
+  const int n_abs = s_nabs;
+  // ---- D: destination of every absorbed slot
+  for (int p = warp; p < k; p += (nthr >> 5)) {
+    if (s_flag[p]) { if (lane == 0) s_dest[p] = -1; continue; }
+    const float *row = S + (size_t)p * k;
+    const int rp = s_rank[p];
+    float best = -INFINITY;
+    int best_q = 0x7fffffff;
+    for (int q = lane; q < k; q += 32) {
+      if (s_flag[q] && s_rank[q] < rp) {
+        const float v = __ldcg(row + q);
+        if (v > best) { best = v; best_q = q; }       // ascending q: the first maximum stays
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oq = __shfl_xor_sync(0xffffffffu, best_q, o);
+      if (ob > best || (ob == best && oq < best_q)) { best = ob; best_q = oq; }
+    }
+    if (lane == 0) {
+      s_dest[p] = best_q < k ? best_q : -1;
+      s_tmp[p] = __float_as_uint(best);
+    }
+  }
+  __syncthreads();      // the bit matrix is dead from here on: its space is reused
+  uint32_t *s_key = s_union;                                  // [nd]
+  int *s_pos = reinterpret_cast<int *>(s_union + nd_max);     // [nv] 1 + final slot, 0 = not in the final list
+  // ---- E: the n_abs pruned tokens of largest attention mass
+  const float *mass_b = a.mass + (size_t)b * a.max_vis;
+  for (int v = tid; v < nv; v += nthr) s_pos[v] = 0;
+  for (int i = tid; i < nd; i += nthr) {
+    const int j = min(max(drop_b[i], 0), nv - 1);
+    s_key[i] = score_key(mass_b[j]);
+  }
+  if (tid == 0) { s_prefix = 0u; s_remaining = n_abs; }
+  __syncthreads();
+  if (n_abs > 0) {
+    uint32_t known = 0u;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int i = tid; i < 256; i += nthr) s_hist[i] = 0;
+      __syncthreads();
+      const uint32_t prefix = s_prefix;
+      for (int i = tid; i < nd; i += nthr) {
+        const uint32_t key = s_key[i];
+        if ((key & known) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1);
+      }
+      __syncthreads();
+      if (tid < 32) {
+        int mine = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) mine += s_hist[255 - 8 * lane - e];
+        int inc = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          int t = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += t;
+        }
+        const int remaining = s_remaining;
+        __syncwarp();
+        const int before = inc - mine;
+        if (before < remaining && remaining <= inc) {
+          int run = before;
+          for (int e = 0; e < 8; ++e) {
+            const int digit = 255 - 8 * lane - e;
+            const int c = s_hist[digit];
+            if (run + c >= remaining) {
+              s_prefix = prefix | ((uint32_t)digit << shift);
+              s_remaining = remaining - run;
+              break;
+            }
+            run += c;
+          }
+        }
+      }
+      known |= 255u << shift;
+      __syncthreads();
+    }
+    const uint32_t kth = s_prefix;
+    const int take_equal = s_remaining;
+    const int per = (nd + nthr - 1) / nthr;
+    const int lo = min(nd, tid * per), hi = min(nd, lo + per);
+    int n_eq = 0;
+    for (int i = lo; i < hi; ++i) n_eq += (s_key[i] == kth);
+    int tot;
+    int e = block_exclusive_scan(n_eq, s_scan, tot);
+    for (int i = lo; i < hi; ++i) {
+      const uint32_t key = s_key[i];
+      if (key > kth || (key == kth && e < take_equal)) s_pos[min(max(drop_b[i], 0), nv - 1)] = 1;
+      e += (key == kth);
+    }
+  }
+  for (int p = tid; p < k; p += nthr)
+    if (s_flag[p]) s_pos[min(max(keep_b[p], 0), nv - 1)] = 1;
+  __syncthreads();
+  // ---- F: final kept list in sequence order
+  {
+    const int per = (nv + nthr - 1) / nthr;
+    const int lo = min(nv, tid * per), hi = min(nv, lo + per);
+    int cnt = 0;
+    for (int v = lo; v < hi; ++v) cnt += s_pos[v];
+    int tot;
+    int run = block_exclusive_scan(cnt, s_scan, tot);
+    for (int v = lo; v < hi; ++v) {
+      if (s_pos[v]) {
+        if (run < k) fk_b[run] = v;
+        s_pos[v] = ++run;
+      }
+    }
+    // fewer than keep_k can only come from malformed input lists: pad
+    for (int j = tot + tid; j < k; j += nthr) fk_b[j] = -1;
+  }
+  __syncthreads();
+  // source list: absorbed slots in ascending order, with the final slot of their anchor
+  {
+    const int per = (k + nthr - 1) / nthr;
+    const int lo = min(k, tid * per), hi = min(k, lo + per);
+    int cnt = 0;
+    for (int p = lo; p < hi; ++p) cnt += !s_flag[p];
+    int tot;
+    int run = block_exclusive_scan(cnt, s_scan, tot);
+    for (int p = lo; p < hi; ++p) {
+      if (!s_flag[p] && run < nd_max) {
+        const int q = s_dest[p];
+        const int slot = q >= 0 ? s_pos[min(max(keep_b[q], 0), nv - 1)] - 1 : -1;
+        si_b[run] = keep_b[p];
+        sa_b[run] = (slot >= 0 && slot < k) ? slot : -1;
+        if (ss_b) ss_b[run] = __uint_as_float(s_tmp[p]);
+        s_key[run] = (uint32_t)((slot >= 0 && slot < k) ? slot : -1);     // for the grouping below
+        ++run;
+      }
+    }
+    for (int j = n_abs + tid; j < nd_max; j += nthr) { si_b[j] = -1; sa_b[j] = -1; if (ss_b) ss_b[j] = 0.f; }
+  }
+  if (tid == 0 && a.n_absorbed) a.n_absorbed[b] = n_abs;
+  __syncthreads();
+  // grouping by destination, stable: thread t owns final slots t, t + blockDim, ...
+  {
+    int *s_cnt = s_order;                     // reuse: the visiting order is no longer needed
+    for (int sl = tid; sl < k; sl += nthr) {
+      int c = 0;
+      for (int i = 0; i < n_abs; ++i) c += ((int)s_key[i] == sl);
+      s_cnt[sl] = c;
+    }
+    __syncthreads();
+    const int per = (k + nthr - 1) / nthr;
+    const int lo = min(k, tid * per), hi = min(k, lo + per);
+    int mine = 0;
+    for (int sl = lo; sl < hi; ++sl) mine += s_cnt[sl];
+    int tot;
+    int run = block_exclusive_scan(mine, s_scan, tot);
+    for (int sl = lo; sl < hi; ++sl) {
+      const int c = s_cnt[sl];
+      seg_b[sl] = run;
+      s_cnt[sl] = run;
+      run += c;
+    }
+    if (tid == 0) seg_b[k] = tot;
+    __syncthreads();
+    for (int sl = tid; sl < k; sl += nthr) {
+      int at = s_cnt[sl];
+      for (int i = 0; i < n_abs; ++i)
+        if ((int)s_key[i] == sl) mem_b[at++] = i;
+    }
+  }
+}
+
+// =======================================================================================
 // merge_compact: grid (keep_k + copy-row groups, B).
 //   blockIdx.x <  keep_k : the block owns one kept visual row.  Its members (the dropped tokens
 //                          assigned to that slot) are first listed in shared memory with their

@@ -484,6 +484,10 @@ head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
 //                   row tile adds the slices in slice order and does the same epilogue.
 // Rows that were kept, or lie past the image span, are computed but not written.
 // The block that finishes a sample's last row tile groups the dropped tokens by destination.
+//   matrix mode:    (a.smat set, one slice) the row operand is the dense kept-row array too, and
+//                   the epilogue writes the whole keep_k x keep_k cosine matrix of the sample,
+//                   S[p][q] = <h_p, h_q> * (1/||h_p|| * 1/||h_q||), for the routing inside the
+//                   kept set; `tmap_h` is then a map of the kept rows with a 128-row box.
 // =======================================================================================
 constexpr int SIM_THREADS = 192;
 constexpr int SIM_A_BYTES = 128 * 128;           // 128 rows x 64 bf16
@@ -506,6 +510,7 @@ struct SimArgs {
   unsigned int *tile_counters;  // [B, max_mt] finished slices per row tile
   float *part;               // [B, max_mt, splits, keep_k, 128] partial dot products (several slices only)
   float *ss_part;            // [B, max_mt, splits, 128]         partial squared norms
+  float *smat;               // [B, keep_k, keep_k] or nullptr: matrix mode
   uint32_t *status;
 };
 
@@ -530,7 +535,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   extern __shared__ uint8_t smem_raw[];
   const int mt = blockIdx.x, b = blockIdx.y, z = blockIdx.z;
   const SampleDesc d = a.desc[b];
-  if (!d.valid || mt * 128 >= d.nv) return;
+  if (!d.valid || mt * 128 >= (a.smat ? a.keep_k : d.nv)) return;
   if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SIM_TIMEOUT) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -572,8 +577,8 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     if (lane == 0) {
       tma_prefetch_desc(&tmap_h);
       tma_prefetch_desc(&tmap_kept);
-      const int row_a = d.row0 + d.v0 + mt * 128;
       const int row_b = b * a.keep_k;
+      const int row_a = a.smat ? row_b + mt * 128 : d.row0 + d.v0 + mt * 128;
       const int rot = (mt * 5 + b * 3) % n_kb;
       int issued = 0;
       for (int it = 0; it < total_it; ++it) {
@@ -620,7 +625,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
                           (kb > 0 || kk > 0) ? 1u : 0u);
             tc_commit(smem_u32(&bk->empty[s]));
             // after the first accumulator the epilogue warps no longer read the stages
-            if (nt > 0) mbar_arrive_n(smem_u32(&bk->empty[s]), 4);
+            if (nt > 0 || a.smat) mbar_arrive_n(smem_u32(&bk->empty[s]), 4);
           }
         }
         if (!bk->abort_flag) tc_commit(smem_u32(&bk->acc_full[buf]));
@@ -634,7 +639,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     // ---- squared norm of this thread's row, from the row tiles of the first accumulator's pass.
     // Row r of a tile is 128 bytes; its 16-byte chunk c sits at chunk position c ^ (r & 7).
     float ssq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    for (int it = 0; it < n_kb; ++it) {
+    for (int it = 0; it < (a.smat ? 0 : n_kb); ++it) {
       const int s = it % a.stages;
       mbar_wait(smem_u32(&bk->full[s]), (it / a.stages) & 1, wc);
       if (!bk->abort_flag) {
@@ -677,7 +682,15 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         uint32_t r[16];
         tmem_ld16(taddr + c, r);
         tmem_wait_ld();
-        if (part) {
+        if (a.smat) {
+          if (v < a.keep_k && !bk->abort_flag) {
+            const float inv_p = __ldg(kinv + v);
+            float *srow = a.smat + ((size_t)b * a.keep_k + v) * a.keep_k + slot0 + c;
+#pragma unroll
+            for (int e = 0; e < 16; ++e)
+              if (c + e < ncol) srow[e] = __uint_as_float(r[e]) * (inv_p * __ldg(kinv + slot0 + c + e));
+          }
+        } else if (part) {
 #pragma unroll
           for (int e = 0; e < 16; ++e)
             if (c + e < ncol) part[(size_t)(slot0 + c + e) * 128 + lrow] = __uint_as_float(r[e]);
@@ -745,6 +758,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         }
       }
     }
+    if (a.smat) finalize = false;
     if (finalize && v < d.nv && !bk->abort_flag) {
       const int role = a.role[(size_t)b * a.max_vis + v];
       if (role < 0) {
@@ -766,6 +780,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     tc_fence_after();
     tmem_dealloc(tmem_base, a.tmem_cols);
   }
+  if (a.smat) return;
   if (!bk->is_last && a.splits > 1) return;     // a slice that did not finalize its row tile
   __syncthreads();
   // the block that finishes the sample's last row tile groups the dropped tokens by destination

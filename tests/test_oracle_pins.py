@@ -597,3 +597,18 @@ def test_planted_slip_in_consolidation_is_caught(label, patch):
         setattr(mod, name, fn)
     with pytest.raises(AssertionError):
         check_hand_consolidation(mod)
+
+
+def test_consolidation_never_absorbs_more_than_the_pool_can_refill():
+    """Fixed budget: with 40 kept of 46 tokens and everything similar, only six slots can be vacated."""
+    rng = np.random.default_rng(24)
+    base = rng.standard_normal(16)
+    h = base[None, :] + 0.01 * rng.standard_normal((46, 16))              # all mutually similar
+    hb = bits(torch.tensor(h, dtype=torch.float32).to(torch.bfloat16))
+    s_hat, mass = rng.uniform(0.1, 1, 46), rng.uniform(0, 5, 46)
+    keep = np.sort(rng.choice(46, 40, replace=False)); drop = np.setdiff1d(np.arange(46), keep)
+    r = O.consolidate_sample(hb, np.arange(46), 0, 46, mass, s_hat, keep, drop, 0.5)
+    assert r["n_absorbed"] == 6 and len(r["final_keep"]) == 40 and set(drop) <= set(r["final_keep"])
+    order = sorted(range(40), key=lambda p: (-s_hat[keep[p]], keep[p]))
+    assert sorted(np.nonzero(r["dest"] >= 0)[0].tolist()) == sorted(order[1:7])   # the first six after the top one
+    assert np.all(r["dest"][order[1:7]] == order[0])
