@@ -398,7 +398,23 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   const int stage_bytes = 2 * (SIM_A_BYTES + n_tile * 128);
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < 2 * n_tile) tmem_cols <<= 1;
-  int stages = (192 * 1024) / stage_bytes;
+  // slices of the hidden dimension, chosen by the cost model of the similarity launch
+  const int max_mt = (k + 127) / 128;
+  const int n_kb = D / 128;
+  int splits = 1;
+  float best_cost = (float)n_kb;
+  for (int c = 2; c <= 8; ++c) {
+    if (n_kb % c != 0) continue;
+    if ((long long)max_mt * B * c > 2LL * ctx->num_sms) break;
+    if ((size_t)B * max_mt * c * ((size_t)k + 1) * 128 * sizeof(float) > ctx->sim_part_bytes) break;
+    if ((size_t)B * max_mt > ctx->cap_tiles) break;
+    const float cost = (float)n_kb / c + 0.5f * (float)k * c / 64.f;
+    if (cost < best_cost) { best_cost = cost; splits = c; }
+  }
+  const long long ctas = (long long)max_mt * B * splits;
+  const bool two_per_sm = ctas > ctx->num_sms && ctas <= 2LL * ctx->num_sms && tmem_cols <= 256 &&
+                          2 * stage_bytes <= 96 * 1024;
+  int stages = ((two_per_sm ? 96 : 192) * 1024) / stage_bytes;
   if (stages > SIM_MAX_STAGES) stages = SIM_MAX_STAGES;
   const size_t smem = (size_t)stages * stage_bytes + SIM_BOOK_BYTES + 1024;
   CUtensorMap map_a, map_b;
@@ -408,13 +424,14 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   float *smat = static_cast<float *>(scratch);
   SimArgs sa;
   sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = n_tile;
-  sa.n_nt = n_nt; sa.stages = stages; sa.splits = 1; sa.max_mt = (k + 127) / 128; sa.tmem_cols = tmem_cols;
+  sa.n_nt = n_nt; sa.stages = stages; sa.splits = splits; sa.max_mt = max_mt; sa.tmem_cols = tmem_cols;
   sa.threshold = p->sim_threshold;
   sa.role = ctx->role; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
-  sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr; sa.tile_counters = nullptr;
-  sa.part = nullptr; sa.ss_part = nullptr; sa.smat = smat; sa.status = ctx->status;
+  sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr; sa.tile_counters = ctx->cnt_tiles;
+  sa.part = ctx->sim_part; sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
+  sa.smat = smat; sa.status = ctx->status;
   mark(ctx, "sim_kept", st);
-  launch_pdl(sim_kernel, dim3((k + 127) / 128, B, 1), dim3(SIM_THREADS), smem, st, map_a, map_b, sa);
+  launch_pdl(sim_kernel, dim3(max_mt, B, splits), dim3(SIM_THREADS), smem, st, map_a, map_b, sa);
   ASAP_TRY(after_launch(ctx, "sim_kept"));
 
   RouteArgs ra;

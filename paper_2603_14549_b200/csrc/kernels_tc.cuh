@@ -484,7 +484,7 @@ head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
 //                   row tile adds the slices in slice order and does the same epilogue.
 // Rows that were kept, or lie past the image span, are computed but not written.
 // The block that finishes a sample's last row tile groups the dropped tokens by destination.
-//   matrix mode:    (a.smat set, one slice) the row operand is the dense kept-row array too, and
+//   matrix mode:    (a.smat set) the row operand is the dense kept-row array too, and
 //                   the epilogue writes the whole keep_k x keep_k cosine matrix of the sample,
 //                   S[p][q] = <h_p, h_q> * (1/||h_p|| * 1/||h_q||), for the routing inside the
 //                   kept set; `tmap_h` is then a map of the kept rows with a 128-row box.
@@ -682,7 +682,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         uint32_t r[16];
         tmem_ld16(taddr + c, r);
         tmem_wait_ld();
-        if (a.smat) {
+        if (a.smat && !part) {
           if (v < a.keep_k && !bk->abort_flag) {
             const float inv_p = __ldg(kinv + v);
             float *srow = a.smat + ((size_t)b * a.keep_k + v) * a.keep_k + slot0 + c;
@@ -746,6 +746,16 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
             for (int t = 0; t < 4; ++t)
 #pragma unroll
               for (int e = 0; e < 16; ++e) acc[e] += x[t][e];
+          }
+          if (a.smat) {
+            if (v < a.keep_k && !bk->abort_flag) {
+              const float inv_p = __ldg(kinv + v);
+              float *srow = a.smat + ((size_t)b * a.keep_k + v) * a.keep_k + s0;
+#pragma unroll
+              for (int e = 0; e < 16; ++e)
+                if (s0 + e < a.keep_k) srow[e] = acc[e] * (inv_p * __ldg(kinv + s0 + e));
+            }
+            continue;
           }
 #pragma unroll
           for (int e = 0; e < 16; ++e) {

@@ -181,6 +181,23 @@ def config(name: str, B: Optional[int] = None, seed: Optional[int] = None,
                       seed, cents[:useB], 0.3, tile, out)
 
 
+def random_stage1(batch: "Batch", b: int, keep_k: int, seed: int):
+    """Stand-in for stage 1's results of sequence b, for exercising stage 2 alone at sizes where the
+    CPU oracle cannot afford stage 1: attention mass (positive, long-tailed), salience (uniform in
+    [0, 1], one exact 0 and one exact 1), a random kept subset and its complement, all seeded.
+    Returns (mass f32 [nv], salience f32 [nv], keep int32 [k] ascending, drop int32 [nv-k] ascending)."""
+    g = _sample_generator(seed, b, stream=20)
+    nv = int(batch.vis_len[b])
+    mass = torch.exp(torch.randn(nv, generator=g)).float()
+    sal = torch.rand(nv, generator=g).float()
+    sal[int(torch.randint(0, nv, (1,), generator=g))] = 0.0
+    sal[int(torch.randint(0, nv, (1,), generator=g))] = 1.0
+    perm = torch.randperm(nv, generator=g)
+    keep = torch.sort(perm[:keep_k]).values.to(torch.int32)
+    drop = torch.sort(perm[keep_k:]).values.to(torch.int32)
+    return mass.numpy(), sal.numpy(), keep.numpy(), drop.numpy()
+
+
 C5_SCHEDULE = (1152, 576, 288)
 
 

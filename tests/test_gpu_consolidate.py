@@ -38,7 +38,7 @@ def _stage1(batch, b, k):
     return f32(ref["mass"]), f32(ref["salience"]), ref["keep_idx"], ref["drop_idx"]
 
 
-def _run(ctx, batch, k, t, salience_override=None):
+def _run(ctx, batch, k, t, salience_override=None, stage1=None):
     B = batch.B
     p = A.Params(keep_k=k, sim_threshold=t)
     inp = A.make_inputs(batch, DEV)
@@ -47,7 +47,7 @@ def _run(ctx, batch, k, t, salience_override=None):
     keep = torch.zeros(B, k, dtype=torch.int32); drop = torch.full((B, mv - k), -1, dtype=torch.int32)
     st1 = []
     for b in range(B):
-        m, s, kp, dp = _stage1(batch, b, k)
+        m, s, kp, dp = (stage1 or _stage1)(batch, b, k)
         if salience_override is not None:
             s = salience_override(b, s)
         nv = int(batch.vis_len[b])
@@ -62,10 +62,10 @@ def _run(ctx, batch, k, t, salience_override=None):
     return out, n_abs.cpu().numpy(), st1
 
 
-def _check(batch, k, t, out, n_abs, st1):
+def _check(batch, k, t, out, n_abs, st1, samples=None):
     ocu = out.out_cu_seqlens.cpu().numpy()
     total_abs = 0
-    for b in range(batch.B):
+    for b in (range(batch.B) if samples is None else samples):
         rows = batch.sample_rows(b)
         v0, nv = int(batch.vis_start[b]), int(batch.vis_len[b])
         m, s, kp, dp = st1[b]
@@ -186,3 +186,22 @@ def test_bit_matrix_in_global_memory_for_large_keep(ctx):
     batch = W.tiny(B=1, n_vis=[3000], text_lens=[8], H=2, keep_k=1400, seed=514, centres=90)
     out, n_abs, st1 = _run(ctx, batch, 1400, 0.85)
     assert _check(batch, 1400, 0.85, out, n_abs, st1) > 0
+
+
+@pytest.fixture(scope="module")
+def big_ctx():
+    c = A.asap_init(0, max_total_tokens=32 * (35 + 2304 + 128) + 2304, max_B=32, max_H=40, max_D=5120,
+                    max_keep_rows=32 * 1152)
+    yield c
+    A.asap_free(c)
+
+
+@pytest.mark.parametrize("name,t,samples", [("c2", 0.8, None), ("c3", 0.8, [0, 7]), ("c5", 0.85, [31])])
+def test_consolidate_at_benchmark_sizes(big_ctx, name, t, samples):
+    """Full batches of the benchmark shapes (hidden sizes 4096 / 5120, keep_k 64 / 320 / 1152) with
+    seeded stand-ins for stage 1's results; the oracle checks the listed sequences."""
+    batch = W.config(name)
+    k = batch.keep_k
+    out, n_abs, st1 = _run(big_ctx, batch, k, t, stage1=lambda bt, b, kk: W.random_stage1(bt, b, kk, 900))
+    assert np.all(n_abs >= 0) and np.all(n_abs <= np.asarray(batch.vis_len) - k)
+    assert _check(batch, k, t, out, n_abs, st1, samples=samples) > 0
