@@ -25,6 +25,9 @@ Parity status of each function (what pins it, see tests/test_oracle_pins.py):
                                  plain top-k gather; twins; anchors are never absorbed; set sizes;
                                  Eq. 5 weight conservation; library sort for the refill).  Not pinned
                                  by the paper: the reading of which anchor absorbs a token.
+  masked_attention      pinned  (library float64 scaled-dot-product attention in the causal case; value
+                                 rows all equal -> output equals that row; one-hot values recover the
+                                 Eq. 4 probabilities, themselves pinned above; hand-worked 3-token case)
   compact / prune_step  pinned  (invariants: k kept ascending; identity at k = N_v;
                                  plain attention top-k with mask and merge off; twins)
   Not pinned by anything the paper prints: that the ranking rule (mean of the Eq. 4
@@ -371,6 +374,25 @@ def consolidate_sample(hidden_bits, pos_ids, v0: int, nv: int, mass, s_hat, keep
     return dict(dest=dest, margin=margin, n_absorbed=len(absorbed), refill=refill, final_keep=final,
                 merged=rows, merged_mask=merged_mask, out_hidden=out_hidden, out_hidden_bits=out_bits,
                 out_pos=np.asarray(pos_ids)[src_row].astype(np.int32), src_row=src_row)
+
+
+# ----------------------------------------------------------------------------------
+# The layer's attention under the SG-BiMask (Eq. 4 applied to the values)
+# ----------------------------------------------------------------------------------
+def masked_attention(q_bits, k_bits, v_bits, v0: int, nv: int, m: Optional[np.ndarray],
+                     mask_enable: bool = True) -> np.ndarray:
+    """Eq. 4: O^h = Softmax(W^h + M_bidir) V^h for every query row of one sequence and every head.
+    q, k, v: bf16 bit patterns [n, H, d]; m: Eq. 3's vector over the image span (ignored with the
+    mask off, which gives the causal attention of Sec. 3.2).  Returns float64 [n, H, d]."""
+    q, k, v = bf16_bits_to_f64(q_bits), bf16_bits_to_f64(k_bits), bf16_bits_to_f64(v_bits)
+    n, H, _ = q.shape
+    rows = np.arange(n)
+    M = mask_matrix(n, rows, v0, nv, m, mask_enable)
+    out = np.empty_like(v)
+    for h in range(H):
+        A = attention_probs(q, k, h, rows, v0, nv, m, mask_enable, M)
+        out[:, h, :] = A @ v[:, h, :]
+    return out
 
 
 def compact_rows(cache: np.ndarray, src_row: np.ndarray) -> np.ndarray:

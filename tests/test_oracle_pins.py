@@ -612,3 +612,53 @@ def test_consolidation_never_absorbs_more_than_the_pool_can_refill():
     order = sorted(range(40), key=lambda p: (-s_hat[keep[p]], keep[p]))
     assert sorted(np.nonzero(r["dest"] >= 0)[0].tolist()) == sorted(order[1:7])   # the first six after the top one
     assert np.all(r["dest"][order[1:7]] == order[0])
+
+
+# ----------------------------------------------------------------------------- Eq. 4 applied to the values
+def _bf16_bits(x):
+    return bits(torch.tensor(np.asarray(x), dtype=torch.float32).to(torch.bfloat16))
+
+
+def test_masked_attention_causal_case_is_library_attention():
+    rng = np.random.default_rng(31)
+    n, H, d = 23, 3, 16
+    qb, kb, vb = (_bf16_bits(rng.standard_normal((n, H, d))) for _ in range(3))
+    got = O.masked_attention(qb, kb, vb, 4, 9, None, mask_enable=False)
+    tq, tk, tv = (torch.from_numpy(O.bf16_bits_to_f64(x)).permute(1, 0, 2) for x in (qb, kb, vb))
+    want = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True).permute(1, 0, 2).numpy()
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-14)
+
+
+def test_masked_attention_hand_worked_three_tokens():
+    """One head, d = 1, all tokens visual, q = 0 so every logit is 0: the weights are the mask's alone.
+    lambda = (.5, .25, 1): row 0 admits key 0 fully and keys 1, 2 with weights .25 and 1;
+    row 1 admits 0, 1 fully and key 2 with weight 1; row 2 is causal.  v = (8, 4, 2)."""
+    lam = np.array([0.5, 0.25, 1.0])
+    z = _bf16_bits(np.zeros((3, 1, 1)))
+    v = _bf16_bits(np.array([8.0, 4.0, 2.0]).reshape(3, 1, 1))
+    out = O.masked_attention(z, z, v, 0, 3, np.log(lam))[:, 0, 0]
+    want = [(8 + .25 * 4 + 1 * 2) / (1 + .25 + 1), (8 + 4 + 1 * 2) / 3, (8 + 4 + 2) / 3]
+    assert np.allclose(out, want, rtol=1e-14)
+
+
+def test_masked_attention_invariants():
+    rng = np.random.default_rng(32)
+    n, H, d, v0, nv = 19, 2, 8, 3, 10
+    qb, kb = (_bf16_bits(rng.standard_normal((n, H, d))) for _ in range(2))
+    m = np.log(rng.uniform(0.05, 1.0, nv))
+    # equal value rows: any convex combination returns that row
+    row = rng.standard_normal((1, H, d))
+    vb = _bf16_bits(np.repeat(row, n, axis=0))
+    out = O.masked_attention(qb, kb, vb, v0, nv, m)
+    assert np.allclose(out, O.bf16_bits_to_f64(vb), rtol=1e-13, atol=1e-15)
+    # one-hot values (d = n): the output IS the probability matrix of Eq. 4
+    q2, k2 = (_bf16_bits(rng.standard_normal((n, 1, n))) for _ in range(2))
+    eye = _bf16_bits(np.eye(n).reshape(n, 1, n))
+    out = O.masked_attention(q2, k2, eye, v0, nv, m)[:, 0, :]
+    A = O.attention_probs(O.bf16_bits_to_f64(q2), O.bf16_bits_to_f64(k2), 0, np.arange(n), v0, nv, m, True)
+    assert np.allclose(out, A, rtol=1e-13, atol=1e-16) and np.allclose(out.sum(axis=1), 1.0)
+    # text and system rows never see the mask; visual rows do
+    vb = _bf16_bits(rng.standard_normal((n, H, d)))
+    on, off = O.masked_attention(qb, kb, vb, v0, nv, m), O.masked_attention(qb, kb, vb, v0, nv, None, False)
+    vis = np.zeros(n, bool); vis[v0:v0 + nv - 1] = True          # the last visual row has no future visual key
+    assert np.array_equal(on[~vis], off[~vis]) and np.all(np.abs(on[vis] - off[vis]).max(axis=(1, 2)) > 1e-6)
