@@ -170,6 +170,23 @@ asap_status asap_consolidate(asap_ctx *ctx, const asap_inputs *in, const asap_pa
                              const int32_t *drop_idx, void *scratch, size_t scratch_bytes,
                              const asap_outputs *out, int32_t *n_absorbed, void *stream);
 
+/* The layer's attention under the salience-guided bidirectional mask (Sec. 4.1, Eq. 3-4):
+ *     out[i, h, :] = sum_j Softmax_j( q_i^h . k_j^h / sqrt(head_dim) + M_ij ) v_j^h
+ * for every row i of every sequence, with M_ij = 0 for j <= i, M_ij = mask_log[b][j - vis_start]
+ * for i < j when both i and j lie in the image span, and -infinity otherwise (other sequences of
+ * the packed batch are never attended).  With p->mask_enable == 0 this is causal attention and
+ * `mask_log` may be NULL; otherwise `mask_log` is the device array [B, max_vis] that asap_score
+ * writes (asap_outputs::mask_log).  Only B, H, head_dim, D, total_tokens, the bounds, cu_seqlens,
+ * the spans, q and k of `in` are read; `p` must be a valid parameter set (as for asap_score).
+ * `v` and `out` are bf16 [total_tokens, H, head_dim] device tensors, 16-byte aligned, that must
+ * not overlap.  `scratch`: caller-owned device memory of at least
+ * asap_attention_scratch_bytes(total_tokens, D) bytes, 16-byte aligned (the transposed values);
+ * nothing is kept in it between calls.  Two launches (plus the validation kernel). */
+size_t asap_attention_scratch_bytes(int32_t total_tokens, int32_t D);
+asap_status asap_attention(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+                           const float *mask_log, const void *v, void *scratch, size_t scratch_bytes,
+                           void *out, void *stream);
+
 /* Steps 1a-5 back to back on `stream`; fills every field of `out`. */
 asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                             const asap_outputs *out, void *stream);

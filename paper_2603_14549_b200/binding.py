@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "ASAP_OK", -1: "ASAP_ERR_INVALID", -2: "ASAP_ERR_ALIGN", -3: 
 
 EXPORTS = ("asap_init", "asap_score", "asap_select", "asap_merge", "asap_prune_step", "asap_check",
            "asap_last_error", "asap_launch_count", "asap_free", "asap_profile", "asap_profile_read", "asap_select_static", "asap_compact_kv",
-           "asap_consolidate", "asap_consolidate_scratch_bytes")
+           "asap_consolidate", "asap_consolidate_scratch_bytes", "asap_attention", "asap_attention_scratch_bytes")
 
 
 class AsapError(RuntimeError):
@@ -97,6 +97,11 @@ def load_library() -> C.CDLL:
     lib.asap_consolidate.argtypes = [C.c_void_p, C.POINTER(CInputs), C.POINTER(CParams), C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(COutputs),
                                      C.c_void_p, C.c_void_p]
+    lib.asap_attention_scratch_bytes.restype = C.c_size_t
+    lib.asap_attention_scratch_bytes.argtypes = [C.c_int32, C.c_int32]
+    lib.asap_attention.restype = C.c_int
+    lib.asap_attention.argtypes = [C.c_void_p, C.POINTER(CInputs), C.POINTER(CParams), C.c_void_p, C.c_void_p,
+                                   C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     lib.asap_check.restype = C.c_int
     lib.asap_check.argtypes = [C.c_void_p, C.c_void_p]
     lib.asap_last_error.restype = C.c_char_p
@@ -266,6 +271,18 @@ def asap_merge(ctx, inp: Inputs, params: Params, salience: torch.Tensor, keep_id
     ci, cp, co = inp.c_struct(), params.c_struct(), out.c_struct()
     _raise(ctx, load_library().asap_merge(ctx, C.byref(ci), C.byref(cp), _ptr(salience), _ptr(keep_idx),
                                           _ptr(drop_idx), C.byref(co), _stream(stream)))
+
+
+def asap_attention_scratch_bytes(total_tokens: int, D: int) -> int:
+    return int(load_library().asap_attention_scratch_bytes(int(total_tokens), int(D)))
+
+
+def asap_attention(ctx, inp: Inputs, params: Params, mask_log: Optional[torch.Tensor], v: torch.Tensor,
+                   scratch: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    """out[i, h, :] = sum_j Softmax_j(q_i.k_j / sqrt(d) + M_ij) v_j; `v`, `out`: bf16 [total_tokens, H, head_dim]."""
+    ci, cp = inp.c_struct(), params.c_struct()
+    _raise(ctx, load_library().asap_attention(ctx, C.byref(ci), C.byref(cp), _ptr(mask_log), _ptr(v), _ptr(scratch),
+                                              int(scratch.numel() * scratch.element_size()), _ptr(out), _stream(stream)))
 
 
 def asap_consolidate_scratch_bytes(B: int, keep_k: int) -> int:

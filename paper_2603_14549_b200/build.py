@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libasap.so")
 SOURCES = ["asap_api.cu"]
-HEADERS = ["common.cuh", "kernels_stream.cuh", "kernels_tc.cuh"]
+HEADERS = ["common.cuh", "kernels_stream.cuh", "kernels_tc.cuh", "kernels_attn.cuh"]
 
 
 def _stale() -> bool:

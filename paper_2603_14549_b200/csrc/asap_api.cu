@@ -13,6 +13,7 @@
 #include "../../include/asap.h"
 #include "kernels_stream.cuh"
 #include "kernels_tc.cuh"
+#include "kernels_attn.cuh"
 
 using namespace asap;
 
@@ -75,9 +76,9 @@ bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 // 2-D bf16 tensor [rows, cols] row-major, box = 64 columns x box_rows rows, 128-byte swizzle.
 bool make_map(asap_ctx *ctx, CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols,
-              uint32_t box_rows) {
+              uint32_t box_rows, uint64_t pitch_elems = 0) {
   cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
+  cuuint64_t strides[1] = {(pitch_elems ? pitch_elems : cols) * 2};
   cuuint32_t box[2] = {64, box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims,
@@ -545,6 +546,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM_BYTES);
   // lowest priority: when both streams have blocks to place, the score kernel's go first and the
   // mass kernels fill what is left of each SM
   int prio_least = 0, prio_greatest = 0;
@@ -598,6 +600,44 @@ asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *
                                                                          out->best_sim, merging(in, p) ? 1 : 0);
   ASAP_TRY(after_launch(ctx, "role_map"));
   return finish(ctx, launch_merge(ctx, in, p, salience, keep_idx, drop_idx, out, st), st);
+}
+
+size_t asap_attention_scratch_bytes(int32_t total_tokens, int32_t D) {
+  if (total_tokens <= 0 || D <= 0) return 0;
+  return align_up((size_t)total_tokens, 8) * (size_t)D * sizeof(__nv_bfloat16);
+}
+
+asap_status asap_attention(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *mask_log,
+                           const void *v, void *scratch, size_t scratch_bytes, void *out, void *stream) {
+  asap_outputs none;
+  memset(&none, 0, sizeof(none));
+  ASAP_TRY(validate(ctx, in, p, &none, NEED_QK));
+  if (!v || !out) return fail(ctx, ASAP_ERR_INVALID, "asap_attention: null v / out");
+  if (!aligned16(v) || !aligned16(out)) return fail(ctx, ASAP_ERR_ALIGN, "asap_attention: v / out must be 16-byte aligned");
+  if (p->mask_enable && !mask_log) return fail(ctx, ASAP_ERR_INVALID, "asap_attention: mask_enable needs mask_log");
+  if (!scratch || !aligned16(scratch) || scratch_bytes < asap_attention_scratch_bytes(in->total_tokens, in->D))
+    return fail(ctx, ASAP_ERR_WORKSPACE, "asap_attention: scratch is null, unaligned or smaller than asap_attention_scratch_bytes");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int total = in->total_tokens, D = in->D;
+  const int total_pad = (int)align_up((size_t)total, 8);
+  CUtensorMap map_q, map_k, map_vt;
+  if (!make_map(ctx, &map_q, in->q, (uint64_t)total, (uint64_t)D, 128) ||
+      !make_map(ctx, &map_k, in->k, (uint64_t)total, (uint64_t)D, 128) ||
+      !make_map(ctx, &map_vt, scratch, (uint64_t)D, (uint64_t)total, 128, (uint64_t)total_pad))
+    return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for q / k / transposed v");
+  ASAP_TRY(launch_prepare(ctx, in, p, nullptr, 0x7fffffff, st));
+  mark(ctx, "transpose_v", st);
+  launch_pdl(transpose_v_kernel, dim3((total_pad + TR_TILE - 1) / TR_TILE, (D + TR_TILE - 1) / TR_TILE), dim3(TR_THREADS), 0, st,
+             static_cast<const __nv_bfloat16 *>(v), static_cast<__nv_bfloat16 *>(scratch), total, total_pad, D);
+  ASAP_TRY(after_launch(ctx, "transpose_v"));
+  AttnArgs aa;
+  aa.desc = ctx->desc; aa.H = in->H; aa.D = D; aa.max_vis = in->max_vis; aa.mask_enable = p->mask_enable ? 1 : 0;
+  aa.scale_log2 = 1.4426950408889634f / sqrtf((float)in->head_dim);
+  aa.mask_log = mask_log; aa.out = static_cast<__nv_bfloat16 *>(out); aa.status = ctx->status;
+  mark(ctx, "attention", st);
+  launch_pdl(attn_kernel, dim3((in->max_seq + 127) / 128, in->H, in->B), dim3(AT_THREADS), (size_t)AT_SMEM_BYTES, st,
+             map_q, map_k, map_vt, aa);
+  return finish(ctx, after_launch(ctx, "attention"), st);
 }
 
 size_t asap_consolidate_scratch_bytes(int32_t B, int32_t keep_k) {
@@ -704,11 +744,12 @@ asap_status asap_check(asap_ctx *ctx, void *stream) {
   if (word == 0) { ctx->err[0] = 0; return ASAP_OK; }
   cudaMemsetAsync(ctx->status, 0, sizeof(uint32_t), st);
   cudaStreamSynchronize(st);
-  return fail(ctx, ASAP_ERR_DEVICE, "device status 0x%x:%s%s%s%s", word,
+  return fail(ctx, ASAP_ERR_DEVICE, "device status 0x%x:%s%s%s%s%s", word,
               (word & STATUS_BAD_SAMPLE) ? " a per-sample span failed validation (sample skipped);" : "",
               (word & STATUS_OUT_CAPACITY) ? " shortened batch exceeds out_rows_capacity (nothing written);" : "",
               (word & STATUS_SCORE_TIMEOUT) ? " a wait timed out in the score kernel;" : "",
-              (word & STATUS_SIM_TIMEOUT) ? " a wait timed out in the similarity kernel;" : "");
+              (word & STATUS_SIM_TIMEOUT) ? " a wait timed out in the similarity kernel;" : "",
+              (word & STATUS_ATTN_TIMEOUT) ? " a wait timed out in the attention kernel;" : "");
 }
 
 asap_status asap_profile(asap_ctx *ctx, int enable) {

@@ -181,6 +181,17 @@ def config(name: str, B: Optional[int] = None, seed: Optional[int] = None,
                       seed, cents[:useB], 0.3, tile, out)
 
 
+def draw_values(batch: "Batch", seed: int) -> torch.Tensor:
+    """Value projections for the layer's attention: iid N(0, 1), bf16 [total, H, head_dim], one seeded
+    stream per sequence (sequence b is the same whatever the batch prefix)."""
+    v = torch.empty(batch.total, batch.H, batch.head_dim, dtype=torch.bfloat16)
+    for b in range(batch.B):
+        rows = batch.sample_rows(b)
+        g = _sample_generator(seed, b, stream=30)
+        v[rows] = torch.randn(rows.stop - rows.start, batch.H, batch.head_dim, generator=g).to(torch.bfloat16)
+    return v
+
+
 def random_stage1(batch: "Batch", b: int, keep_k: int, seed: int):
     """Stand-in for stage 1's results of sequence b, for exercising stage 2 alone at sizes where the
     CPU oracle cannot afford stage 1: attention mass (positive, long-tailed), salience (uniform in

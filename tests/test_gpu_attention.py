@@ -1,0 +1,108 @@
+"""asap_attention (Eq. 4 applied to the values: the layer's attention under the SG-BiMask) against
+the CPU oracle, through the C ABI, every output element.
+
+The mask vector m_j given to both sides is the oracle's (Eq. 1-3), rounded to fp32.
+Tolerance: |g - o| <= max(2e-2, 2^-7 |o|) -- the bar of the merged rows: probabilities enter the
+second contraction as bf16 (relative error 2^-9 each, averaged over a row), the output is rounded to
+bf16 once (2^-9 relative)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import asap_oracle as O
+from paper_2603_14549_b200 import binding as A
+from paper_2603_14549_b200 import workloads as W
+from tests.helpers import bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = A.asap_init(0, max_total_tokens=40000, max_B=16, max_H=8, max_D=1024)
+    yield c
+    A.asap_free(c)
+
+
+def _mask_vectors(batch, lambda_max):
+    mv = int(batch.vis_len.max())
+    m = torch.zeros(batch.B, mv)
+    ms = []
+    for b in range(batch.B):
+        rows = batch.sample_rows(b)
+        q, k = O.bf16_bits_to_f64(bits(batch.q[rows])), O.bf16_bits_to_f64(bits(batch.k[rows]))
+        v0, nv = int(batch.vis_start[b]), int(batch.vis_len[b])
+        mb = O.mask_log(O.salience(O.attention_mass(q, k, v0, nv)), lambda_max).astype(np.float32)
+        m[b, :nv] = torch.from_numpy(mb)
+        ms.append(mb.astype(np.float64))
+    return m, ms
+
+
+def _run(ctx, batch, v, m, mask_enable=True):
+    inp = A.make_inputs(batch, DEV)
+    out = torch.full((batch.total, batch.H, batch.head_dim), 7.0, dtype=torch.bfloat16, device=DEV)
+    scratch = torch.empty(A.asap_attention_scratch_bytes(batch.total, batch.D), dtype=torch.uint8, device=DEV)
+    p = A.Params(keep_k=int(batch.vis_len.min()), mask_enable=mask_enable)
+    A.asap_attention(ctx, inp, p, None if m is None else m.to(DEV), v.to(DEV), scratch, out)
+    torch.cuda.synchronize(); A.asap_check(ctx)
+    return out.cpu()
+
+
+def _compare(batch, v, out, ms, mask_enable=True):
+    worst = 0.0
+    for b in range(batch.B):
+        rows = batch.sample_rows(b)
+        ref = O.masked_attention(bits(batch.q[rows]), bits(batch.k[rows]), bits(v[rows]), int(batch.vis_start[b]),
+                                 int(batch.vis_len[b]), ms[b] if mask_enable else None, mask_enable)
+        g = O.bf16_bits_to_f64(bits(out[rows]))
+        err = np.abs(g - ref)
+        assert np.all(err <= np.maximum(2e-2, np.abs(ref) * 2.0 ** -7)), (b, err.max(), np.unravel_index(err.argmax(), err.shape))
+        worst = max(worst, err.max())
+    return worst
+
+
+@pytest.mark.parametrize("nvs,texts,lam", [
+    ([300, 170, 520], [9, 30, 4], 1.0),          # ragged; sequence starts off the 8-row grid
+    ([130, 257], [1, 140], 0.3),                 # text longer than a tile; image span ends one past a tile edge
+    ([64], [3], 1.0),                            # a single, partly filled tile
+], ids=["ragged3", "longtext", "single"])
+def test_attention_matches_oracle(ctx, nvs, texts, lam):
+    batch = W.tiny(B=len(nvs), n_vis=nvs, text_lens=texts, H=2, keep_k=8, seed=600 + len(nvs))
+    v = W.draw_values(batch, 77)
+    m, ms = _mask_vectors(batch, lam)
+    out = _run(ctx, batch, v, m)
+    print("attention max abs err", _compare(batch, v, out, ms))
+
+
+def test_mask_off_is_causal_attention_and_only_visual_rows_differ(ctx):
+    batch = W.tiny(B=2, n_vis=[200, 333], text_lens=[17, 5], H=2, keep_k=8, seed=610)
+    v = W.draw_values(batch, 78)
+    m, ms = _mask_vectors(batch, 1.0)
+    off = _run(ctx, batch, v, None, mask_enable=False)
+    _compare(batch, v, off, ms, mask_enable=False)
+    on = _run(ctx, batch, v, m)
+    for b in range(2):
+        rows = batch.sample_rows(b)
+        v0, nv = int(batch.vis_start[b]), int(batch.vis_len[b])
+        a, c = bits(on[rows]), bits(off[rows])
+        vis = np.zeros(rows.stop - rows.start, bool); vis[v0:v0 + nv - 1] = True
+        assert np.array_equal(a[~vis], c[~vis])             # system, text and the last visual row: bit-identical
+        assert np.any(a[vis] != c[vis])
+
+
+def test_attention_argument_errors(ctx):
+    batch = W.tiny(B=1, n_vis=[100], text_lens=[4], H=2, keep_k=8, seed=611)
+    inp = A.make_inputs(batch, DEV)
+    v = W.draw_values(batch, 79).to(DEV)
+    out = torch.empty_like(v)
+    big = torch.empty(A.asap_attention_scratch_bytes(batch.total, batch.D), dtype=torch.uint8, device=DEV)
+    n0 = A.asap_launch_count(ctx)
+    with pytest.raises(A.AsapError) as e:
+        A.asap_attention(ctx, inp, A.Params(keep_k=8), None, v, big, out)          # mask on, no vector
+    assert e.value.status == -1
+    with pytest.raises(A.AsapError) as e:
+        A.asap_attention(ctx, inp, A.Params(keep_k=8, mask_enable=False), None, v, big[:64], out)
+    assert e.value.status == -3
+    assert A.asap_launch_count(ctx) == n0
+    assert A.asap_attention_scratch_bytes(13, 256) == 16 * 256 * 2
