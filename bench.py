@@ -355,6 +355,41 @@ def run_cuda(args):
                 "absorbed_per_sequence": float(n_abs.float().mean()), "kernel_us": ck}
         del scratch, out2
 
+    # ---- the layer's attention under the SG-BiMask (Eq. 4 applied to the values), timed apart from the
+    # step with the step's own mask vector
+    attn = None
+    if args.attention_iters > 0:
+        v_dev = W.draw_values(batch, 4242).to(device)
+        a_out = torch.empty_like(v_dev)
+        a_scr = torch.empty(A.asap_attention_scratch_bytes(batch.total, batch.D), dtype=torch.uint8, device=device)
+        acall = lambda i: A.asap_attention(ctx, copies[i % n_copies], params, out.mask_log, v_dev, a_scr, a_out, stream)
+        for i in range(2):
+            acall(i)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a0.record(stream)
+        for i in range(args.attention_iters):
+            acall(i)
+        a1.record(stream)
+        torch.cuda.synchronize()
+        A.asap_check(ctx)
+        A.asap_profile(ctx, True)
+        for i in range(min(args.attention_iters, 10)):
+            acall(i)
+        torch.cuda.synchronize()
+        ak = {name: ms / max(n, 1) * 1e3 for name, (n, ms) in A.asap_profile_read(ctx).items()}
+        A.asap_profile(ctx, False)
+        # admitted (query, key) pairs: the causal triangle plus, for rows of the image span, the later keys of the span
+        pairs = 0
+        for b_ in range(batch.B):
+            n_, nv_ = int(batch.cu_seqlens[b_ + 1] - batch.cu_seqlens[b_]), int(batch.vis_len[b_])
+            pairs += n_ * (n_ + 1) // 2 + nv_ * (nv_ - 1) // 2
+        a_us = a0.elapsed_time(a1) / args.attention_iters * 1e3
+        a_flops = 4.0 * batch.head_dim * pairs * batch.H
+        attn = {"us": a_us, "admitted_pairs": pairs, "flops": a_flops, "TFLOPs": a_flops / a_us / 1e6,
+                "frac_of_bf16_peak": a_flops / a_us / 1e6 / peaks["bf16_tflops"], "kernel_us": ak}
+        del v_dev, a_out, a_scr
+
     # ---- end to end from pinned host memory
     e2e = None
     if not args.no_e2e:
@@ -450,7 +485,7 @@ def run_cuda(args):
         "latency_us": {"p10": per_step[len(per_step) // 10] * 1e3, "p50": per_step[len(per_step) // 2] * 1e3,
                        "p90": per_step[(len(per_step) * 9) // 10] * 1e3},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "kernels": kernels,
-        "cpu_baseline": cpu, "kv_compaction": kv, "consolidate_within_kept": cons,
+        "cpu_baseline": cpu, "kv_compaction": kv, "consolidate_within_kept": cons, "masked_attention": attn,
     }
     print(json.dumps(line))
     R.shutdown()
@@ -471,6 +506,8 @@ def main():
                     help="also time KV-cache compaction of this many layers (0 = skip)")
     ap.add_argument("--consolidate-threshold", type=float, default=0.8,
                     help="also time asap_consolidate (Sec. 4.2 inside the kept set) with this threshold t")
+    ap.add_argument("--attention-iters", type=int, default=10,
+                    help="also time asap_attention (the layer's attention under the SG-BiMask) this many times (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--ref-sequences", type=int, default=2,

@@ -380,15 +380,16 @@ def consolidate_sample(hidden_bits, pos_ids, v0: int, nv: int, mass, s_hat, keep
 # The layer's attention under the SG-BiMask (Eq. 4 applied to the values)
 # ----------------------------------------------------------------------------------
 def masked_attention(q_bits, k_bits, v_bits, v0: int, nv: int, m: Optional[np.ndarray],
-                     mask_enable: bool = True) -> np.ndarray:
+                     mask_enable: bool = True, rows: Optional[np.ndarray] = None) -> np.ndarray:
     """Eq. 4: O^h = Softmax(W^h + M_bidir) V^h for every query row of one sequence and every head.
     q, k, v: bf16 bit patterns [n, H, d]; m: Eq. 3's vector over the image span (ignored with the
-    mask off, which gives the causal attention of Sec. 3.2).  Returns float64 [n, H, d]."""
+    mask off, which gives the causal attention of Sec. 3.2).  `rows`: the query rows wanted (default
+    all).  Returns float64 [len(rows), H, d]."""
     q, k, v = bf16_bits_to_f64(q_bits), bf16_bits_to_f64(k_bits), bf16_bits_to_f64(v_bits)
-    n, H, _ = q.shape
-    rows = np.arange(n)
+    n, H, d = q.shape
+    rows = np.arange(n) if rows is None else np.asarray(rows)
     M = mask_matrix(n, rows, v0, nv, m, mask_enable)
-    out = np.empty_like(v)
+    out = np.empty((len(rows), H, d))
     for h in range(H):
         A = attention_probs(q, k, h, rows, v0, nv, m, mask_enable, M)
         out[:, h, :] = A @ v[:, h, :]

@@ -106,3 +106,41 @@ def test_attention_argument_errors(ctx):
     assert e.value.status == -3
     assert A.asap_launch_count(ctx) == n0
     assert A.asap_attention_scratch_bytes(13, 256) == 16 * 256 * 2
+
+
+@pytest.fixture(scope="module")
+def big_ctx():
+    c = A.asap_init(0, max_total_tokens=64 * (35 + 2880 + 256), max_B=64, max_H=40, max_D=5120)
+    yield c
+    A.asap_free(c)
+
+
+@pytest.mark.parametrize("name,B,samples", [("c2", None, [0, 15]), ("c4", 4, [3]), ("c5", 2, [1])])
+def test_attention_at_benchmark_sizes_sampled_rows(big_ctx, name, B, samples):
+    """Benchmark shapes at full width (32 / 40 heads); the oracle checks 48 sampled query rows of the
+    listed sequences (system, image-span and text rows, the span's first and last rows among them)."""
+    batch = W.config(name, B=B)
+    v = W.draw_values(batch, 80)
+    mv = int(batch.vis_len.max())
+    m = torch.zeros(batch.B, mv)
+    ms = {}
+    for b in range(batch.B):
+        rows = batch.sample_rows(b)
+        nv = int(batch.vis_len[b])
+        if b in samples:
+            q, k = O.bf16_bits_to_f64(bits(batch.q[rows])), O.bf16_bits_to_f64(bits(batch.k[rows]))
+            mb = O.mask_log(O.salience(O.attention_mass(q, k, int(batch.vis_start[b]), nv)), 1.0).astype(np.float32)
+        else:                                                         # unchecked sequences: any valid vector
+            mb = np.log(np.linspace(0.01, 1.0, nv)).astype(np.float32)
+        m[b, :nv] = torch.from_numpy(mb)
+        ms[b] = mb.astype(np.float64)
+    out = _run(big_ctx, batch, v, m)
+    rng = np.random.default_rng(81)
+    for b in samples:
+        rows = batch.sample_rows(b)
+        n, v0, nv = rows.stop - rows.start, int(batch.vis_start[b]), int(batch.vis_len[b])
+        pick = np.unique(np.concatenate([[0, v0 - 1, v0, v0 + nv - 1, v0 + nv, n - 1], rng.integers(0, n, 42)]))
+        ref = O.masked_attention(bits(batch.q[rows]), bits(batch.k[rows]), bits(v[rows]), v0, nv, ms[b], True, rows=pick)
+        g = O.bf16_bits_to_f64(bits(out[rows][pick]))
+        err = np.abs(g - ref)
+        assert np.all(err <= np.maximum(2e-2, np.abs(ref) * 2.0 ** -7)), (b, err.max())
