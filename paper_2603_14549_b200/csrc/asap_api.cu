@@ -635,7 +635,7 @@ asap_status asap_attention(asap_ctx *ctx, const asap_inputs *in, const asap_para
   aa.scale_log2 = 1.4426950408889634f / sqrtf((float)in->head_dim);
   aa.mask_log = mask_log; aa.out = static_cast<__nv_bfloat16 *>(out); aa.status = ctx->status;
   mark(ctx, "attention", st);
-  launch_pdl(attn_kernel, dim3((in->max_seq + 127) / 128, in->H, in->B), dim3(AT_THREADS), (size_t)AT_SMEM_BYTES, st,
+  launch_pdl(attn_kernel, dim3((in->max_seq + 255) / 256, in->H, in->B), dim3(AT_THREADS), (size_t)AT_SMEM_BYTES, st,
              map_q, map_k, map_vt, aa);
   return finish(ctx, after_launch(ctx, "attention"), st);
 }

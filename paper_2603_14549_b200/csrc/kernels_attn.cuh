@@ -3,15 +3,18 @@
 //
 //   transpose_v_kernel  V [tokens, D] -> V^T [D, tokens] (row pitch padded to 8 tokens), so that
 //                       a value tile can be loaded as a K-major MMA operand like every other tile.
-//   attn_kernel         one block per (128 query rows, head, sequence).  For every tile of 128
-//                       keys:  S = Q K^T on tcgen05 into tensor memory, the softmax warps turn S
-//                       into probabilities relative to the running row maximum (Eq. 3's m_j is
-//                       added for the future keys of the image span on rows of the image span,
-//                       nothing else above the diagonal is admitted), write them as a bf16
-//                       operand tile into shared memory, and  O_tile = P V  runs on tcgen05 again;
-//                       the softmax warps fold O_tile into their fp32 running output with the
-//                       usual rescaling.  M_bidir is never materialised: it is the vector m_j
-//                       plus position tests.
+//   attn_kernel         one block per (two tiles of 128 query rows, head, sequence); the two row
+//                       tiles share every key / value tile and take turns on the tensor pipe.
+//                       For every tile of 128 keys:  S = Q K^T on tcgen05 into tensor memory; the
+//                       row tile's four softmax warps read S once (one thread per row), add Eq. 3's
+//                       m_j for the future keys of the image span on rows of the image span (nothing
+//                       else above the diagonal is admitted), turn the logits into probabilities
+//                       relative to a reference maximum and store them as bf16 over S's own columns;
+//                       O += P V then runs with P read from tensor memory and O accumulated in
+//                       tensor memory.  The reference maximum only moves (and O is only rescaled)
+//                       when a row's maximum has grown by more than 2^8; the final division by the
+//                       row sum makes the result independent of the reference.  M_bidir is never
+//                       materialised: it is the vector m_j plus position tests.
 //
 // Key tiles start at the sequence's first packed row rounded DOWN to a multiple of 8, because the
 // token coordinate is the contiguous one of V^T and a TMA copy must start on a 16-byte boundary;
@@ -61,15 +64,16 @@ transpose_v_kernel(const __nv_bfloat16 *__restrict__ v, __nv_bfloat16 *__restric
 }
 
 // ---------------------------------------------------------------------------------------
-constexpr int AT_THREADS = 192;                 // warp 0: copies, warp 1: MMA issue, warps 2-5: softmax
+constexpr int AT_THREADS = 320;                 // warp 0: copies, warp 1: MMA issue, warps 2-9: two softmax groups
 constexpr int AT_TILE_BYTES = 128 * 128 * 2;    // 128 rows x 128 bf16 as two 64-column blocks of 16 KB
 constexpr int AT_BLOCK_BYTES = AT_TILE_BYTES / 2;
 constexpr int AT_STAGES = 2;                    // a stage = one key tile + one value tile
 constexpr int AT_MAIN_BYTES = 2 * AT_TILE_BYTES + AT_STAGES * 2 * AT_TILE_BYTES;
-constexpr int AT_BOOK_BYTES = 2048;
+constexpr int AT_BOOK_BYTES = 3072;
 constexpr int AT_SMEM_BYTES = AT_MAIN_BYTES + AT_BOOK_BYTES;
-constexpr uint32_t AT_TMEM_COLS = 512;          // S (two buffers of 128 columns) and O_tile (128 columns)
+constexpr uint32_t AT_TMEM_COLS = 512;          // per row tile: S / P (128 columns) and O (128 columns)
 constexpr long long AT_WAIT_LIMIT = 2000000000LL;
+constexpr float AT_RESCALE_STEP = 8.0f;         // log2 units the row maximum may outgrow the reference
 static_assert(AT_SMEM_BYTES <= 195 * 1024, "the attention block must stay inside the 196 KB carve-out");
 
 struct AttnArgs {
@@ -82,37 +86,43 @@ struct AttnArgs {
 };
 
 struct AttnBook {
-  uint64_t full[AT_STAGES], empty[AT_STAGES], q_full, s_full[2], s_free[2], p_ready, pv_done, o_free;
+  uint64_t full[AT_STAGES], empty[AT_STAGES], q_full, s_full[2], p_ready[2], pv_done[2];
   uint32_t tmem_base;
   int abort_flag;
-  float m_tile[2][128];
+  float m_tile[2][2][128];     // [row tile][key tile parity][key]
 };
 static_assert(sizeof(AttnBook) <= AT_BOOK_BYTES, "attention kernel bookkeeping exceeds its shared-memory slot");
+
+// keys a tile of query rows [q_lo, q_lo + 128) can see: up to its last row (causal), and to the end
+// of the image span if one of its rows lies inside the span and the mask is on
+__device__ __forceinline__ int attn_key_end(const SampleDesc &d, int q_lo, int mask_enable, bool &sees_span) {
+  const int q_hi = min(q_lo + 128, d.n);
+  sees_span = mask_enable && q_lo < d.v0 + d.nv && q_hi > d.v0;
+  return min(d.n, sees_span ? max(q_hi, d.v0 + d.nv) : q_hi);
+}
 
 __global__ void __launch_bounds__(AT_THREADS, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
             const __grid_constant__ CUtensorMap tmap_vt, AttnArgs a) {
   pdl_enter();
   extern __shared__ __align__(1024) uint8_t at_smem[];
-  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;     // long rows first
+  const int pair = (int)gridDim.x - 1 - (int)blockIdx.x;     // long rows first
   const int h = blockIdx.y, b = blockIdx.z;
   const SampleDesc d = a.desc[b];
-  const int q_lo = qt * 128;
-  if (!d.valid || q_lo >= d.n) return;
+  const int q_base = pair * 256;
+  if (!d.valid || q_base >= d.n) return;
   if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_ATTN_TIMEOUT) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t base = smem_u32(at_smem);
-  const uint32_t q_smem = base, p_smem = base + AT_TILE_BYTES, ring = base + 2 * AT_TILE_BYTES;
+  const uint32_t q_smem = base, ring = base + 2 * AT_TILE_BYTES;
   AttnBook *bk = reinterpret_cast<AttnBook *>(at_smem + AT_MAIN_BYTES);
 
-  // keys this row tile can see: up to its last row (causal), and to the end of the image span
-  // if one of its rows lies inside the span and the mask is on
-  const int q_hi = min(q_lo + 128, d.n);
-  const bool sees_span = a.mask_enable && q_lo < d.v0 + d.nv && q_hi > d.v0;
-  const int j_end = min(d.n, sees_span ? max(q_hi, d.v0 + d.nv) : q_hi);
   const int delta = d.row0 & 7;
   const int kbase = d.row0 - delta;
-  const int n_kt = (j_end + delta + 127) / 128;
+  bool sees0 = false, sees1 = false;
+  const int n_kt0 = (attn_key_end(d, q_base, a.mask_enable, sees0) + delta + 127) / 128;
+  const int n_kt1 = q_base + 128 < d.n ? (attn_key_end(d, q_base + 128, a.mask_enable, sees1) + delta + 127) / 128 : 0;
+  const int n_max = max(n_kt0, n_kt1);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < AT_STAGES; ++s) {
@@ -120,13 +130,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
       mbar_init(smem_u32(&bk->empty[s]), 1);
     }
     mbar_init(smem_u32(&bk->q_full), 1);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&bk->s_full[i]), 1);
-      mbar_init(smem_u32(&bk->s_free[i]), 128);
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(smem_u32(&bk->s_full[g]), 1);
+      mbar_init(smem_u32(&bk->p_ready[g]), 128);
+      mbar_init(smem_u32(&bk->pv_done[g]), 1);
     }
-    mbar_init(smem_u32(&bk->p_ready), 128);
-    mbar_init(smem_u32(&bk->pv_done), 1);
-    mbar_init(smem_u32(&bk->o_free), 128);
     bk->abort_flag = 0;
     fence_barrier_init();
   }
@@ -145,11 +153,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
       tma_prefetch_desc(&tmap_q);
       tma_prefetch_desc(&tmap_k);
       tma_prefetch_desc(&tmap_vt);
-      mbar_expect_tx(smem_u32(&bk->q_full), AT_TILE_BYTES);
-      tma_load_2d(q_smem, &tmap_q, smem_u32(&bk->q_full), h * 128, d.row0 + q_lo);
-      tma_load_2d(q_smem + AT_BLOCK_BYTES, &tmap_q, smem_u32(&bk->q_full), h * 128 + 64, d.row0 + q_lo);
+      const int n_q = n_kt1 > 0 ? 2 : 1;
+      mbar_expect_tx(smem_u32(&bk->q_full), n_q * AT_TILE_BYTES);
+      for (int g = 0; g < n_q; ++g) {
+        tma_load_2d(q_smem + g * AT_TILE_BYTES, &tmap_q, smem_u32(&bk->q_full), h * 128, d.row0 + q_base + g * 128);
+        tma_load_2d(q_smem + g * AT_TILE_BYTES + AT_BLOCK_BYTES, &tmap_q, smem_u32(&bk->q_full), h * 128 + 64,
+                    d.row0 + q_base + g * 128);
+      }
       int issued = 0;
-      for (int kt = 0; kt < n_kt; ++kt) {
+      for (int kt = 0; kt < n_max; ++kt) {
         const int s = kt % AT_STAGES;
         if (kt >= AT_STAGES) mbar_wait(smem_u32(&bk->empty[s]), ((kt / AT_STAGES) - 1) & 1, wc);
         if (bk->abort_flag) break;
@@ -175,172 +187,165 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_bf16(128, 128);
-      const uint32_t o_tmem = tmem_base + 256;
-      auto issue_s = [&](int kt) {
-        const int s = kt % AT_STAGES, buf = kt & 1;
+      // S of row tile g for key tile kt.  Issued after the P V of key tile kt - 1 of the same row tile,
+      // whose P it overwrites; the tensor pipe runs one thread's MMAs in issue order.
+      auto issue_s = [&](int g, int kt) {
+        const int s = kt % AT_STAGES;
         mbar_wait(smem_u32(&bk->full[s]), (kt / AT_STAGES) & 1, wc);
-        if (kt >= 2) mbar_wait(smem_u32(&bk->s_free[buf]), ((kt >> 1) - 1) & 1, wc);
         tc_fence_after();
         if (bk->abort_flag) return;
-        const uint32_t kb = ring + s * 2 * AT_TILE_BYTES;
+        const uint32_t qa = q_smem + g * AT_TILE_BYTES, kb = ring + s * 2 * AT_TILE_BYTES;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          tc_mma_bf16(tmem_base + buf * 128, umma_desc_sw128(q_smem + (kk >> 2) * AT_BLOCK_BYTES + (kk & 3) * 32),
+          tc_mma_bf16(tmem_base + g * 256, umma_desc_sw128(qa + (kk >> 2) * AT_BLOCK_BYTES + (kk & 3) * 32),
                       umma_desc_sw128(kb + (kk >> 2) * AT_BLOCK_BYTES + (kk & 3) * 32), idesc, kk > 0 ? 1u : 0u);
-        tc_commit(smem_u32(&bk->s_full[buf]));
+        tc_commit(smem_u32(&bk->s_full[g]));
       };
       mbar_wait(smem_u32(&bk->q_full), 0, wc);
-      issue_s(0);
-      for (int kt = 0; kt < n_kt; ++kt) {
-        if (kt + 1 < n_kt) issue_s(kt + 1);
+      issue_s(0, 0);
+      if (n_kt1 > 0) issue_s(1, 0);
+      for (int kt = 0; kt < n_max; ++kt) {
         const int s = kt % AT_STAGES;
-        mbar_wait(smem_u32(&bk->p_ready), kt & 1, wc);
-        if (kt >= 1) mbar_wait(smem_u32(&bk->o_free), (kt - 1) & 1, wc);
-        tc_fence_after();
-        if (!bk->abort_flag) {
-          const uint32_t vb = ring + s * 2 * AT_TILE_BYTES + AT_TILE_BYTES;
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            tc_mma_bf16(o_tmem, umma_desc_sw128(p_smem + (kk >> 2) * AT_BLOCK_BYTES + (kk & 3) * 32),
-                        umma_desc_sw128(vb + (kk >> 2) * AT_BLOCK_BYTES + (kk & 3) * 32), idesc, kk > 0 ? 1u : 0u);
-          tc_commit(smem_u32(&bk->pv_done));
-          tc_commit(smem_u32(&bk->empty[s]));
+        for (int g = 0; g < 2; ++g) {
+          const int n_g = g == 0 ? n_kt0 : n_kt1;
+          if (kt >= n_g) continue;
+          mbar_wait(smem_u32(&bk->p_ready[g]), kt & 1, wc);
+          tc_fence_after();
+          if (!bk->abort_flag) {
+            const uint32_t vb = ring + s * 2 * AT_TILE_BYTES + AT_TILE_BYTES;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)
+              tc_mma_bf16_ta(tmem_base + g * 256 + 128, tmem_base + g * 256 + kk * 8,
+                             umma_desc_sw128(vb + (kk >> 2) * AT_BLOCK_BYTES + (kk & 3) * 32), idesc,
+                             (kt > 0 || kk > 0) ? 1u : 0u);
+            tc_commit(smem_u32(&bk->pv_done[g]));
+          }
+          if (kt + 1 < n_g) issue_s(g, kt + 1);
         }
+        if (!bk->abort_flag) tc_commit(smem_u32(&bk->empty[s]));
       }
     }
   } else {
+    const int g = (warp - 2) >> 2;                // row tile of this softmax group
     const int quarter = warp & 3;                 // the TMEM lanes this warp may read
     const int lrow = quarter * 32 + lane;
+    const int q_lo = q_base + g * 128;
     const int i = q_lo + lrow;                    // sequence-relative query row
     const bool vis_row = a.mask_enable && i >= d.v0 && i < d.v0 + d.nv;
     const int hi_adm = min(d.n - 1, vis_row ? max(i, d.v0 + d.nv - 1) : i);   // last admitted key
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t s_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + g * 256;
+    const uint32_t o_addr = s_addr + 128;
     const float *mlog_b = a.mask_log ? a.mask_log + (size_t)b * a.max_vis : nullptr;
-    uint8_t *p_row = at_smem + AT_TILE_BYTES + lrow * 128;
-    const int st = threadIdx.x - 64;              // 0..127 among the softmax threads
+    const int st = (threadIdx.x - 64) & 127;      // 0..127 inside the group
+    const int my_kt = g == 0 ? n_kt0 : n_kt1;
+    const bool my_sees = g == 0 ? sees0 : sees1;
 
-    float o_acc[128];
-#pragma unroll
-    for (int c = 0; c < 128; ++c) o_acc[c] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
-
-    for (int kt = 0; kt < n_kt; ++kt) {
-      const int buf = kt & 1;
+    // Logits stay in the units the MMA produced (q.k); the scale log2(e)/sqrt(d) enters inside the
+    // exponential's multiply-add.  m_ref is the reference maximum in those units.
+    const float step_raw = AT_RESCALE_STEP / a.scale_log2;
+    const float m_to_raw = 1.4426950408889634f / a.scale_log2;
+    float m_ref = -INFINITY, l_run = 0.f;
+    for (int kt = 0; kt < my_kt; ++kt) {
       const int j0 = kt * 128 - delta;            // sequence-relative key of column 0
-      // a tile strictly below the diagonal for every row of the block needs no mask at all
+      // a tile strictly below the diagonal for every row of the row tile needs no mask at all
       const bool plain = j0 >= 0 && j0 + 127 <= q_lo && j0 + 127 < d.n;
-      const bool soft = !plain && sees_span && j0 + 127 > q_lo;    // may hold future keys of the span
+      const bool soft = !plain && my_sees && j0 + 127 > q_lo;      // may hold future keys of the span
+      const float *mt = bk->m_tile[g][kt & 1];
       if (soft) {
         const int j = j0 + st;
         float mv = 0.f;
-        if (mlog_b && j >= d.v0 && j < d.v0 + d.nv) mv = __ldg(mlog_b + (j - d.v0)) * 1.4426950408889634f;
-        bk->m_tile[buf][st] = mv;
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (mlog_b && j >= d.v0 && j < d.v0 + d.nv) mv = __ldg(mlog_b + (j - d.v0)) * m_to_raw;
+        bk->m_tile[g][kt & 1][st] = mv;
+        if (g == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
+        else asm volatile("bar.sync 2, 128;" ::: "memory");
       }
-      const float *mt = bk->m_tile[buf];
-      mbar_wait(smem_u32(&bk->s_full[buf]), (kt >> 1) & 1, wc);
+      mbar_wait(smem_u32(&bk->s_full[g]), kt & 1, wc);
       tc_fence_after();
-      const uint32_t s_addr = lane_addr + buf * 128;
-      // ---- pass 1: row maximum of the admitted logits
-      float mx = m_run;
-#pragma unroll 1
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(s_addr + c0, r);
-        tmem_wait_ld();
-        if (plain) {
+      // ---- the row's 128 logits, once: four loads in flight, one wait
+      uint32_t xr[128];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]) * a.scale_log2);
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const int j = j0 + c0 + e;
-            float x = __uint_as_float(r[e]) * a.scale_log2;
-            if (soft && j > i) x += mt[c0 + e];
-            if (j >= 0 && j <= hi_adm) mx = fmaxf(mx, x);
-          }
-        }
-      }
-      const float alpha = fast_exp2(m_run - mx);           // first tile: exp2(-inf) = 0
-      // ---- fold the previous tile's P V into the running output
-      if (kt > 0) {
-        mbar_wait(smem_u32(&bk->pv_done), (kt - 1) & 1, wc);
-        tc_fence_after();
-#pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t r[32];
-          tmem_ld32(lane_addr + 256 + c0, r);
-          tmem_wait_ld();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) o_acc[c0 + e] = fmaf(o_acc[c0 + e], alpha_prev, __uint_as_float(r[e]));
-        }
-        tc_fence_before();
-        mbar_arrive(smem_u32(&bk->o_free));
-      }
-      // ---- pass 2: probabilities relative to the new maximum, as a bf16 operand tile
-      float l_tile = 0.f;
-#pragma unroll 1
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(s_addr + c0, r);
-        tmem_wait_ld();
-        float pv[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int j = j0 + c0 + e;
-          float x = __uint_as_float(r[e]) * a.scale_log2;
-          if (!plain) {
-            if (soft && j > i) x += mt[c0 + e];
-            if (!(j >= 0 && j <= hi_adm)) x = -INFINITY;
-          }
-          pv[e] = fast_exp2(x - mx);
-        }
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {                       // four 16-byte chunks of eight keys
-          uint4 w;
-          w.x = pack2_rn(pv[8 * g + 0], pv[8 * g + 1]);
-          w.y = pack2_rn(pv[8 * g + 2], pv[8 * g + 3]);
-          w.z = pack2_rn(pv[8 * g + 4], pv[8 * g + 5]);
-          w.w = pack2_rn(pv[8 * g + 6], pv[8 * g + 7]);
-          // the row sum uses the rounded values the MMA will see
-          l_tile += (bf16_lo(w.x) + bf16_hi(w.x)) + (bf16_lo(w.y) + bf16_hi(w.y)) +
-                    (bf16_lo(w.z) + bf16_hi(w.z)) + (bf16_lo(w.w) + bf16_hi(w.w));
-          const int col = c0 + 8 * g;                       // first key of the chunk
-          const int blk = col >> 6, chunk = (col & 63) >> 3;
-          *reinterpret_cast<uint4 *>(p_row + blk * AT_BLOCK_BYTES + ((chunk ^ (lrow & 7)) << 4)) = w;
-        }
-      }
-      l_run = l_run * alpha + l_tile;
-      m_run = mx;
-      alpha_prev = alpha;
-      tc_fence_before();
-      fence_proxy_async();                                  // the MMA reads P through the async proxy
-      mbar_arrive(smem_u32(&bk->s_free[buf]));
-      mbar_arrive(smem_u32(&bk->p_ready));
-    }
-    // ---- last tile's P V, normalisation, store
-    mbar_wait(smem_u32(&bk->pv_done), (n_kt - 1) & 1, wc);
-    tc_fence_after();
-    const float inv_l = l_run > 0.f ? 1.0f / l_run : 0.f;
-    const bool store = i < d.n && !bk->abort_flag;
-    uint4 *orow = reinterpret_cast<uint4 *>(a.out + ((size_t)(d.row0 + i) * a.H + h) * 128);
-#pragma unroll
-    for (int c0 = 0; c0 < 128; c0 += 32) {
-      uint32_t r[32];
-      tmem_ld32(lane_addr + 256 + c0, r);
+      for (int c0 = 0; c0 < 128; c0 += 32) tmem_ld32p(s_addr + c0, xr + c0);
       tmem_wait_ld();
-      // the last fold needs no rescaling: O_tile is already relative to the final maximum
+      float mx = m_ref;
+      if (plain) {
 #pragma unroll
-      for (int e = 0; e < 32; ++e) o_acc[c0 + e] = fmaf(o_acc[c0 + e], alpha_prev, __uint_as_float(r[e])) * inv_l;
-      if (store) {
+        for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(xr[c]));
+      } else {
+        const int di = i - j0, lo = -j0, hi = hi_adm - j0;      // column of the diagonal, first / last admitted column
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          uint4 w;
-          w.x = pack2_rn(o_acc[c0 + 8 * g + 0], o_acc[c0 + 8 * g + 1]);
-          w.y = pack2_rn(o_acc[c0 + 8 * g + 2], o_acc[c0 + 8 * g + 3]);
-          w.z = pack2_rn(o_acc[c0 + 8 * g + 4], o_acc[c0 + 8 * g + 5]);
-          w.w = pack2_rn(o_acc[c0 + 8 * g + 6], o_acc[c0 + 8 * g + 7]);
-          orow[(c0 >> 3) + g] = w;
+        for (int c = 0; c < 128; ++c) {
+          float v = __uint_as_float(xr[c]);
+          if (soft && c > di) v += mt[c];
+          if (c < lo || c > hi) v = -INFINITY;
+          xr[c] = __float_as_uint(v);
+          mx = fmaxf(mx, v);
+        }
+      }
+      // ---- move the reference (and rescale O) only when some row of the warp outgrew it
+      if (kt == 0) {
+        m_ref = mx;
+      } else {
+        const bool need = mx > m_ref + step_raw;
+        if (__any_sync(0xffffffffu, need)) {
+          // O holds every earlier P V: the S just waited for was committed after them
+          const float f = need ? fast_exp2((m_ref - mx) * a.scale_log2) : 1.0f;
+#pragma unroll
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(o_addr + c0, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
+            tmem_st32(o_addr + c0, r);
+          }
+          l_run *= f;
+          if (need) m_ref = mx;
+        }
+      }
+      // ---- probabilities relative to the reference, stored as bf16 over S's first 64 columns
+      const float neg_ref = -m_ref * a.scale_log2;
+      float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t w[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(xr[c0 + 2 * e]), a.scale_log2, neg_ref));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(xr[c0 + 2 * e + 1]), a.scale_log2, neg_ref));
+          l0 += p0;
+          l1 += p1;
+          w[e] = pack2_rn(p0, p1);
+        }
+        tmem_st16(s_addr + (c0 >> 1), w);
+      }
+      l_run += l0 + l1;
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&bk->p_ready[g]));
+    }
+    // ---- normalisation and store
+    if (my_kt > 0) {
+      mbar_wait(smem_u32(&bk->pv_done[g]), (my_kt - 1) & 1, wc);
+      tc_fence_after();
+      const float inv_l = l_run > 0.f ? 1.0f / l_run : 0.f;
+      const bool store = i < d.n && !bk->abort_flag;
+      uint4 *orow = reinterpret_cast<uint4 *>(a.out + ((size_t)(d.row0 + i) * a.H + h) * 128);
+#pragma unroll
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(o_addr + c0, r);
+        tmem_wait_ld();
+        if (store) {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint4 w;
+            w.x = pack2_rn(__uint_as_float(r[8 * q4 + 0]) * inv_l, __uint_as_float(r[8 * q4 + 1]) * inv_l);
+            w.y = pack2_rn(__uint_as_float(r[8 * q4 + 2]) * inv_l, __uint_as_float(r[8 * q4 + 3]) * inv_l);
+            w.z = pack2_rn(__uint_as_float(r[8 * q4 + 4]) * inv_l, __uint_as_float(r[8 * q4 + 5]) * inv_l);
+            w.w = pack2_rn(__uint_as_float(r[8 * q4 + 6]) * inv_l, __uint_as_float(r[8 * q4 + 7]) * inv_l);
+            orow[(c0 >> 3) + q4] = w;
+          }
         }
       }
     }
