@@ -326,7 +326,7 @@ def run_cuda(args):
     # ---- stage 2 as Sec. 4.2 words it (routing inside the kept set, refill by attention mass), timed
     # apart from the step on the step's own stage-1 results
     cons = None
-    if args.consolidate_threshold is not None and keep_k < int(batch.vis_len.max()):
+    if args.consolidate_iters > 0 and keep_k < int(batch.vis_len.max()):
         import dataclasses
         p2 = dataclasses.replace(params, sim_threshold=args.consolidate_threshold)
         st1 = [t.clone() for t in (out.mass, out.salience, out.keep_idx, out.drop_idx)]
@@ -340,18 +340,18 @@ def run_cuda(args):
         c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         c0.record(stream)
-        for i in range(50):
+        for i in range(args.consolidate_iters):
             call(i)
         c1.record(stream)
         torch.cuda.synchronize()
         A.asap_check(ctx)
         A.asap_profile(ctx, True)
-        for i in range(50):
+        for i in range(args.consolidate_iters):
             call(i)
         torch.cuda.synchronize()
         ck = {name: ms / max(n, 1) * 1e3 for name, (n, ms) in A.asap_profile_read(ctx).items()}
         A.asap_profile(ctx, False)
-        cons = {"threshold": args.consolidate_threshold, "us": c0.elapsed_time(c1) / 50 * 1e3,
+        cons = {"threshold": args.consolidate_threshold, "us": c0.elapsed_time(c1) / args.consolidate_iters * 1e3,
                 "absorbed_per_sequence": float(n_abs.float().mean()), "kernel_us": ck}
         del scratch, out2
 
@@ -506,6 +506,7 @@ def main():
                     help="also time KV-cache compaction of this many layers (0 = skip)")
     ap.add_argument("--consolidate-threshold", type=float, default=0.8,
                     help="also time asap_consolidate (Sec. 4.2 inside the kept set) with this threshold t")
+    ap.add_argument("--consolidate-iters", type=int, default=50, help="timed asap_consolidate calls (0 = skip)")
     ap.add_argument("--attention-iters", type=int, default=10,
                     help="also time asap_attention (the layer's attention under the SG-BiMask) this many times (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -637,6 +637,67 @@ __device__ __forceinline__ void csr_block(const SampleDesc &d, int b, int max_vi
 constexpr int ROUTE_THREADS = 1024;
 constexpr int ROUTE_LANE_WORDS = 4;                     // keep_k <= 32 * 32 * 4
 
+// The sequential part of the routing, run by one warp, 32 candidates of the visiting order at a
+// time.  Lane l holds words l, l + 32, ... of the union of the anchors' rows (LW words per lane;
+// LW = 1 covers keep_k <= 1024).  Per group of 32: (1) each lane looks up whether its candidate is
+// already covered by an anchor of an earlier group; (2) each lane gathers its candidate's row
+// restricted to the group (32 bits); (3) the group is resolved in order from those 32 x 32 bits, in
+// registers, by every lane alike; (4) the group's anchors add their full rows to the union.  Only
+// step (3) is a dependent chain, and it touches no memory.  Returns the number of absorbed slots.
+template <int LW>
+__device__ __forceinline__ int route_walk(const int *s_order, const uint32_t *mask, int *s_flag, int k, int kw,
+                                          int nd, int lane) {
+  const unsigned full = 0xffffffffu;
+  uint32_t supp[LW];
+#pragma unroll
+  for (int i = 0; i < LW; ++i) supp[i] = 0u;
+  int n_abs = 0;
+  for (int r0 = 0; r0 < k; r0 += 32) {
+    const bool valid = r0 + lane < k;
+    const int p = valid ? s_order[r0 + lane] : 0;
+    const int w = p >> 5;
+    uint32_t word = 0u;
+#pragma unroll
+    for (int i = 0; i < LW; ++i) {
+      const uint32_t got = __shfl_sync(full, supp[i], w & 31);
+      if ((w >> 5) == i) word = got;
+    }
+    uint32_t blk = __ballot_sync(full, valid && ((word >> (p & 31)) & 1u));
+    uint32_t intra = 0u;
+#pragma unroll
+    for (int u = 0; u < 32; ++u) {
+      const int pu = __shfl_sync(full, p, u);
+      const uint32_t bit = (mask[(size_t)p * kw + (pu >> 5)] >> (pu & 31)) & 1u;
+      if (valid && r0 + u < k) intra |= bit << u;
+    }
+    uint32_t absorbed_bits = 0u;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+      const uint32_t row_t = __shfl_sync(full, intra, t);
+      const bool ab = ((blk >> t) & 1u) && n_abs < nd && r0 + t < k;
+      if (ab) {
+        ++n_abs;
+        absorbed_bits |= 1u << t;
+      } else {
+        blk |= row_t & ~((2u << t) - 1u);          // an anchor covers later candidates only
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+      const int pt = __shfl_sync(full, p, t);
+      if (r0 + t < k && !((absorbed_bits >> t) & 1u)) {
+#pragma unroll
+        for (int i = 0; i < LW; ++i) {
+          const int ww = i * 32 + lane;
+          if (ww < kw) supp[i] |= mask[(size_t)pt * kw + ww];
+        }
+      }
+    }
+    if (valid) s_flag[p] = ((absorbed_bits >> lane) & 1u) ? 0 : 1;
+  }
+  return n_abs;
+}
+
 struct RouteArgs {
   const SampleDesc *desc;
   int max_vis, keep_k, kw;        // kw = ceil(keep_k / 32)
@@ -718,31 +779,9 @@ route_kernel(RouteArgs a) {
   __syncthreads();
   // ---- C: greedy walk by one warp; the union lives in registers, word w in lane w % 32
   if (warp == 0) {
-    uint32_t supp[ROUTE_LANE_WORDS];
-#pragma unroll
-    for (int i = 0; i < ROUTE_LANE_WORDS; ++i) supp[i] = 0u;
-    int n_abs = 0;
-    for (int r = 0; r < k; ++r) {
-      const int p = s_order[r];
-      const int w = p >> 5;
-      uint32_t word = 0u;
-#pragma unroll
-      for (int i = 0; i < ROUTE_LANE_WORDS; ++i)
-        if ((w >> 5) == i) word = supp[i];
-      word = __shfl_sync(0xffffffffu, word, w & 31);
-      const bool absorbed = ((word >> (p & 31)) & 1u) && n_abs < nd;
-      if (absorbed) {
-        ++n_abs;
-      } else {
-#pragma unroll
-        for (int i = 0; i < ROUTE_LANE_WORDS; ++i) {
-          const int ww = i * 32 + lane;
-          if (ww < kw) supp[i] |= mask[(size_t)p * kw + ww];
-        }
-      }
-      if (lane == 0) s_flag[p] = absorbed ? 0 : 1;
-    }
-    if (lane == 0) s_nabs = n_abs;
+    const int n_abs_w = kw <= 32 ? route_walk<1>(s_order, mask, s_flag, k, kw, nd, lane)
+                                 : route_walk<ROUTE_LANE_WORDS>(s_order, mask, s_flag, k, kw, nd, lane);
+    if (lane == 0) s_nabs = n_abs_w;
   }
   __syncthreads();
   const int n_abs = s_nabs;
