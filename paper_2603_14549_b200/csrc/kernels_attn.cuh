@@ -6,7 +6,8 @@
 //   attn_kernel         one block per (two tiles of 128 query rows, head, sequence); the two row
 //                       tiles share every key / value tile and take turns on the tensor pipe.
 //                       For every tile of 128 keys:  S = Q K^T on tcgen05 into tensor memory; the
-//                       row tile's four softmax warps read S once (one thread per row), add Eq. 3's
+//                       row tile's eight softmax warps read S once (two threads per row, 64 keys
+//                       each, exchanging their maxima through shared memory), add Eq. 3's
 //                       m_j for the future keys of the image span on rows of the image span (nothing
 //                       else above the diagonal is admitted), turn the logits into probabilities
 //                       relative to a reference maximum and store them as bf16 over S's own columns;
@@ -64,7 +65,7 @@ transpose_v_kernel(const __nv_bfloat16 *__restrict__ v, __nv_bfloat16 *__restric
 }
 
 // ---------------------------------------------------------------------------------------
-constexpr int AT_THREADS = 320;                 // warp 0: copies, warp 1: MMA issue, warps 2-9: two softmax groups
+constexpr int AT_THREADS = 576;                 // warp 0: copies, warp 1: MMA issue, warps 2-17: two softmax groups of eight
 constexpr int AT_TILE_BYTES = 128 * 128 * 2;    // 128 rows x 128 bf16 as two 64-column blocks of 16 KB
 constexpr int AT_BLOCK_BYTES = AT_TILE_BYTES / 2;
 constexpr int AT_STAGES = 2;                    // a stage = one key tile + one value tile
@@ -89,9 +90,19 @@ struct AttnBook {
   uint64_t full[AT_STAGES], empty[AT_STAGES], q_full, s_full[2], p_ready[2], pv_done[2];
   uint32_t tmem_base;
   int abort_flag;
-  float m_tile[2][2][128];     // [row tile][key tile parity][key]
+  float m_tile[2][128];        // [row tile][key]: Eq. 3's addend for the keys of the current tile
+  uint32_t row_max[2][128];    // [row tile][row]: running row maximum as an order-preserving integer
 };
 static_assert(sizeof(AttnBook) <= AT_BOOK_BYTES, "attention kernel bookkeeping exceeds its shared-memory slot");
+
+// order-preserving integer image of a float (no NaN here) and its inverse, for atomicMax
+__device__ __forceinline__ uint32_t attn_key(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float attn_unkey(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 
 // keys a tile of query rows [q_lo, q_lo + 128) can see: up to its last row (causal), and to the end
 // of the image span if one of its rows lies inside the span and the mask is on
@@ -132,12 +143,35 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
     mbar_init(smem_u32(&bk->q_full), 1);
     for (int g = 0; g < 2; ++g) {
       mbar_init(smem_u32(&bk->s_full[g]), 1);
-      mbar_init(smem_u32(&bk->p_ready[g]), 128);
+      mbar_init(smem_u32(&bk->p_ready[g]), 256);
       mbar_init(smem_u32(&bk->pv_done[g]), 1);
     }
     bk->abort_flag = 0;
     fence_barrier_init();
+    // the query tiles and the first key / value tiles are requested right away, while the other
+    // warps are still setting up (this thread is the copy thread)
+    tma_prefetch_desc(&tmap_q);
+    tma_prefetch_desc(&tmap_k);
+    tma_prefetch_desc(&tmap_vt);
+    const int n_q = n_kt1 > 0 ? 2 : 1;
+    mbar_expect_tx(smem_u32(&bk->q_full), n_q * AT_TILE_BYTES);
+    for (int g = 0; g < n_q; ++g) {
+      tma_load_2d(q_smem + g * AT_TILE_BYTES, &tmap_q, smem_u32(&bk->q_full), h * 128, d.row0 + q_base + g * 128);
+      tma_load_2d(q_smem + g * AT_TILE_BYTES + AT_BLOCK_BYTES, &tmap_q, smem_u32(&bk->q_full), h * 128 + 64,
+                  d.row0 + q_base + g * 128);
+    }
+    for (int kt = 0; kt < min(n_max, AT_STAGES); ++kt) {
+      const uint32_t dst = ring + kt * 2 * AT_TILE_BYTES;
+      const uint32_t bar = smem_u32(&bk->full[kt]);
+      const int key0 = kbase + kt * 128;
+      mbar_expect_tx(bar, 2 * AT_TILE_BYTES);
+      tma_load_2d(dst, &tmap_k, bar, h * 128, key0);
+      tma_load_2d(dst + AT_BLOCK_BYTES, &tmap_k, bar, h * 128 + 64, key0);
+      tma_load_2d(dst + AT_TILE_BYTES, &tmap_vt, bar, key0, h * 128);
+      tma_load_2d(dst + AT_TILE_BYTES + AT_BLOCK_BYTES, &tmap_vt, bar, key0 + 64, h * 128);
+    }
   }
+  if (threadIdx.x < 256) (&bk->row_max[0][0])[threadIdx.x] = 0u;      // below every encoded float
   if (warp == 1) {
     tmem_alloc(smem_u32(&bk->tmem_base), AT_TMEM_COLS);
     tmem_relinquish();
@@ -150,18 +184,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
 
   if (warp == 0) {
     if (lane == 0) {
-      tma_prefetch_desc(&tmap_q);
-      tma_prefetch_desc(&tmap_k);
-      tma_prefetch_desc(&tmap_vt);
-      const int n_q = n_kt1 > 0 ? 2 : 1;
-      mbar_expect_tx(smem_u32(&bk->q_full), n_q * AT_TILE_BYTES);
-      for (int g = 0; g < n_q; ++g) {
-        tma_load_2d(q_smem + g * AT_TILE_BYTES, &tmap_q, smem_u32(&bk->q_full), h * 128, d.row0 + q_base + g * 128);
-        tma_load_2d(q_smem + g * AT_TILE_BYTES + AT_BLOCK_BYTES, &tmap_q, smem_u32(&bk->q_full), h * 128 + 64,
-                    d.row0 + q_base + g * 128);
-      }
-      int issued = 0;
-      for (int kt = 0; kt < n_max; ++kt) {
+      int issued = min(n_max, AT_STAGES);          // the first tiles were requested during set-up
+      for (int kt = issued; kt < n_max; ++kt) {
         const int s = kt % AT_STAGES;
         if (kt >= AT_STAGES) mbar_wait(smem_u32(&bk->empty[s]), ((kt / AT_STAGES) - 1) & 1, wc);
         if (bk->abort_flag) break;
@@ -227,19 +251,27 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
       }
     }
   } else {
-    const int g = (warp - 2) >> 2;                // row tile of this softmax group
+    // Two threads per query row: warps w and w + 4 of a group own the same 32 rows (tensor-memory
+    // lanes) and one half of the tile's 128 key columns each.
+    const int sw = warp - 2;
+    const int g = sw >> 3;                        // row tile of this softmax group
+    const int hf = (sw >> 2) & 1;                 // column half
     const int quarter = warp & 3;                 // the TMEM lanes this warp may read
     const int lrow = quarter * 32 + lane;
     const int q_lo = q_base + g * 128;
     const int i = q_lo + lrow;                    // sequence-relative query row
     const bool vis_row = a.mask_enable && i >= d.v0 && i < d.v0 + d.nv;
     const int hi_adm = min(d.n - 1, vis_row ? max(i, d.v0 + d.nv - 1) : i);   // last admitted key
-    const uint32_t s_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + g * 256;
-    const uint32_t o_addr = s_addr + 128;
+    const uint32_t s_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + g * 256;
+    const uint32_t s_addr = s_row + hf * 64;      // this thread's 64 logits
+    const uint32_t p_addr = s_row + hf * 32;      // its 64 probabilities, packed in 32 columns
+    const uint32_t o_addr = s_row + 128 + hf * 64;   // its 64 columns of O
     const float *mlog_b = a.mask_log ? a.mask_log + (size_t)b * a.max_vis : nullptr;
-    const int st = (threadIdx.x - 64) & 127;      // 0..127 inside the group
+    const int st = (threadIdx.x - 64) & 255;      // 0..255 inside the group
     const int my_kt = g == 0 ? n_kt0 : n_kt1;
     const bool my_sees = g == 0 ? sees0 : sees1;
+    const int pair_bar = 1 + g * 4 + quarter;     // named barrier of the two warps that share these rows
+    const int group_bar = 9 + g;
 
     // Logits stay in the units the MMA produced (q.k); the scale log2(e)/sqrt(d) enters inside the
     // exponential's multiply-add.  m_ref is the reference maximum in those units.
@@ -251,30 +283,34 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
       // a tile strictly below the diagonal for every row of the row tile needs no mask at all
       const bool plain = j0 >= 0 && j0 + 127 <= q_lo && j0 + 127 < d.n;
       const bool soft = !plain && my_sees && j0 + 127 > q_lo;      // may hold future keys of the span
-      const float *mt = bk->m_tile[g][kt & 1];
-      if (soft) {
+      const float *mt = bk->m_tile[g] + hf * 64;
+      float mv = 0.f;
+      if (soft && st < 128) {
         const int j = j0 + st;
-        float mv = 0.f;
         if (mlog_b && j >= d.v0 && j < d.v0 + d.nv) mv = __ldg(mlog_b + (j - d.v0)) * m_to_raw;
-        bk->m_tile[g][kt & 1][st] = mv;
-        if (g == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
-        else asm volatile("bar.sync 2, 128;" ::: "memory");
       }
       mbar_wait(smem_u32(&bk->s_full[g]), kt & 1, wc);
       tc_fence_after();
-      // ---- the row's 128 logits, once: four loads in flight, one wait
-      uint32_t xr[128];
-#pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) tmem_ld32p(s_addr + c0, xr + c0);
+      if (soft) {
+        // every thread of the group has finished the previous tile (its arrival was needed for
+        // the S just waited for), so the addends can be replaced
+        if (st < 128) bk->m_tile[g][st] = mv;
+        asm volatile("bar.sync %0, 256;" ::"r"(group_bar) : "memory");
+      }
+      // ---- this thread's 64 logits, once
+      uint32_t xr[64];
+      tmem_ld32p(s_addr, xr);
+      tmem_ld32p(s_addr + 32, xr + 32);
       tmem_wait_ld();
-      float mx = m_ref;
+      float mx = -INFINITY;
       if (plain) {
 #pragma unroll
-        for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(xr[c]));
+        for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(xr[c]));
       } else {
-        const int di = i - j0, lo = -j0, hi = hi_adm - j0;      // column of the diagonal, first / last admitted column
+        // columns relative to this half: the diagonal, the first and the last admitted column
+        const int di = i - j0 - hf * 64, lo = -j0 - hf * 64, hi = hi_adm - j0 - hf * 64;
 #pragma unroll
-        for (int c = 0; c < 128; ++c) {
+        for (int c = 0; c < 64; ++c) {
           float v = __uint_as_float(xr[c]);
           if (soft && c > di) v += mt[c];
           if (c < lo || c > hi) v = -INFINITY;
@@ -282,6 +318,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
           mx = fmaxf(mx, v);
         }
       }
+      // ---- the running row maximum over both halves and all tiles so far.  (The partner has read
+      // its logits by the time it passes this barrier, so the probabilities may overwrite them.)
+      atomicMax(&bk->row_max[g][lrow], attn_key(mx));
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+      mx = attn_unkey(bk->row_max[g][lrow]);
       // ---- move the reference (and rescale O) only when some row of the warp outgrew it
       if (kt == 0) {
         m_ref = mx;
@@ -291,13 +332,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
           // O holds every earlier P V: the S just waited for was committed after them
           const float f = need ? fast_exp2((m_ref - mx) * a.scale_log2) : 1.0f;
 #pragma unroll
-          for (int c0 = 0; c0 < 128; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld32(o_addr + c0, r);
+          for (int c0 = 0; c0 < 64; c0 += 16) {
+            uint32_t r[16];
+            tmem_ld16(o_addr + c0, r);
             tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
-            tmem_st32(o_addr + c0, r);
+            for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
+            tmem_st16(o_addr + c0, r);
           }
           l_run *= f;
           if (need) m_ref = mx;
@@ -307,7 +348,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
       const float neg_ref = -m_ref * a.scale_log2;
       float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
+      for (int c0 = 0; c0 < 64; c0 += 32) {
         uint32_t w[16];
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
@@ -317,22 +358,32 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
           l1 += p1;
           w[e] = pack2_rn(p0, p1);
         }
-        tmem_st16(s_addr + (c0 >> 1), w);
+        tmem_st16(p_addr + (c0 >> 1), w);
       }
       l_run += l0 + l1;
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(smem_u32(&bk->p_ready[g]));
     }
-    // ---- normalisation and store
+    // ---- normalisation and store: the two halves of a row add their sums first
     if (my_kt > 0) {
+      // the row's slot of maxima is free once both threads have read the last one
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+      if (hf == 0) bk->row_max[g][lrow] = __float_as_uint(l_run);
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+      if (hf == 1) {
+        l_run += __uint_as_float(bk->row_max[g][lrow]);
+        bk->row_max[g][lrow] = __float_as_uint(l_run);
+      }
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+      if (hf == 0) l_run = __uint_as_float(bk->row_max[g][lrow]);
       mbar_wait(smem_u32(&bk->pv_done[g]), (my_kt - 1) & 1, wc);
       tc_fence_after();
       const float inv_l = l_run > 0.f ? 1.0f / l_run : 0.f;
       const bool store = i < d.n && !bk->abort_flag;
-      uint4 *orow = reinterpret_cast<uint4 *>(a.out + ((size_t)(d.row0 + i) * a.H + h) * 128);
+      uint4 *orow = reinterpret_cast<uint4 *>(a.out + ((size_t)(d.row0 + i) * a.H + h) * 128 + hf * 64);
 #pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
+      for (int c0 = 0; c0 < 64; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(o_addr + c0, r);
         tmem_wait_ld();
