@@ -1,6 +1,6 @@
 """Benchmark of the ASAP prune step on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1..c5] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1..c6] [--impl reference]
 
 A step is one pass of the whole prune step (attention mass, salience, mask, masked ranking
 scores, top-k, cosine assignment, weighted merge, compaction) over one synthetic batch.  The
@@ -49,6 +49,7 @@ WORKLOADS = {
     "c3": "LLaVA-NeXT-7B batch 8: 35 system + 2304 visual + 64 text, D=4096, 32x128 heads, keep 320",
     "c4": "LLaVA-NeXT AnyRes batch 64: 35 system + 2880 visual + text U[32,256], D=4096, 32x128 heads, keep 576",
     "c5": "13B-shaped batch 32, first step of 2304->1152: 35 system + 2304 visual + 128 text, D=5120, 40x128 heads",
+    "c6": "InternVL-2.5-8B-shaped batch 8: 35 system + 1536 visual (6 tiles of 256) + 64 text, D=4096, 32x128 heads, keep 510",
 }
 
 

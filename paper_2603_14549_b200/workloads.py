@@ -152,11 +152,11 @@ def _ragged(B: int, lo: int, hi: int, seed: int) -> List[int]:
 
 def config(name: str, B: Optional[int] = None, seed: Optional[int] = None,
            keep_k: Optional[int] = None) -> Batch:
-    """The five benchmark shapes.  `B` may be lowered (never raised) to draw a prefix
+    """The benchmark shapes (c1-c5: LLaVA-1.5 / LLaVA-NeXT; c6: InternVL-2.5-shaped).  `B` may be lowered (never raised) to draw a prefix
     of the batch: sample b is identical whatever B is, because each sample has its own
     generator and the ragged text lengths are drawn for the full batch first."""
     name = name.lower()
-    idx = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4}[name]
+    idx = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "c6": 5}[name]
     seed = BASE_SEED + idx if seed is None else seed
     if name == "c1":      # LLaVA-1.5-7B single step
         fullB, nv, H, k = 1, 576, 32, 192
@@ -173,6 +173,9 @@ def config(name: str, B: Optional[int] = None, seed: Optional[int] = None,
     elif name == "c4":    # LLaVA-NeXT AnyRes max resolution, 5 tiles
         fullB, nv, H, k = 64, 2880, 32, 576
         texts, cents, tile, out = _ragged(fullB, 32, 256, seed), [64] * fullB, None, 0.0
+    elif name == "c6":    # InternVL-2.5-8B-shaped: six 448 x 448 tiles of 256 tokens, budget ~510 (Sec. 5.4)
+        fullB, nv, H, k = 8, 1536, 32, 510
+        texts, cents, tile, out = [64] * fullB, [32] * fullB, 256, 0.0
     else:                 # c5: 13B-shaped, progressive
         fullB, nv, H, k = 32, 2304, 40, 1152
         texts, cents, tile, out = [128] * fullB, [48] * fullB, 576, 0.0

@@ -16,6 +16,12 @@ def test_printed_flops_are_reproduced(row):
     assert abs(got - row["tflops"]) < 1e-3, (got, row)
 
 
+@pytest.mark.parametrize("row", GOLD["other_backbones"], ids=lambda r: f"{r['tokens']} tokens, m={r['m']}")
+def test_printed_flops_of_the_other_backbone(row):
+    got = row["layers"] * F.layer_flops(row["tokens"], row["d"], row["m"]) / 1e12
+    assert abs(got - row["tflops"]) < 1e-3, (got, row)
+
+
 def test_schedule_and_ratio():
     d, m, L = GOLD["d"], GOLD["m"], GOLD["layers"]
     full = F.schedule_flops([(L, 576)], d, m)

@@ -159,6 +159,17 @@ def test_c3_full_size_sampled(big_ctx, k):
     print("c3 full parity maxima", stats)
 
 
+@pytest.mark.parametrize("k", [510, 340])
+def test_c6_internvl_shape_full_size_sampled(big_ctx, k):
+    """InternVL-2.5-8B-shaped batch (1536 visual tokens in six tiles of 256) at the two budgets of
+    Sec. 5.4 (~510 and ~340 tokens); neither is a multiple of 16, so the similarity kernel's kept-slot
+    tiles are ragged.  The oracle checks two sequences."""
+    stats = {}
+    batch = W.config("c6", keep_k=k)
+    run_step(big_ctx, batch, A.Params(keep_k=k), samples=[0, 7], stats=stats)
+    print("c6 full parity maxima", stats)
+
+
 def test_c4_full_size_sampled(big_ctx):
     """The AnyRes throughput shape at full size (64 sequences, 2880 visual tokens, ragged text up
     to 256 rows = two ranking-row tiles); the oracle checks the first and the last sequence."""
