@@ -90,7 +90,7 @@ struct AttnBook {
   uint64_t full[AT_STAGES], empty[AT_STAGES], q_full, s_full[2], p_ready[2], pv_done[2];
   uint32_t tmem_base;
   int abort_flag;
-  float m_tile[2][128];        // [row tile][key]: Eq. 3's addend for the keys of the current tile
+  alignas(16) float m_tile[2][128];   // [row tile][key]: Eq. 3's addend for the keys of the current tile
   uint32_t row_max[2][128];    // [row tile][row]: running row maximum as an order-preserving integer
 };
 static_assert(sizeof(AttnBook) <= AT_BOOK_BYTES, "attention kernel bookkeeping exceeds its shared-memory slot");
@@ -284,7 +284,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
       const bool plain = j0 >= 0 && j0 + 127 <= q_lo && j0 + 127 < d.n;
       const bool soft = !plain && my_sees && j0 + 127 > q_lo;      // may hold future keys of the span
       const float *mt = bk->m_tile[g] + hf * 64;
-      float mv = 0.f;
+      // addend of key j for a query row of the span that lies before it: m_j inside the
+      // span, -infinity outside (such a key is never admitted above the diagonal)
+      float mv = -INFINITY;
       if (soft && st < 128) {
         const int j = j0 + st;
         if (mlog_b && j >= d.v0 && j < d.v0 + d.nv) mv = __ldg(mlog_b + (j - d.v0)) * m_to_raw;
@@ -302,22 +304,54 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
       tmem_ld32p(s_addr, xr);
       tmem_ld32p(s_addr + 32, xr + 32);
       tmem_wait_ld();
-      float mx = -INFINITY;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};     // four independent chains
       if (plain) {
 #pragma unroll
-        for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(xr[c]));
+        for (int c = 0; c < 64; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(xr[c]));
       } else {
         // columns relative to this half: the diagonal, the first and the last admitted column
         const int di = i - j0 - hf * 64, lo = -j0 - hf * 64, hi = hi_adm - j0 - hf * 64;
+        if (soft && j0 > q_lo + 127) {
+          // the whole tile lies above the diagonal of every row of the row tile: a row of the span
+          // admits exactly the keys of the span (finite addend), any other row admits nothing.  Two
+          // additions per logit on the FMA pipe instead of compares and selects on the half-rate one.
+          const float rowoff = vis_row ? 0.f : -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          float v = __uint_as_float(xr[c]);
-          if (soft && c > di) v += mt[c];
-          if (c < lo || c > hi) v = -INFINITY;
-          xr[c] = __float_as_uint(v);
-          mx = fmaxf(mx, v);
+          for (int c4 = 0; c4 < 64; c4 += 4) {
+            const float4 m4 = *reinterpret_cast<const float4 *>(mt + c4);
+            const float add[4] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float v = __uint_as_float(xr[c4 + e]) + (add[e] + rowoff);
+              xr[c4 + e] = __float_as_uint(v);
+              mx4[e] = fmaxf(mx4[e], v);
+            }
+          }
+        } else if (soft) {
+          // the addends are loaded unconditionally (four per load) and selected, so the loop has no branch
+#pragma unroll
+          for (int c4 = 0; c4 < 64; c4 += 4) {
+            const float4 m4 = *reinterpret_cast<const float4 *>(mt + c4);
+            const float add[4] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int c = c4 + e;
+              float v = __uint_as_float(xr[c]) + (c > di ? add[e] : 0.f);
+              v = (c < lo || c > hi) ? -INFINITY : v;
+              xr[c] = __float_as_uint(v);
+              mx4[e] = fmaxf(mx4[e], v);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 64; ++c) {
+            const float v = (c < lo || c > hi) ? -INFINITY : __uint_as_float(xr[c]);
+            xr[c] = __float_as_uint(v);
+            mx4[c & 3] = fmaxf(mx4[c & 3], v);
+          }
         }
       }
+      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       // ---- the running row maximum over both halves and all tiles so far.  (The partner has read
       // its logits by the time it passes this barrier, so the probabilities may overwrite them.)
       atomicMax(&bk->row_max[g][lrow], attn_key(mx));
