@@ -769,11 +769,19 @@ route_kernel(RouteArgs a) {
   // ---- B: bit matrix, one warp per row, coalesced
   for (int p = warp; p < k; p += (nthr >> 5)) {
     const float *row = S + (size_t)p * k;
-    for (int w = 0; w < kw; ++w) {
-      const int q = w * 32 + lane;
-      const bool hit = q < k && q != p && __ldcg(row + q) > a.threshold;
-      const unsigned bits = __ballot_sync(0xffffffffu, hit);
-      if (lane == 0) mask[(size_t)p * kw + w] = bits;
+    for (int w0 = 0; w0 < kw; w0 += 16) {             // sixteen loads in flight per lane
+      float v[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const int q = (w0 + e) * 32 + lane;
+        v[e] = q < k ? __ldcg(row + q) : -INFINITY;
+      }
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const int q = (w0 + e) * 32 + lane;
+        const unsigned bits = __ballot_sync(0xffffffffu, q < k && q != p && v[e] > a.threshold);
+        if (lane == 0 && w0 + e < kw) mask[(size_t)p * kw + w0 + e] = bits;
+      }
     }
   }
   __syncthreads();
@@ -792,11 +800,16 @@ route_kernel(RouteArgs a) {
     const int rp = s_rank[p];
     float best = -INFINITY;
     int best_q = 0x7fffffff;
-    for (int q = lane; q < k; q += 32) {
-      if (s_flag[q] && s_rank[q] < rp) {
-        const float v = __ldcg(row + q);
-        if (v > best) { best = v; best_q = q; }       // ascending q: the first maximum stays
+    for (int q0 = lane; q0 < k; q0 += 32 * 8) {       // eight loads in flight per lane
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int q = q0 + 32 * e;
+        v[e] = (q < k && s_flag[q] && s_rank[q] < rp) ? __ldcg(row + q) : -INFINITY;
       }
+#pragma unroll
+      for (int e = 0; e < 8; ++e)                     // ascending q: the first maximum stays
+        if (v[e] > best) { best = v[e]; best_q = q0 + 32 * e; }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -920,13 +933,14 @@ route_kernel(RouteArgs a) {
   }
   if (tid == 0 && a.n_absorbed) a.n_absorbed[b] = n_abs;
   __syncthreads();
-  // grouping by destination, stable: thread t owns final slots t, t + blockDim, ...
+  // grouping by destination (counting sort, stable in source order)
   {
     int *s_cnt = s_order;                     // reuse: the visiting order is no longer needed
-    for (int sl = tid; sl < k; sl += nthr) {
-      int c = 0;
-      for (int i = 0; i < n_abs; ++i) c += ((int)s_key[i] == sl);
-      s_cnt[sl] = c;
+    for (int sl = tid; sl < k; sl += nthr) s_cnt[sl] = 0;
+    __syncthreads();
+    for (int i = tid; i < n_abs; i += nthr) {
+      const int sl = (int)s_key[i];
+      if (sl >= 0 && sl < k) atomicAdd(&s_cnt[sl], 1);
     }
     __syncthreads();
     const int per = (k + nthr - 1) / nthr;
@@ -943,10 +957,23 @@ route_kernel(RouteArgs a) {
     }
     if (tid == 0) seg_b[k] = tot;
     __syncthreads();
-    for (int sl = tid; sl < k; sl += nthr) {
-      int at = s_cnt[sl];
-      for (int i = 0; i < n_abs; ++i)
-        if ((int)s_key[i] == sl) mem_b[at++] = i;
+    // one warp walks the sources 32 at a time in ascending order, so members stay ascending inside a slot
+    if (warp == 0) {
+      for (int base = 0; base < n_abs; base += 32) {
+        const int i = base + lane;
+        int sl = i < n_abs ? (int)s_key[i] : -1;
+        if (sl >= k) sl = -1;
+        const unsigned peers = __match_any_sync(0xffffffffu, sl);
+        const int rank = __popc(peers & ((1u << lane) - 1u));
+        int at = 0;
+        if (sl >= 0) at = s_cnt[sl];
+        __syncwarp();
+        if (sl >= 0) {
+          mem_b[at + rank] = i;
+          if (rank == 0) s_cnt[sl] = at + __popc(peers);
+        }
+        __syncwarp();
+      }
     }
   }
 }
