@@ -10,6 +10,8 @@ widened exactly to float64 before any arithmetic.
 
 Parity status of each function (what pins it, see tests/test_oracle_pins.py):
   attention_mass        pinned  (closed form via the summed query; hand-worked fixture)
+  attention_mass_heads  pinned  (its head mean is attention_mass; one head = attention_mass; the
+                                 per-head step with identical heads equals the default step)
   salience / mask_log   pinned  (hand-worked fixture; extremes; affine invariance)
   mask_matrix           pinned  (hand-enumerated 5x5 fixture; causal limit)
   attention_probs /
@@ -102,6 +104,14 @@ def attention_mass(q: np.ndarray, k: np.ndarray, v0: int, nv: int) -> np.ndarray
     return s / H
 
 
+def attention_mass_heads(q: np.ndarray, k: np.ndarray, v0: int, nv: int) -> np.ndarray:
+    """Eq. 1 kept per head: s^h_j = sum over visual queries i of W^h[i, j].  [H, nv].  (The variant in
+    which every head has its own salience and mask; the default combines the heads by their mean.)"""
+    H = q.shape[1]
+    qv, kv = q[v0:v0 + nv], k[v0:v0 + nv]
+    return np.stack([alignment(qv, kv, h).sum(axis=0) for h in range(H)])
+
+
 def salience(s: np.ndarray, eps: float = EPS_DEFAULT) -> np.ndarray:
     """Eq. 2: min-max normalisation over the image span."""
     s_min, s_max = s.min(), s.max()
@@ -149,12 +159,18 @@ def attention_probs(q: np.ndarray, k: np.ndarray, h: int, rows: np.ndarray, v0: 
 def rank_scores(q: np.ndarray, k: np.ndarray, v0: int, nv: int, r0: int, nr: int,
                 m: Optional[np.ndarray], mask_enable: bool) -> np.ndarray:
     """Ranking score of visual key j: the mean, over heads and over the ranking query rows
-    r0 .. r0+nr-1, of the Eq. 4 attention probability A[i, j]."""
+    r0 .. r0+nr-1, of the Eq. 4 attention probability A[i, j].  `m` is Eq. 3's vector [nv], or
+    one vector per head [H, nv] in the per-head variant."""
     H = q.shape[1]
     rows = np.arange(r0, r0 + nr)
     r = np.zeros(nv, dtype=np.float64)
-    M = mask_matrix(k.shape[0], rows, v0, nv, m, mask_enable)
+    per_head = m is not None and np.ndim(m) == 2
+    M = None if per_head else mask_matrix(k.shape[0], rows, v0, nv, m, mask_enable)
     for h in range(H):
+        if per_head:
+            A = attention_probs(q, k, h, rows, v0, nv, m[h], mask_enable)
+            r += A[:, v0:v0 + nv].sum(axis=0)
+            continue
         A = attention_probs(q, k, h, rows, v0, nv, m, mask_enable, M)
         r += A[:, v0:v0 + nv].sum(axis=0)
     return r / (H * nr)
@@ -228,21 +244,33 @@ def prune_sample(q_bits, k_bits, hidden_bits, pos_ids, v0: int, nv: int, r0: int
                  keep_k: int, lambda_max: float = 1.0, eps: float = EPS_DEFAULT,
                  sim_threshold: float = -math.inf, mask_enable: bool = True,
                  merge_enable: bool = True, assign_override: Optional[np.ndarray] = None,
-                 keep_override: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+                 keep_override: Optional[np.ndarray] = None, per_head: bool = False) -> Dict[str, np.ndarray]:
     """The prune step for one sequence [prefix | visual span | suffix].
 
     q_bits, k_bits: uint16 [n, H, d]; hidden_bits: uint16 [n, D]; pos_ids: int32 [n].
     keep_override / assign_override replace the oracle's own top-k / assignment (used by
-    the tests when a decision falls inside the stated tie band)."""
+    the tests when a decision falls inside the stated tie band).
+    per_head: Eq. 1-3 separately for every head (s^h, s_hat^h, m^h); head h's logits get head h's
+    mask; one token has one merge weight, the mean over heads of s_hat^h."""
     q = bf16_bits_to_f64(q_bits)
     k = bf16_bits_to_f64(k_bits)
     hid = bf16_bits_to_f64(hidden_bits)
     n = q.shape[0]
 
-    s = attention_mass(q, k, v0, nv)
-    s_hat = salience(s, eps)
-    m = mask_log(s_hat, lambda_max, eps)
-    r = rank_scores(q, k, v0, nv, r0, nr, m, mask_enable)
+    m_heads = None
+    if per_head:
+        s_heads = attention_mass_heads(q, k, v0, nv)
+        s_hat_heads = np.stack([salience(sh, eps) for sh in s_heads])
+        m_heads = np.stack([mask_log(x, lambda_max, eps) for x in s_hat_heads])
+        s = s_heads.mean(axis=0)
+        s_hat = s_hat_heads.mean(axis=0)
+        m = mask_log(s_hat, lambda_max, eps)
+        r = rank_scores(q, k, v0, nv, r0, nr, m_heads, mask_enable)
+    else:
+        s = attention_mass(q, k, v0, nv)
+        s_hat = salience(s, eps)
+        m = mask_log(s_hat, lambda_max, eps)
+        r = rank_scores(q, k, v0, nv, r0, nr, m, mask_enable)
 
     keep, drop = select_topk(r, keep_k)
     if keep_override is not None:
@@ -268,7 +296,7 @@ def prune_sample(q_bits, k_bits, hidden_bits, pos_ids, v0: int, nv: int, r0: int
     # rows that are pure copies must keep their exact bit pattern
     out_bits[:v0] = hidden_bits[:v0]
     out_bits[v0 + len(keep):] = hidden_bits[v0 + nv:]
-    return dict(mass=s, salience=s_hat, mask_log=m, rank_score=r, keep_idx=keep, drop_idx=drop,
+    return dict(mass=s, salience=s_hat, mask_log=m, mask_log_heads=m_heads, rank_score=r, keep_idx=keep, drop_idx=drop,
                 assign=assign, best_sim=best, margin=margin, merged=merged,
                 out_hidden=out_hidden, out_hidden_bits=out_bits,
                 out_pos=np.asarray(pos_ids)[src_row].astype(np.int32), src_row=src_row)
@@ -388,10 +416,11 @@ def masked_attention(q_bits, k_bits, v_bits, v0: int, nv: int, m: Optional[np.nd
     q, k, v = bf16_bits_to_f64(q_bits), bf16_bits_to_f64(k_bits), bf16_bits_to_f64(v_bits)
     n, H, d = q.shape
     rows = np.arange(n) if rows is None else np.asarray(rows)
-    M = mask_matrix(n, rows, v0, nv, m, mask_enable)
+    per_head = m is not None and np.ndim(m) == 2            # one mask vector per head
+    M = None if per_head else mask_matrix(n, rows, v0, nv, m, mask_enable)
     out = np.empty((len(rows), H, d))
     for h in range(H):
-        A = attention_probs(q, k, h, rows, v0, nv, m, mask_enable, M)
+        A = attention_probs(q, k, h, rows, v0, nv, m[h] if per_head else m, mask_enable, M)
         out[:, h, :] = A @ v[:, h, :]
     return out
 

@@ -662,3 +662,47 @@ def test_masked_attention_invariants():
     on, off = O.masked_attention(qb, kb, vb, v0, nv, m), O.masked_attention(qb, kb, vb, v0, nv, None, False)
     vis = np.zeros(n, bool); vis[v0:v0 + nv - 1] = True          # the last visual row has no future visual key
     assert np.array_equal(on[~vis], off[~vis]) and np.all(np.abs(on[vis] - off[vis]).max(axis=(1, 2)) > 1e-6)
+
+
+# ----------------------------------------------------------------------------- per-head variant of Eq. 1-3
+def test_per_head_masses_average_to_the_default_mass():
+    q, k = _rand_qk(30, 4, 16, 41)
+    sh = O.attention_mass_heads(q, k, 5, 20)
+    assert sh.shape == (4, 20)
+    assert np.allclose(sh.mean(axis=0), O.attention_mass(q, k, 5, 20), rtol=1e-13, atol=1e-13)
+    q1, k1 = q[:, :1], k[:, :1]
+    assert np.allclose(O.attention_mass_heads(q1, k1, 5, 20)[0], O.attention_mass(q1, k1, 5, 20), rtol=1e-14)
+
+
+def test_per_head_step_with_identical_heads_is_the_default_step():
+    rng = np.random.default_rng(42)
+    n, H, d, D, v0, nv = 40, 3, 8, 24, 4, 28
+    q1, k1 = rng.standard_normal((n, 1, d)), rng.standard_normal((n, 1, d))
+    qb, kb = _bf16_bits(np.repeat(q1, H, axis=1)), _bf16_bits(np.repeat(k1, H, axis=1))
+    hb = _bf16_bits(rng.standard_normal((n, D)))
+    kw = dict(lambda_max=0.7)
+    a = O.prune_sample(qb, kb, hb, np.arange(n), v0, nv, v0, n - v0, 9, per_head=True, **kw)     # ranking rows: image + text
+    b = O.prune_sample(qb, kb, hb, np.arange(n), v0, nv, v0, n - v0, 9, per_head=False, **kw)
+    for name in ("mass", "salience", "mask_log", "rank_score"):
+        assert np.allclose(a[name], b[name], rtol=1e-12, atol=1e-14), name
+    assert np.array_equal(a["keep_idx"], b["keep_idx"]) and np.array_equal(a["out_hidden_bits"], b["out_hidden_bits"])
+    assert np.allclose(a["mask_log_heads"], np.repeat(b["mask_log"][None], H, axis=0), rtol=1e-12, atol=1e-14)
+
+
+def test_per_head_masks_differ_and_follow_a_head_permutation():
+    rng = np.random.default_rng(43)
+    n, H, d, v0, nv = 36, 3, 8, 3, 25
+    qb, kb = _bf16_bits(rng.standard_normal((n, H, d))), _bf16_bits(rng.standard_normal((n, H, d)))
+    hb = _bf16_bits(rng.standard_normal((n, H * d)))
+    a = O.prune_sample(qb, kb, hb, np.arange(n), v0, nv, v0, n - v0, 8, per_head=True, lambda_max=0.9)
+    assert np.abs(a["mask_log_heads"][0] - a["mask_log_heads"][1]).max() > 1e-3
+    for h in range(H):                                       # every head's salience spans exactly [0, 1)
+        lam = np.exp(a["mask_log_heads"][h]) / 0.9
+        assert lam.max() > 0.99 and lam.min() <= 1e-6 / 0.9 + 1e-12
+    perm = [2, 0, 1]
+    b = O.prune_sample(qb[:, perm], kb[:, perm], hb, np.arange(n), v0, nv, v0, n - v0, 8, per_head=True, lambda_max=0.9)
+    assert np.allclose(b["mask_log_heads"], a["mask_log_heads"][perm], rtol=1e-13, atol=1e-14)
+    assert np.allclose(b["rank_score"], a["rank_score"], rtol=1e-12, atol=1e-15)
+    # a per-head mask really is used per head: the default step on the same data ranks differently
+    c = O.prune_sample(qb, kb, hb, np.arange(n), v0, nv, v0, n - v0, 8, per_head=False, lambda_max=0.9)
+    assert np.abs(c["rank_score"] - a["rank_score"]).max() > 1e-6
