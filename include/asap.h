@@ -95,6 +95,10 @@ typedef struct {
   float sim_threshold;  /* Sec. 4.2 threshold t: merge only if cosine similarity > t; -INFINITY = always */
   int32_t mask_enable;  /* 0: Eq. 3 is replaced by the causal mask of Sec. 3.2 */
   int32_t merge_enable; /* 0: kept tokens are copied unmerged, assign = -1 */
+  int32_t per_head_mask; /* 0: one salience and one mask for all heads, from the head-mean attention mass
+                            (the reading used throughout).  1: Eq. 1-3 separately per head -- s_j^h, s_hat_j^h,
+                            m_j^h -- head h's logits get head h's mask (asap_outputs::mask_log_heads), and a
+                            token's Eq. 5 weight is the mean over heads of s_hat_j^h.  Needs an even H. */
 } asap_params;
 
 /* Results.  Per-sequence arrays are padded to the stated pitch; entries past vis_len[b]
@@ -116,6 +120,9 @@ typedef struct {
   int32_t out_rows_capacity; /* rows available in out_hidden / out_pos / src_row; the step needs
                                 total_tokens - sum_b vis_len[b] + B * keep_k, which is at most
                                 total_tokens - B * (min_vis - keep_k) */
+  float *mask_log_heads;     /* [B, H, max_vis] m_j^h; written (and required) only with per_head_mask.  In that
+                                mode `mass` is the head mean of s_j^h, `salience` the head mean of s_hat_j^h and
+                                `mask_log` Eq. 3 of that mean (not used by the step itself). */
 } asap_outputs;
 
 /* Creates a context on `device` and takes all scratch memory the step will ever need for
@@ -176,7 +183,8 @@ asap_status asap_consolidate(asap_ctx *ctx, const asap_inputs *in, const asap_pa
  * for i < j when both i and j lie in the image span, and -infinity otherwise (other sequences of
  * the packed batch are never attended).  With p->mask_enable == 0 this is causal attention and
  * `mask_log` may be NULL; otherwise `mask_log` is the device array [B, max_vis] that asap_score
- * writes (asap_outputs::mask_log).  Only B, H, head_dim, D, total_tokens, the bounds, cu_seqlens,
+ * writes (asap_outputs::mask_log), or with p->per_head_mask the array [B, H, max_vis] of
+ * asap_outputs::mask_log_heads (head h then uses its own vector).  Only B, H, head_dim, D, total_tokens, the bounds, cu_seqlens,
  * the spans, q and k of `in` are read; `p` must be a valid parameter set (as for asap_score).
  * `v` and `out` are bf16 [total_tokens, H, head_dim] device tensors, 16-byte aligned, that must
  * not overlap.  `scratch`: caller-owned device memory of at least

@@ -45,7 +45,8 @@ class CInputs(C.Structure):
 
 class CParams(C.Structure):
     _fields_ = [("keep_k", C.c_int32), ("lambda_max", C.c_float), ("eps", C.c_float),
-                ("sim_threshold", C.c_float), ("mask_enable", C.c_int32), ("merge_enable", C.c_int32)]
+                ("sim_threshold", C.c_float), ("mask_enable", C.c_int32), ("merge_enable", C.c_int32),
+                ("per_head_mask", C.c_int32)]
 
 
 class CKernelTime(C.Structure):
@@ -57,7 +58,7 @@ class COutputs(C.Structure):
                 ("rank_score", C.c_void_p), ("keep_idx", C.c_void_p), ("drop_idx", C.c_void_p),
                 ("assign", C.c_void_p), ("best_sim", C.c_void_p), ("out_hidden", C.c_void_p),
                 ("out_pos", C.c_void_p), ("src_row", C.c_void_p), ("out_cu_seqlens", C.c_void_p),
-                ("out_rows_capacity", C.c_int32)]
+                ("out_rows_capacity", C.c_int32), ("mask_log_heads", C.c_void_p)]
 
 
 _lib = None
@@ -176,10 +177,11 @@ class Params:
     sim_threshold: float = -math.inf
     mask_enable: bool = True
     merge_enable: bool = True
+    per_head_mask: bool = False
 
     def c_struct(self) -> CParams:
         return CParams(self.keep_k, self.lambda_max, self.eps, self.sim_threshold, int(self.mask_enable),
-                       int(self.merge_enable))
+                       int(self.merge_enable), int(self.per_head_mask))
 
 
 @dataclasses.dataclass
@@ -196,15 +198,17 @@ class Outputs:
     out_pos: torch.Tensor
     src_row: torch.Tensor
     out_cu_seqlens: torch.Tensor
+    mask_log_heads: Optional[torch.Tensor] = None
 
     def c_struct(self) -> COutputs:
         return COutputs(_ptr(self.mass), _ptr(self.salience), _ptr(self.mask_log), _ptr(self.rank_score),
                         _ptr(self.keep_idx), _ptr(self.drop_idx), _ptr(self.assign), _ptr(self.best_sim),
                         _ptr(self.out_hidden), _ptr(self.out_pos), _ptr(self.src_row),
-                        _ptr(self.out_cu_seqlens), int(self.out_hidden.shape[0]))
+                        _ptr(self.out_cu_seqlens), int(self.out_hidden.shape[0]), _ptr(self.mask_log_heads))
 
 
-def alloc_outputs(inp: Inputs, keep_k: int, best_sim: bool = True, fill: bool = False) -> Outputs:
+def alloc_outputs(inp: Inputs, keep_k: int, best_sim: bool = True, fill: bool = False,
+                  per_head: bool = False) -> Outputs:
     """Caller-owned output tensors with the capacities the header states."""
     dev = inp.cu_seqlens.device
     B, mv = inp.B, inp.max_vis
@@ -219,7 +223,8 @@ def alloc_outputs(inp: Inputs, keep_k: int, best_sim: bool = True, fill: bool = 
                    best_sim=f32(B, nd) if best_sim else None,
                    out_hidden=torch.zeros(rows, inp.D, dtype=torch.bfloat16, device=dev) if fill
                    else torch.empty(rows, inp.D, dtype=torch.bfloat16, device=dev),
-                   out_pos=i32(rows), src_row=i32(rows), out_cu_seqlens=i32(B + 1))
+                   out_pos=i32(rows), src_row=i32(rows), out_cu_seqlens=i32(B + 1),
+                   mask_log_heads=f32(B, inp.H, mv) if per_head else None)
 
 
 def _stream(stream) -> int:

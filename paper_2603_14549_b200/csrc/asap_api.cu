@@ -137,6 +137,9 @@ asap_status validate(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
   }
   if ((need & NEED_SCORE_OUT) && (!out->mass || !out->salience || !out->mask_log || !out->rank_score))
     return fail(ctx, ASAP_ERR_INVALID, "null score output (mass / salience / mask_log / rank_score)");
+  if ((need & NEED_SCORE_OUT) && p->per_head_mask && !out->mask_log_heads)
+    return fail(ctx, ASAP_ERR_INVALID, "per_head_mask needs asap_outputs::mask_log_heads");
+  if (p->per_head_mask && (in->H & 1)) return fail(ctx, ASAP_ERR_UNSUPPORTED, "per_head_mask needs an even number of heads");
   const bool has_drops = in->max_vis > p->keep_k;   // otherwise the dropped-token arrays are empty
   if ((need & NEED_SELECT_OUT) && (!out->keep_idx || (!out->drop_idx && has_drops)))
     return fail(ctx, ASAP_ERR_INVALID, "null keep_idx / drop_idx");
@@ -232,8 +235,17 @@ asap_status launch_mass(asap_ctx *ctx, const asap_inputs *in, const asap_params 
   if (after_qsum && cudaEventRecord(after_qsum, st) != cudaSuccess)
     return fail(ctx, ASAP_ERR_CUDA, "event after the query-sum kernel");
 
-  const float scale = 1.0f / ((float)in->H * sqrtf((float)in->head_dim));
   const int row_blocks = (in->max_vis + MASS_ROWS - 1) / MASS_ROWS;
+  if (p->per_head_mask) {
+    // the per-head masses go through the scratch the score kernel fills afterwards
+    mark(ctx, "mass_heads", st);
+    launch_pdl(mass_heads_kernel, dim3(row_blocks, B), dim3(MASS_THREADS), (size_t)(D + 2 * in->H) * sizeof(float), st,
+               static_cast<const __nv_bfloat16 *>(in->k), ctx->desc, D, in->H, in->max_vis,
+               1.0f / sqrtf((float)in->head_dim), p->lambda_max, p->eps, ctx->qbar, ctx->score_partial, out->mass,
+               out->salience, out->mask_log, out->mask_log_heads, out->rank_score, ctx->cnt_mass);
+    return after_launch(ctx, "mass_heads");
+  }
+  const float scale = 1.0f / ((float)in->H * sqrtf((float)in->head_dim));
   mark(ctx, "mass_salience", st);
   launch_pdl(mass_salience_kernel, dim3(row_blocks, B), dim3(MASS_THREADS), (size_t)D * sizeof(float), st,
              static_cast<const __nv_bfloat16 *>(in->k), ctx->desc, D, in->max_vis, scale, p->lambda_max, p->eps,
@@ -252,7 +264,10 @@ asap_status launch_rank(asap_ctx *ctx, const asap_inputs *in, const asap_params 
   ScoreArgs sa;
   sa.pa = prepare_args(ctx, in, p, nullptr, 0x7fffffff); sa.pa.write_desc = 0; sa.B = B; sa.H = in->H; sa.max_vis = in->max_vis; sa.mask_enable = p->mask_enable ? 1 : 0;
   sa.scale_log2 = 1.4426950408889634f / sqrtf((float)in->head_dim);
-  sa.mask_log = out->mask_log; sa.partial = ctx->score_partial; sa.status = ctx->status;
+  sa.mask_log = p->per_head_mask ? out->mask_log_heads : out->mask_log;
+  sa.mask_b_stride = p->per_head_mask ? in->H * in->max_vis : in->max_vis;
+  sa.mask_h_stride = p->per_head_mask ? in->max_vis : 0;
+  sa.partial = ctx->score_partial; sa.status = ctx->status;
   mark(ctx, "score", st);
   const int items = B * in->H;
   launch_pdl(score_kernel, dim3(items < ctx->num_sms ? items : ctx->num_sms), dim3(SC_THREADS), SC_SMEM_BYTES, st,
@@ -634,6 +649,8 @@ asap_status asap_attention(asap_ctx *ctx, const asap_inputs *in, const asap_para
   aa.desc = ctx->desc; aa.H = in->H; aa.D = D; aa.max_vis = in->max_vis; aa.mask_enable = p->mask_enable ? 1 : 0;
   aa.scale_log2 = 1.4426950408889634f / sqrtf((float)in->head_dim);
   aa.mask_log = mask_log; aa.out = static_cast<__nv_bfloat16 *>(out); aa.status = ctx->status;
+  aa.mask_b_stride = p->per_head_mask ? in->H * in->max_vis : in->max_vis;
+  aa.mask_h_stride = p->per_head_mask ? in->max_vis : 0;
   mark(ctx, "attention", st);
   launch_pdl(attn_kernel, dim3((in->max_seq + 255) / 256, in->H, in->B), dim3(AT_THREADS), (size_t)AT_SMEM_BYTES, st,
              map_q, map_k, map_vt, aa);
@@ -674,7 +691,7 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
   // mass kernels then run on the context's side stream next to the score kernel, and rejoin before
   // the merge, which is the first consumer of the salience.  With caller-given ranking rows (which may
   // be visual) and while per-kernel timing is on, everything runs in order on `stream`.
-  const bool overlap = in->rank_start == nullptr && !ctx->prof_on && ctx->side != nullptr;
+  const bool overlap = in->rank_start == nullptr && !ctx->prof_on && ctx->side != nullptr && !p->per_head_mask;
   if (!overlap) {
     ASAP_TRY(launch_mass(ctx, in, p, out, true, out->out_cu_seqlens, out->out_rows_capacity, st));
     ASAP_TRY(launch_rank(ctx, in, p, out, false, st));

@@ -81,7 +81,8 @@ struct AttnArgs {
   const SampleDesc *desc;
   int H, D, max_vis, mask_enable;
   float scale_log2;            // log2(e) / sqrt(head_dim)
-  const float *mask_log;       // [B, max_vis] m_j (natural log), may be null with the mask off
+  const float *mask_log;       // [B, max_vis] m_j (natural log) or [B, H, max_vis]; may be null with the mask off
+  int mask_b_stride, mask_h_stride;   // max_vis, 0   or   H * max_vis, max_vis
   __nv_bfloat16 *out;          // [tokens, H, 128]
   uint32_t *status;
 };
@@ -266,7 +267,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
     const uint32_t s_addr = s_row + hf * 64;      // this thread's 64 logits
     const uint32_t p_addr = s_row + hf * 32;      // its 64 probabilities, packed in 32 columns
     const uint32_t o_addr = s_row + 128 + hf * 64;   // its 64 columns of O
-    const float *mlog_b = a.mask_log ? a.mask_log + (size_t)b * a.max_vis : nullptr;
+    const float *mlog_b = a.mask_log ? a.mask_log + (size_t)b * a.mask_b_stride + (size_t)h * a.mask_h_stride : nullptr;
     const int st = (threadIdx.x - 64) & 255;      // 0..255 inside the group
     const int my_kt = g == 0 ? n_kt0 : n_kt1;
     const bool my_sees = g == 0 ? sees0 : sees1;

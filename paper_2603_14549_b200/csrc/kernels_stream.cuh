@@ -283,6 +283,129 @@ mass_salience_kernel(const __nv_bfloat16 *__restrict__ k, const SampleDesc *__re
 }
 
 // =======================================================================================
+// mass_heads: Eq. 1-3 kept per head (the variant with one salience and one mask per head).
+//   s_j^h = qbar^h . k_j^h / sqrt(d): one warp per visual key row; a 16-byte vector of the row lies
+//   inside one head (16 vectors per head), so the two halves of the warp reduce two heads per pass.
+//   The block that finishes last for a sample then does, per head, the min-max normalisation (Eq. 2)
+//   and the mask vector (Eq. 3), and per token the head means: mass = mean_h s^h (equal to the
+//   default mass), salience = mean_h s_hat^h (the Eq. 5 weight), mask_log = Eq. 3 of that mean.
+// grid (row blocks, B); 8 warps x 4 rows each.  s_heads: scratch [B, H, max_vis].
+// Dynamic shared memory: D + 2 H floats.
+// =======================================================================================
+__global__ void __launch_bounds__(MASS_THREADS)
+mass_heads_kernel(const __nv_bfloat16 *__restrict__ k, const SampleDesc *__restrict__ desc, int D, int H,
+                  int max_vis, float scale, float lambda_max, float eps, const float *__restrict__ qbar,
+                  float *__restrict__ s_heads, float *__restrict__ mass, float *__restrict__ salience,
+                  float *__restrict__ mask_log, float *__restrict__ mask_log_heads,
+                  float *__restrict__ rank_score, unsigned int *__restrict__ counters) {
+  pdl_enter();
+  extern __shared__ float s_q[];   // [D] then lo[H], inv[H]
+  __shared__ int s_last;
+  const int b = blockIdx.y;
+  const SampleDesc d = desc[b];
+  float *mass_b = mass + (size_t)b * max_vis;
+  float *sal_b = salience + (size_t)b * max_vis, *msk_b = mask_log + (size_t)b * max_vis;
+  float *mh_b = mask_log_heads + (size_t)b * H * max_vis;
+  float *sh_b = s_heads + (size_t)b * H * max_vis;
+  if (!d.valid) {
+    for (int j = blockIdx.x * MASS_THREADS + threadIdx.x; j < max_vis; j += gridDim.x * MASS_THREADS) {
+      mass_b[j] = 0.f; sal_b[j] = 0.f; msk_b[j] = 0.f;
+      rank_score[(size_t)b * max_vis + j] = 0.f;   // the score kernel skips the sample
+      for (int h = 0; h < H; ++h) mh_b[(size_t)h * max_vis + j] = 0.f;
+    }
+    return;
+  }
+  const int nblocks = (d.nv + MASS_ROWS - 1) / MASS_ROWS;
+  if ((int)blockIdx.x >= nblocks) return;
+  for (int c = threadIdx.x * 4; c < D; c += MASS_THREADS * 4)
+    *reinterpret_cast<float4 *>(s_q + c) = __ldcg(reinterpret_cast<const float4 *>(qbar + (size_t)b * D + c));
+  __syncthreads();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int j0 = blockIdx.x * MASS_ROWS + warp * MASS_ROWS_PER_WARP;
+  const int nvec = D / 8;
+  const uint4 *rowp[MASS_ROWS_PER_WARP];
+#pragma unroll
+  for (int r = 0; r < MASS_ROWS_PER_WARP; ++r) {
+    const int j = min(j0 + r, d.nv - 1);   // clamp: duplicates are discarded below
+    rowp[r] = reinterpret_cast<const uint4 *>(k + (size_t)(d.row0 + d.v0 + j) * D);
+  }
+  for (int v0 = 0; v0 < nvec; v0 += 32) {      // one pass = 32 vectors = two heads
+    const int v = v0 + lane;
+    uint4 kv[MASS_ROWS_PER_WARP];
+#pragma unroll
+    for (int r = 0; r < MASS_ROWS_PER_WARP; ++r)
+      if (v < nvec) kv[r] = __ldg(rowp[r] + v);
+    float4 qa = make_float4(0.f, 0.f, 0.f, 0.f), qb = qa;
+    if (v < nvec) {
+      qa = *reinterpret_cast<const float4 *>(s_q + v * 8);
+      qb = *reinterpret_cast<const float4 *>(s_q + v * 8 + 4);
+    }
+    const int h = (v0 >> 4) + (lane >> 4);      // head of this half of the warp
+#pragma unroll
+    for (int r = 0; r < MASS_ROWS_PER_WARP; ++r) {
+      float part = 0.f;
+      if (v < nvec) {
+        float f[8];
+        unpack8(kv[r], f);
+        part = f[0] * qa.x + f[1] * qa.y + f[2] * qa.z + f[3] * qa.w + f[4] * qb.x + f[5] * qb.y + f[6] * qb.z +
+               f[7] * qb.w;
+      }
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);   // inside the 16 lanes
+      if ((lane & 15) == 0 && h < H && j0 + r < d.nv) sh_b[(size_t)h * max_vis + j0 + r] = part * scale;
+    }
+  }
+
+  // ---- last block of the sample ----
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned int old = atomicAdd(counters + b, 1u);
+    s_last = (old == (unsigned int)(nblocks - 1));
+    if (s_last) counters[b] = 0u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  float *s_lo = s_q + D, *s_inv = s_lo + H;
+  for (int h = warp; h < H; h += MASS_THREADS / 32) {           // Eq. 2's extremes, one warp per head
+    float lo = INFINITY, hi = -INFINITY;
+    for (int j = lane; j < d.nv; j += 32) {
+      const float sv = __ldcg(sh_b + (size_t)h * max_vis + j);
+      lo = fminf(lo, sv); hi = fmaxf(hi, sv);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (lane == 0) { s_lo[h] = lo; s_inv[h] = 1.0f / ((hi - lo) + eps); }
+  }
+  __syncthreads();
+  const float inv_h = 1.0f / (float)H;
+  for (int j = threadIdx.x; j < max_vis; j += MASS_THREADS) {
+    if (j < d.nv) {
+      float acc_s = 0.f, acc_sh = 0.f;
+      for (int h = 0; h < H; ++h) {                               // heads in order
+        const float sv = __ldcg(sh_b + (size_t)h * max_vis + j);
+        const float sh = (sv - s_lo[h]) * s_inv[h];
+        mh_b[(size_t)h * max_vis + j] = logf(fmaxf(lambda_max * sh, eps));
+        acc_s += sv;
+        acc_sh += sh;
+      }
+      const float sal = acc_sh * inv_h;
+      mass_b[j] = acc_s * inv_h;
+      sal_b[j] = sal;
+      msk_b[j] = logf(fmaxf(lambda_max * sal, eps));
+    } else {
+      mass_b[j] = 0.f; sal_b[j] = 0.f; msk_b[j] = 0.f;
+      for (int h = 0; h < H; ++h) mh_b[(size_t)h * max_vis + j] = 0.f;
+    }
+  }
+}
+
+// =======================================================================================
 // select: exact top-k by radix select over order-preserving 32-bit keys, equal scores resolved
 // toward the lower index, outputs in ascending index order.  One block per sample.
 // =======================================================================================

@@ -66,7 +66,8 @@ struct ScoreArgs {
                               // for the validation kernel (it writes nothing but scratch)
   int B, H, max_vis, mask_enable;
   float scale_log2;           // log2(e) / sqrt(head_dim)
-  const float *mask_log;      // [B, max_vis]  m_j (natural log)
+  const float *mask_log;      // [B, max_vis] m_j (natural log), or [B, H, max_vis] with a mask per head
+  int mask_b_stride, mask_h_stride;   // max_vis, 0   or   H * max_vis, max_vis
   float *partial;             // [B, H, max_vis] per-head sums over ranking rows
   uint32_t *status;
 };
@@ -258,7 +259,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       if (!d.valid) continue;
       const int n_rt = (d.nr + 127) / 128;
       float *part = a.partial + ((size_t)b * a.H + h) * a.max_vis;
-      const float *mlog = a.mask_log + (size_t)b * a.max_vis;
+      const float *mlog = a.mask_log + (size_t)b * a.mask_b_stride + (size_t)h * a.mask_h_stride;
       const int v_end = d.v0 + d.nv;
       {
         // visual keys beyond the tiles the first row tile visits in pass 2 (possible only when

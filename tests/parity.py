@@ -45,7 +45,8 @@ def compare_sample(batch, b, params, out, rank_start=None, rank_len=None, stats=
     qb, kb, hb = bits(batch.q[rows]), bits(batch.k[rows]), bits(batch.hidden[rows])
     pos = batch.pos_ids[rows].numpy()
     okw = dict(lambda_max=params.lambda_max, eps=params.eps, sim_threshold=params.sim_threshold,
-               mask_enable=params.mask_enable, merge_enable=params.merge_enable)
+               mask_enable=params.mask_enable, merge_enable=params.merge_enable,
+               per_head=bool(getattr(params, "per_head_mask", False)))
     ref = O.prune_sample(qb, kb, hb, pos, v0, nv, r0, nr, k, **okw)
 
     g = lambda t: t[b].detach().cpu().numpy()
@@ -61,6 +62,11 @@ def compare_sample(batch, b, params, out, rank_start=None, rank_len=None, stats=
     lam_g = np.exp(g(out.mask_log).astype(np.float64)[:nv])
     lam_o = np.exp(ref["mask_log"])
     assert np.max(np.abs(lam_g - lam_o)) <= 1e-4, f"mask_log sample {b}: {np.max(np.abs(lam_g - lam_o)):.3e}"
+    if okw["per_head"]:                                  # one mask vector per head, same bar
+        mh = out.mask_log_heads[b].detach().cpu().numpy().astype(np.float64)      # [H, max_vis]
+        err_h = np.abs(np.exp(mh[:, :nv]) - np.exp(ref["mask_log_heads"]))
+        assert err_h.max() <= 1e-4, f"mask_log_heads sample {b}: {err_h.max():.3e}"
+        assert np.all(mh[:, nv:] == 0.0), "mask_log_heads padding not zero"
 
     # ---- top-k
     keep_g = g(out.keep_idx)

@@ -144,3 +144,26 @@ def test_attention_at_benchmark_sizes_sampled_rows(big_ctx, name, B, samples):
         g = O.bf16_bits_to_f64(bits(out[rows][pick]))
         err = np.abs(g - ref)
         assert np.all(err <= np.maximum(2e-2, np.abs(ref) * 2.0 ** -7)), (b, err.max())
+
+
+def test_attention_with_a_mask_per_head(ctx):
+    """per_head_mask: head h adds its own Eq. 3 vector (asap_outputs::mask_log_heads layout [B, H, max_vis])."""
+    batch = W.tiny(B=2, n_vis=[200, 333], text_lens=[17, 5], H=2, keep_k=8, seed=612)
+    v = W.draw_values(batch, 83)
+    mv = int(batch.vis_len.max())
+    m = torch.zeros(batch.B, batch.H, mv)
+    ms = []
+    for b in range(batch.B):
+        rows = batch.sample_rows(b)
+        q, k = O.bf16_bits_to_f64(bits(batch.q[rows])), O.bf16_bits_to_f64(bits(batch.k[rows]))
+        v0, nv = int(batch.vis_start[b]), int(batch.vis_len[b])
+        mh = np.stack([O.mask_log(O.salience(sh), 0.8) for sh in O.attention_mass_heads(q, k, v0, nv)]).astype(np.float32)
+        m[b, :, :nv] = torch.from_numpy(mh)
+        ms.append(mh.astype(np.float64))
+    inp = A.make_inputs(batch, DEV)
+    out = torch.full((batch.total, batch.H, batch.head_dim), 7.0, dtype=torch.bfloat16, device=DEV)
+    scratch = torch.empty(A.asap_attention_scratch_bytes(batch.total, batch.D), dtype=torch.uint8, device=DEV)
+    A.asap_attention(ctx, inp, A.Params(keep_k=8, per_head_mask=True), m.to(DEV), v.to(DEV), scratch, out)
+    torch.cuda.synchronize(); A.asap_check(ctx)
+    _compare(batch, v, out.cpu(), ms)
+    assert float((m[0, 0] - m[0, 1]).abs().max()) > 1e-3

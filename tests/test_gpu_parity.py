@@ -24,7 +24,7 @@ def ctx():
 
 def run_step(ctx, batch, params, rank_start=None, rank_len=None, samples=None, stats=None):
     inp = A.make_inputs(batch, DEV, rank_start, rank_len)
-    out = A.alloc_outputs(inp, params.keep_k, fill=True)
+    out = A.alloc_outputs(inp, params.keep_k, fill=True, per_head=params.per_head_mask)
     A.asap_prune_step(ctx, inp, params, out)
     torch.cuda.synchronize()
     A.asap_check(ctx)
@@ -49,6 +49,23 @@ def test_visual_ranking_rows_use_the_soft_mask(ctx, lambda_max):
     rs = batch.vis_start.clone()
     rl = batch.vis_len + batch.text_len            # ranking rows = image span + text span
     run_step(ctx, batch, A.Params(keep_k=32, lambda_max=lambda_max), rs, rl)
+
+
+@pytest.mark.parametrize("lambda_max", [1.0, 0.3])
+def test_per_head_masks_with_visual_ranking_rows(ctx, lambda_max):
+    """Eq. 1-3 per head: four heads with their own salience and mask vector; the ranking rows include
+    the image span, so every head's logits are really shifted by that head's mask."""
+    batch = W.tiny(B=2, n_vis=[300, 129], text_lens=[20, 7], H=4, keep_k=32, seed=105, centres=8)
+    rs = batch.vis_start.clone()
+    rl = batch.vis_len + batch.text_len
+    inp, out = run_step(ctx, batch, A.Params(keep_k=32, lambda_max=lambda_max, per_head_mask=True), rs, rl)
+    mh = out.mask_log_heads.cpu()
+    assert float((mh[0, 0, :300] - mh[0, 1, :300]).abs().max()) > 1e-3      # the heads' masks do differ
+
+
+def test_per_head_masks_with_text_ranking_rows(ctx):
+    batch = W.tiny(B=3, n_vis=[130, 257, 64], text_lens=[5, 17, 33], H=2, keep_k=16, seed=106, centres=6)
+    run_step(ctx, batch, A.Params(keep_k=16, per_head_mask=True))
 
 
 def test_ranking_rows_partly_visual_and_mask_off(ctx):

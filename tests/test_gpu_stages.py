@@ -49,6 +49,31 @@ def test_score_entry_point_alone(ctx):
     assert int(out.keep_idx.min()) == -7          # untouched by asap_score
 
 
+def test_score_entry_point_per_head(ctx):
+    batch = W.tiny(B=2, n_vis=[140, 260], text_lens=[9, 3], H=4, keep_k=10, seed=305)
+    p = A.Params(keep_k=10, lambda_max=0.6, per_head_mask=True)
+    inp = A.make_inputs(batch, DEV)
+    out = A.alloc_outputs(inp, 10, fill=True, per_head=True)
+    A.asap_score(ctx, inp, p, out)
+    torch.cuda.synchronize(); A.asap_check(ctx)
+    for b in range(2):
+        rows = batch.sample_rows(b)
+        ref = O.prune_sample(bits(batch.q[rows]), bits(batch.k[rows]), bits(batch.hidden[rows]),
+                             batch.pos_ids[rows].numpy(), int(batch.vis_start[b]), int(batch.vis_len[b]),
+                             int(batch.text_start[b]), int(batch.text_len[b]), 10, lambda_max=0.6, per_head=True)
+        nv = int(batch.vis_len[b])
+        for name in ("mass", "salience", "rank_score"):
+            g = getattr(out, name)[b, :nv].cpu().numpy().astype(np.float64)
+            o = ref[name]
+            err = np.abs(g - o) / np.maximum(np.abs(o), 1e-3 * np.abs(o).max())
+            assert err.max() <= 1e-3, (name, b, err.max())
+        mh = out.mask_log_heads[b, :, :nv].cpu().numpy().astype(np.float64)
+        assert np.abs(np.exp(mh) - np.exp(ref["mask_log_heads"])).max() <= 1e-4
+    with pytest.raises(A.AsapError) as e:                      # the per-head array is required in this mode
+        A.asap_score(ctx, inp, p, A.alloc_outputs(inp, 10))
+    assert e.value.status == -1
+
+
 def test_select_is_bit_exact_with_ties(ctx):
     """asap_select on given fp32 scores must reproduce the stable top-k exactly, ties included."""
     g = torch.Generator().manual_seed(5)
