@@ -330,17 +330,24 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     }
     // a grid between one and two blocks per SM runs as one wave if two blocks fit on an SM:
     // give each block half of the shared memory and of the tensor memory then
+    // Several slot tiles whose accumulators fit tensor memory together: one pass over the hidden
+    // dimension with all of them live, so the visual rows are read once (a stage is then one 64-column
+    // block of the rows and of every slot tile).
+    // Taken only while three such stages still fit (up to 384 slots): with two, the shorter copies
+    // cost more than the second read of the rows (measured: 320 slots 87 -> 77 us, 510 slots 91 -> 96 us).
+    const bool wide = n_nt >= 2 && n_nt * n_tile <= 512 && 3 * (SIM_A_BYTES + n_nt * n_tile * 128) <= 192 * 1024;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < 2 * n_tile) tmem_cols <<= 1;
+    while ((int)tmem_cols < (wide ? n_nt * n_tile : 2 * n_tile)) tmem_cols <<= 1;
+    const int stage_bytes_used = wide ? SIM_A_BYTES + n_nt * n_tile * 128 : stage_bytes;
     const long long ctas = (long long)max_mt * B * splits;
-    const bool two_per_sm = ctas > ctx->num_sms && ctas <= 2LL * ctx->num_sms && tmem_cols <= 256 &&
+    const bool two_per_sm = !wide && ctas > ctx->num_sms && ctas <= 2LL * ctx->num_sms && tmem_cols <= 256 &&
                             2 * stage_bytes <= 96 * 1024;
     // at most 192 KB of tiles: the block then fits the 196 KB shared-memory carve-out, which leaves
     // the SM its 32 KB of L1
-    int stages = ((two_per_sm ? 96 : 192) * 1024) / stage_bytes;
+    int stages = ((two_per_sm ? 96 : 192) * 1024) / stage_bytes_used;
     if (stages > SIM_MAX_STAGES) stages = SIM_MAX_STAGES;
-    const size_t smem = (size_t)stages * stage_bytes + SIM_BOOK_BYTES + 1024;
-    if ((size_t)(SIM_THREADS / 32 + 1) * k * sizeof(int) > (size_t)stages * stage_bytes)
+    const size_t smem = (size_t)stages * stage_bytes_used + SIM_BOOK_BYTES + 1024;
+    if ((size_t)(SIM_THREADS / 32 + 1) * k * sizeof(int) > (size_t)stages * stage_bytes_used)
       return fail(ctx, ASAP_ERR_UNSUPPORTED, "keep_k = %d is too large for the merge path", k);
     CUtensorMap map_h, map_kept;
     if (!make_map(ctx, &map_h, in->hidden, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
@@ -349,6 +356,7 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     SimArgs sa;
     sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = n_tile;
     sa.n_nt = n_nt; sa.stages = stages; sa.splits = splits; sa.max_mt = max_mt; sa.tmem_cols = tmem_cols;
+    sa.wide = wide ? 1 : 0;
     sa.threshold = p->sim_threshold;
     sa.role = ctx->role; sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
     sa.best_sim = out->best_sim; sa.seg = ctx->seg; sa.members = ctx->members; sa.counters = ctx->cnt_sim;
@@ -441,6 +449,7 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   SimArgs sa;
   sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = n_tile;
   sa.n_nt = n_nt; sa.stages = stages; sa.splits = splits; sa.max_mt = max_mt; sa.tmem_cols = tmem_cols;
+  sa.wide = 0;
   sa.threshold = p->sim_threshold;
   sa.role = ctx->role; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
   sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr; sa.tile_counters = ctx->cnt_tiles;

@@ -485,6 +485,10 @@ head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
 //                   row tile adds the slices in slice order and does the same epilogue.
 // Rows that were kept, or lie past the image span, are computed but not written.
 // The block that finishes a sample's last row tile groups the dropped tokens by destination.
+//   one pass:       (a.wide, when all kept slots fit the 512 tensor-memory columns) the accumulators of
+//                   all slot tiles are live at once and a stage is one 64-column block of the rows
+//                   plus the matching block of EVERY slot tile, so the visual rows are read from
+//                   memory once instead of once per slot tile.
 //   matrix mode:    (a.smat set) the row operand is the dense kept-row array too, and
 //                   the epilogue writes the whole keep_k x keep_k cosine matrix of the sample,
 //                   S[p][q] = <h_p, h_q> * (1/||h_p|| * 1/||h_q||), for the routing inside the
@@ -499,6 +503,7 @@ constexpr int SIM_MAX_STAGES = 8;
 struct SimArgs {
   const SampleDesc *desc;
   int D, max_vis, keep_k, n_tile, n_nt, stages, splits, max_mt;
+  int wide;                  // 1: one pass, all slot tiles' accumulators live at once
   uint32_t tmem_cols;        // power of two >= 2 * n_tile: two accumulators
   float threshold;
   const int32_t *role;       // [B, max_vis]
@@ -545,7 +550,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   // a stage holds two adjacent 64-column blocks (256 contiguous bytes of every row):
   // [ rows, block 0 | rows, block 1 | kept, block 0 | kept, block 1 ]
   const int b_bytes = a.n_tile * 128;
-  const int stage_bytes = 2 * (SIM_A_BYTES + b_bytes);
+  const int stage_bytes = a.wide ? SIM_A_BYTES + a.n_nt * b_bytes : 2 * (SIM_A_BYTES + b_bytes);
   SimBook *bk = reinterpret_cast<SimBook *>(base_ptr + (size_t)a.stages * stage_bytes);
 
   if (threadIdx.x == 0) {
@@ -570,9 +575,10 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   tc_fence_after();
   const uint32_t tmem_base = bk->tmem_base;
   WaitCtx wc{&bk->abort_flag, a.status, STATUS_SIM_TIMEOUT, TC_WAIT_LIMIT};
-  const int n_kb = (a.D / 128) / a.splits;         // 128-column steps of this slice
+  // steps of this slice: 128 columns each, or 64 in the one-pass layout
+  const int n_kb = a.wide ? (a.D / 64) / a.splits : (a.D / 128) / a.splits;
   const int kb0 = z * n_kb;
-  const int total_it = a.n_nt * n_kb;
+  const int total_it = a.wide ? n_kb : a.n_nt * n_kb;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -590,6 +596,14 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         if (bk->abort_flag) break;
         const uint32_t dst = base + s * stage_bytes;
         mbar_expect_tx(smem_u32(&bk->full[s]), stage_bytes);
+        if (a.wide) {
+          tma_load_2d(dst, &tmap_h, smem_u32(&bk->full[s]), kb * 64, row_a);
+          for (int t = 0; t < a.n_nt; ++t)
+            tma_load_2d(dst + SIM_A_BYTES + t * b_bytes, &tmap_kept, smem_u32(&bk->full[s]), kb * 64,
+                        row_b + t * a.n_tile);
+          issued = it + 1;
+          continue;
+        }
         tma_load_2d(dst, &tmap_h, smem_u32(&bk->full[s]), kb * 128, row_a);
         tma_load_2d(dst + SIM_A_BYTES, &tmap_h, smem_u32(&bk->full[s]), kb * 128 + 64, row_a);
         tma_load_2d(dst + 2 * SIM_A_BYTES, &tmap_kept, smem_u32(&bk->full[s]), kb * 128, row_b + nt * a.n_tile);
@@ -609,7 +623,25 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_bf16(128, a.n_tile);
       int it = 0;
-      for (int nt = 0; nt < a.n_nt; ++nt) {
+      if (a.wide) {
+        for (int kb = 0; kb < n_kb; ++kb) {
+          const int s = kb % a.stages;
+          mbar_wait(smem_u32(&bk->full[s]), (kb / a.stages) & 1, wc);
+          tc_fence_after();
+          if (!bk->abort_flag) {
+            const uint32_t sa = base + s * stage_bytes, sb = sa + SIM_A_BYTES;
+            for (int t = 0; t < a.n_nt; ++t)
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk)
+                tc_mma_bf16(tmem_base + t * a.n_tile, umma_desc_sw128(sa + kk * 32),
+                            umma_desc_sw128(sb + t * b_bytes + kk * 32), idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+            tc_commit(smem_u32(&bk->empty[s]));
+            if (a.smat) mbar_arrive_n(smem_u32(&bk->empty[s]), 4);
+          }
+        }
+        if (!bk->abort_flag) tc_commit(smem_u32(&bk->acc_full[0]));
+      }
+      for (int nt = 0; nt < (a.wide ? 0 : a.n_nt); ++nt) {
         const int buf = nt & 1;
         if (nt >= 2) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((nt >> 1) - 1) & 1, wc);
         const uint32_t dcol = tmem_base + buf * (a.tmem_cols >> 1);
@@ -646,6 +678,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       if (!bk->abort_flag) {
 #pragma unroll
         for (int hb = 0; hb < 2; ++hb) {
+          if (hb == 1 && a.wide) break;                  // one 64-column block of the rows per stage
           const uint4 *row = reinterpret_cast<const uint4 *>(base_ptr + (size_t)s * stage_bytes +
                                                              hb * SIM_A_BYTES + lrow * 128);
 #pragma unroll
@@ -672,10 +705,11 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       a.ss_part[tile * 128 + lrow] = ss;
     }
     for (int nt = 0; nt < a.n_nt; ++nt) {
-      const int buf = nt & 1;
-      mbar_wait(smem_u32(&bk->acc_full[buf]), (nt >> 1) & 1, wc);
+      const int buf = a.wide ? 0 : (nt & 1);
+      mbar_wait(smem_u32(&bk->acc_full[buf]), a.wide ? 0 : ((nt >> 1) & 1), wc);
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (a.tmem_cols >> 1);
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) +
+                             (a.wide ? nt * a.n_tile : buf * (a.tmem_cols >> 1));
       const int slot0 = nt * a.n_tile;
       const int ncol = min(a.n_tile, a.keep_k - slot0);   // kept slots in this accumulator
 #pragma unroll 1

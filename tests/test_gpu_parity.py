@@ -38,6 +38,14 @@ def test_ragged_multi_tile(ctx):
     run_step(ctx, batch, A.Params(keep_k=16))
 
 
+@pytest.mark.parametrize("k", [300, 512, 257])
+def test_two_slot_tiles_in_one_pass(ctx, k):
+    """257 .. 512 kept slots: two slot tiles whose accumulators share tensor memory, one pass over the
+    hidden dimension (300 and 257 leave a ragged second slot tile, 512 fills every column)."""
+    batch = W.tiny(B=2, n_vis=[700, 650], text_lens=[12, 40], H=2, keep_k=k, seed=107, centres=30)
+    run_step(ctx, batch, A.Params(keep_k=k))
+
+
 def test_text_longer_than_one_row_tile(ctx):
     batch = W.tiny(B=2, n_vis=[200, 140], text_lens=[150, 129], H=2, keep_k=40, seed=102, centres=8)
     run_step(ctx, batch, A.Params(keep_k=40))
