@@ -46,6 +46,16 @@ def test_two_slot_tiles_in_one_pass(ctx, k):
     run_step(ctx, batch, A.Params(keep_k=k))
 
 
+def test_many_row_tiles_and_three_slot_tiles(ctx):
+    """A batch large enough that the similarity kernel runs unsliced with more blocks than SMs
+    (15 sequences x 19 row tiles) and three slot tiles (600 kept slots).  Odd and even numbers of row
+    tiles, a ragged last tile of one row; the oracle checks three sequences."""
+    nvs = [2350 if b % 2 else 2432 for b in range(15)]
+    nvs[0] = 2305                                               # 19 row tiles, one row in the last
+    batch = W.tiny(B=15, n_vis=nvs, text_lens=[6 + b for b in range(15)], H=2, keep_k=600, seed=108, centres=40)
+    run_step(ctx, batch, A.Params(keep_k=600), samples=[0, 1, 14])
+
+
 def test_text_longer_than_one_row_tile(ctx):
     batch = W.tiny(B=2, n_vis=[200, 140], text_lens=[150, 129], H=2, keep_k=40, seed=102, centres=8)
     run_step(ctx, batch, A.Params(keep_k=40))
