@@ -300,6 +300,33 @@ def run_cuda(args):
     ktimes = A.asap_profile_read(ctx)
     A.asap_profile(ctx, False)
 
+    # ---- the same steps replayed from a CUDA graph (one graph holding one step per device copy of
+    # the inputs, so the rotation through the copies is kept); reported beside the headline, not as it
+    graph = None
+    if args.graph_iters > 0:
+        cap = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(cap):
+            for i in range(n_copies):
+                A.asap_prune_step(ctx, copies[i], params, out, cap)
+            cap.synchronize()
+            g.capture_begin()
+            for i in range(n_copies):
+                A.asap_prune_step(ctx, copies[i], params, out, cap)
+            g.capture_end()
+            g.replay()
+            cap.synchronize()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(cap)
+            for _ in range(args.graph_iters):
+                g.replay()
+            g1.record(cap)
+            cap.synchronize()
+        A.asap_check(ctx)
+        graph = {"us_per_step": g0.elapsed_time(g1) / (args.graph_iters * n_copies) * 1e3,
+                 "steps": args.graph_iters * n_copies, "steps_per_graph": n_copies}
+        del g
+
     # ---- KV-cache compaction of the layers up to the pruning layer (next-row feature, timed apart
     # from the step: keys and values of `kv_layers` layers gathered with the step's row map)
     kv = None
@@ -486,7 +513,7 @@ def run_cuda(args):
         "latency_us": {"p10": per_step[len(per_step) // 10] * 1e3, "p50": per_step[len(per_step) // 2] * 1e3,
                        "p90": per_step[(len(per_step) * 9) // 10] * 1e3},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "kernels": kernels,
-        "cpu_baseline": cpu, "kv_compaction": kv, "consolidate_within_kept": cons, "masked_attention": attn,
+        "cpu_baseline": cpu, "kv_compaction": kv, "consolidate_within_kept": cons, "masked_attention": attn, "graph_replay": graph,
     }
     print(json.dumps(line))
     R.shutdown()
@@ -507,6 +534,8 @@ def main():
                     help="also time KV-cache compaction of this many layers (0 = skip)")
     ap.add_argument("--consolidate-threshold", type=float, default=0.8,
                     help="also time asap_consolidate (Sec. 4.2 inside the kept set) with this threshold t")
+    ap.add_argument("--graph-iters", type=int, default=40,
+                    help="replays of a CUDA graph holding one step per input copy (0 = skip)")
     ap.add_argument("--consolidate-iters", type=int, default=50, help="timed asap_consolidate calls (0 = skip)")
     ap.add_argument("--attention-iters", type=int, default=10,
                     help="also time asap_attention (the layer's attention under the SG-BiMask) this many times (0 = skip)")

@@ -195,7 +195,10 @@ asap_status asap_attention(asap_ctx *ctx, const asap_inputs *in, const asap_para
                            const float *mask_log, const void *v, void *scratch, size_t scratch_bytes,
                            void *out, void *stream);
 
-/* Steps 1a-5 back to back on `stream`; fills every field of `out`. */
+/* Steps 1a-5 back to back on `stream`; fills every field of `out`.  The call may be recorded by a
+ * stream capture (it allocates nothing and does not synchronise; the context's side stream forks from
+ * and joins back into `stream` inside the call) and the graph replayed on new contents of the same
+ * buffers. */
 asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                             const asap_outputs *out, void *stream);
 

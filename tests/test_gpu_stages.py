@@ -251,3 +251,37 @@ def test_kv_cache_compaction_follows_the_row_map(ctx):
         assert torch.all(d[n_out:] == 7.0)                          # capacity tail untouched
     with pytest.raises(A.AsapError):                                # 65 tensors: refused before any launch
         A.asap_compact_kv(ctx, out.src_row, out.out_cu_seqlens[batch.B:], src * 11, dst * 11)
+
+
+def test_prune_step_can_be_captured_into_a_cuda_graph(ctx):
+    """The step allocates nothing, never synchronises, and its side stream forks from and joins back
+    into the caller's stream inside the call, so a stream capture records it whole; a replay on new
+    input contents (same buffers) gives what a direct call gives, bit for bit."""
+    batch = W.tiny(B=3, n_vis=[300, 170, 520], text_lens=[9, 30, 4], H=2, keep_k=48, seed=306, centres=8)
+    other = W.tiny(B=3, n_vis=[300, 170, 520], text_lens=[9, 30, 4], H=2, keep_k=48, seed=307, centres=8)
+    inp = A.make_inputs(batch, DEV)
+    p = A.Params(keep_k=48)
+    out = A.alloc_outputs(inp, 48, fill=True)
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        A.asap_prune_step(ctx, inp, p, out, s)
+        s.synchronize()
+        g.capture_begin()
+        A.asap_prune_step(ctx, inp, p, out, s)
+        g.capture_end()
+    for src in (other, batch):
+        for name in ("q", "k", "hidden"):                       # new contents, same device buffers
+            getattr(inp, name).copy_(getattr(src, name).to(DEV))
+        ref = A.alloc_outputs(inp, 48, fill=True)
+        A.asap_prune_step(ctx, inp, p, ref)
+        torch.cuda.synchronize()
+        for t in (out.out_hidden, out.keep_idx, out.rank_score, out.out_pos):
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize(); A.asap_check(ctx)
+        n_out = int(ref.out_cu_seqlens[-1])                  # rows past it are untouched capacity
+        for name in ("keep_idx", "drop_idx", "assign", "rank_score", "salience", "out_cu_seqlens"):
+            assert torch.equal(getattr(out, name), getattr(ref, name)), name
+        for name in ("out_hidden", "out_pos", "src_row"):
+            assert torch.equal(getattr(out, name)[:n_out], getattr(ref, name)[:n_out]), name
