@@ -167,3 +167,22 @@ def test_attention_with_a_mask_per_head(ctx):
     torch.cuda.synchronize(); A.asap_check(ctx)
     _compare(batch, v, out.cpu(), ms)
     assert float((m[0, 0] - m[0, 1]).abs().max()) > 1e-3
+
+
+def test_attention_skips_a_bad_sequence(ctx):
+    batch = W.tiny(B=2, n_vis=[200, 150], text_lens=[4, 4], H=2, keep_k=8, seed=613)
+    v = W.draw_values(batch, 84)
+    good = _run(ctx, batch, v, None, mask_enable=False)
+    inp = A.make_inputs(batch, DEV)
+    bad = batch.vis_len.clone(); bad[0] = 9999
+    inp.vis_len = bad.to(DEV)
+    out = torch.full((batch.total, batch.H, batch.head_dim), 7.0, dtype=torch.bfloat16, device=DEV)
+    scratch = torch.empty(A.asap_attention_scratch_bytes(batch.total, batch.D), dtype=torch.uint8, device=DEV)
+    A.asap_attention(ctx, inp, A.Params(keep_k=8, mask_enable=False), None, v.to(DEV), scratch, out)
+    torch.cuda.synchronize()
+    with pytest.raises(A.AsapError) as e:
+        A.asap_check(ctx)
+    assert e.value.status == -6
+    r0, r1 = batch.sample_rows(0), batch.sample_rows(1)
+    assert torch.all(out[r0].float() == 7.0)                    # skipped: untouched
+    assert torch.equal(out[r1].cpu(), good[r1])

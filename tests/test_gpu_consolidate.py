@@ -205,3 +205,32 @@ def test_consolidate_at_benchmark_sizes(big_ctx, name, t, samples):
     out, n_abs, st1 = _run(big_ctx, batch, k, t, stage1=lambda bt, b, kk: W.random_stage1(bt, b, kk, 900))
     assert np.all(n_abs >= 0) and np.all(n_abs <= np.asarray(batch.vis_len) - k)
     assert _check(batch, k, t, out, n_abs, st1, samples=samples) > 0
+
+
+def test_a_bad_sequence_is_skipped_and_flagged(ctx):
+    """Device-side validation: a sequence whose span does not fit its length is skipped (outputs -1 / 0
+    rows untouched), the status word says so, the other sequence is processed normally."""
+    batch = W.tiny(B=2, n_vis=[200, 150], text_lens=[4, 4], H=2, keep_k=40, seed=515, centres=5)
+    good_out, good_abs, st1 = _run(ctx, batch, 40, 0.8)
+    inp = A.make_inputs(batch, DEV)
+    bad_len = batch.vis_len.clone(); bad_len[0] = 9999
+    inp.vis_len = bad_len.to(DEV)
+    mv = inp.max_vis
+    mass = torch.zeros(2, mv); sal = torch.zeros(2, mv)
+    keep = torch.zeros(2, 40, dtype=torch.int32); drop = torch.full((2, mv - 40), -1, dtype=torch.int32)
+    for b in range(2):
+        m, s, kp, dp = st1[b]
+        nv = int(batch.vis_len[b])
+        mass[b, :nv] = torch.from_numpy(m).float(); sal[b, :nv] = torch.from_numpy(s).float()
+        keep[b] = torch.from_numpy(kp); drop[b, :nv - 40] = torch.from_numpy(dp)
+    out = A.alloc_outputs(inp, 40, fill=True)
+    scratch = torch.empty(A.asap_consolidate_scratch_bytes(2, 40), dtype=torch.uint8, device=DEV)
+    n_abs = torch.full((2,), -7, dtype=torch.int32, device=DEV)
+    A.asap_consolidate(ctx, inp, A.Params(keep_k=40, sim_threshold=0.8), mass.to(DEV), sal.to(DEV), keep.to(DEV),
+                       drop.to(DEV), scratch, out, n_abs)
+    torch.cuda.synchronize()
+    with pytest.raises(A.AsapError) as e:
+        A.asap_check(ctx)
+    assert e.value.status == -6 and "validation" in str(e.value)
+    assert torch.all(out.keep_idx[0] == -1) and int(n_abs[0]) == 0
+    assert torch.equal(out.keep_idx[1], good_out.keep_idx[1]) and int(n_abs[1]) == int(good_abs[1])
