@@ -489,6 +489,13 @@ select_kernel(const float *__restrict__ rank_score, const SampleDesc *__restrict
       if (j < nv) {
         const float *p = head_partial + (size_t)b * H * max_vis + j;
         int hh = 0;
+        for (; hh + 32 <= H; hh += 32) {         // 32 loads in flight: one round trip for 32 heads
+          float v[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = __ldcg(p + (size_t)(hh + e) * max_vis);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) tot += v[e];
+        }
         for (; hh + 8 <= H; hh += 8) {
           float v[8];
 #pragma unroll
