@@ -7,7 +7,10 @@ scores, top-k, cosine assignment, weighted merge, compaction) over one synthetic
 default workload is the LLaVA-1.5-7B-shaped batch of 16 sequences (576 visual tokens, ragged
 text, keep 64).  One JSON line is printed by rank 0:
 
-  value          visual tokens per second, inputs resident in HBM, all ranks together
+  value          visual tokens per second, inputs resident in HBM, all ranks together; the timed steps
+                 are replayed from a CUDA graph holding one step per device copy of the inputs
+                 (config.timed_as; --no-graph times directly launched steps, which the line also
+                 reports as direct_launch)
   e2e            the same with inputs in pinned host memory: every step copies them to the
                  device, runs the step through the C ABI and reads the shortened batch back
   roofline       the kernel with the largest share of the step, against the measured peak
@@ -253,7 +256,8 @@ def run_cuda(args):
                       max_keep_rows=batch.B * keep_k)
     copies = device_copies(A, batch, device, n_copies)
     out = A.alloc_outputs(copies[0], keep_k)
-    stream = torch.cuda.current_stream()
+    stream = torch.cuda.Stream(device=device)     # a stream of our own: the legacy stream cannot be captured
+    torch.cuda.set_stream(stream)
 
     rank_visual = args.rank_rows == "visual+text"
     if rank_visual:       # Eq. 3 acts on these rows; the score kernel becomes a dense, tensor-pipe-heavy pass
@@ -274,21 +278,48 @@ def run_cuda(args):
         step(i)
     torch.cuda.synchronize()
     A.asap_check(ctx)
-    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    # The timed steps are replayed from a CUDA graph that holds one step per device copy of the inputs
+    # (the library's calls are capturable: no allocation, no synchronisation, the side stream joins back
+    # inside the call), K / copies replays = exactly K steps.  --no-graph, or a K that the number of
+    # copies does not divide, times directly launched steps instead.
+    graph, per_replay = None, 1
+    if not args.no_graph and args.steps % n_copies == 0:
+        try:
+            c0 = A.asap_launch_count(ctx)
+            graph = torch.cuda.CUDAGraph()
+            graph.capture_begin()
+            for i in range(n_copies):
+                step(i)
+            graph.capture_end()
+            launches_per_replay = A.asap_launch_count(ctx) - c0
+            graph.replay()
+            torch.cuda.synchronize()
+            A.asap_check(ctx)
+            per_replay = n_copies
+        except Exception as ex:                      # capture not available: fall back to direct launches
+            print(f"bench.py: graph capture failed ({ex!r}); timing directly launched steps", file=sys.stderr)
+            graph, per_replay = None, 1
+    n_marks = args.steps // per_replay
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_marks + 1)]
     launches0 = A.asap_launch_count(ctx)
     R.barrier(); torch.cuda.synchronize()
     wall_begin = time.time()
     marks[0].record(stream)
-    for i in range(args.steps):
-        step(args.warmup + i)
+    for i in range(n_marks):
+        if graph is not None:
+            graph.replay()
+        else:
+            step(args.warmup + i)
         marks[i + 1].record(stream)
     torch.cuda.synchronize(); R.barrier()
     wall_end = time.time()
     clocks = sampler.stop(wall_begin, wall_end) if rank == 0 else None
-    launches = A.asap_launch_count(ctx) - launches0
+    launches = launches_per_replay * n_marks if graph is not None else A.asap_launch_count(ctx) - launches0
     total_ms = marks[0].elapsed_time(marks[-1])
-    per_step = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
+    per_step = sorted(marks[i].elapsed_time(marks[i + 1]) / per_replay for i in range(n_marks))
     A.asap_check(ctx)
+    timed_as = (f"CUDA graph of {n_copies} steps (one per input copy) replayed {n_marks} times" if graph is not None
+                else "directly launched steps")
     total_ms_max = R.max_over_ranks(total_ms, device)
     units_all = R.sum_over_ranks(units, device)
 
@@ -300,32 +331,19 @@ def run_cuda(args):
     ktimes = A.asap_profile_read(ctx)
     A.asap_profile(ctx, False)
 
-    # ---- the same steps replayed from a CUDA graph (one graph holding one step per device copy of
-    # the inputs, so the rotation through the copies is kept); reported beside the headline, not as it
-    graph = None
-    if args.graph_iters > 0:
-        cap = torch.cuda.Stream()
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(cap):
-            for i in range(n_copies):
-                A.asap_prune_step(ctx, copies[i], params, out, cap)
-            cap.synchronize()
-            g.capture_begin()
-            for i in range(n_copies):
-                A.asap_prune_step(ctx, copies[i], params, out, cap)
-            g.capture_end()
-            g.replay()
-            cap.synchronize()
-            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            g0.record(cap)
-            for _ in range(args.graph_iters):
-                g.replay()
-            g1.record(cap)
-            cap.synchronize()
-        A.asap_check(ctx)
-        graph = {"us_per_step": g0.elapsed_time(g1) / (args.graph_iters * n_copies) * 1e3,
-                 "steps": args.graph_iters * n_copies, "steps_per_graph": n_copies}
-        del g
+    # ---- the same steps launched directly through the API, reported beside the headline
+    direct = None
+    if graph is not None and args.direct_steps > 0:
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for i in range(3):
+            step(i)
+        torch.cuda.synchronize()
+        d0.record(stream)
+        for i in range(args.direct_steps):
+            step(i)
+        d1.record(stream)
+        torch.cuda.synchronize()
+        direct = {"us_per_step": d0.elapsed_time(d1) / args.direct_steps * 1e3, "steps": args.direct_steps}
 
     # ---- KV-cache compaction of the layers up to the pruning layer (next-row feature, timed apart
     # from the step: keys and values of `kv_layers` layers gathered with the step's row map)
@@ -509,11 +527,12 @@ def run_cuda(args):
                    "visual_tokens_per_gpu": units, "keep_k": keep_k, "ranking_rows": "image span + text span" if rank_visual else "text span",
                    "l2": f"inputs rotate over {n_copies} device copies ({n_copies * in_bytes / 2**20:.0f} MiB) "
                          f"so no step finds its inputs in the {L2_BYTES // 2**20} MiB L2",
+                   "timed_as": timed_as,
                    "parallelism": "replicas only (one batch per GPU, no collective)"},
         "latency_us": {"p10": per_step[len(per_step) // 10] * 1e3, "p50": per_step[len(per_step) // 2] * 1e3,
                        "p90": per_step[(len(per_step) * 9) // 10] * 1e3},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "kernels": kernels,
-        "cpu_baseline": cpu, "kv_compaction": kv, "consolidate_within_kept": cons, "masked_attention": attn, "graph_replay": graph,
+        "cpu_baseline": cpu, "kv_compaction": kv, "consolidate_within_kept": cons, "masked_attention": attn, "direct_launch": direct,
     }
     print(json.dumps(line))
     R.shutdown()
@@ -534,8 +553,9 @@ def main():
                     help="also time KV-cache compaction of this many layers (0 = skip)")
     ap.add_argument("--consolidate-threshold", type=float, default=0.8,
                     help="also time asap_consolidate (Sec. 4.2 inside the kept set) with this threshold t")
-    ap.add_argument("--graph-iters", type=int, default=40,
-                    help="replays of a CUDA graph holding one step per input copy (0 = skip)")
+    ap.add_argument("--no-graph", action="store_true", help="time directly launched steps instead of graph replays")
+    ap.add_argument("--direct-steps", type=int, default=500,
+                    help="also time this many directly launched steps when the headline is a graph replay (0 = skip)")
     ap.add_argument("--consolidate-iters", type=int, default=50, help="timed asap_consolidate calls (0 = skip)")
     ap.add_argument("--attention-iters", type=int, default=10,
                     help="also time asap_attention (the layer's attention under the SG-BiMask) this many times (0 = skip)")
