@@ -234,3 +234,12 @@ def test_a_bad_sequence_is_skipped_and_flagged(ctx):
     assert e.value.status == -6 and "validation" in str(e.value)
     assert torch.all(out.keep_idx[0] == -1) and int(n_abs[0]) == 0
     assert torch.equal(out.keep_idx[1], good_out.keep_idx[1]) and int(n_abs[1]) == int(good_abs[1])
+
+
+def test_threshold_minus_infinity_absorbs_until_the_pool_is_empty(ctx):
+    """t = -inf: every token after the first is similar enough to some anchor, so the walk absorbs until
+    the pruned pool cannot refill another slot (here nv - k = 30 and 50 of the 59 candidates)."""
+    batch = W.tiny(B=2, n_vis=[90, 110], text_lens=[4, 4], H=2, keep_k=60, seed=516, centres=7)
+    out, n_abs, st1 = _run(ctx, batch, 60, -math.inf)
+    assert n_abs.tolist() == [30, 50]
+    _check(batch, 60, -math.inf, out, n_abs, st1)

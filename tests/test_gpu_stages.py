@@ -285,3 +285,13 @@ def test_prune_step_can_be_captured_into_a_cuda_graph(ctx):
             assert torch.equal(getattr(out, name), getattr(ref, name)), name
         for name in ("out_hidden", "out_pos", "src_row"):
             assert torch.equal(getattr(out, name)[:n_out], getattr(ref, name)[:n_out]), name
+
+
+def test_per_head_mask_needs_an_even_number_of_heads(ctx):
+    batch = W.tiny(B=1, n_vis=[100], text_lens=[4], H=3, keep_k=8, seed=308)
+    inp = A.make_inputs(batch, DEV)
+    out = A.alloc_outputs(inp, 8, per_head=True)
+    n0 = A.asap_launch_count(ctx)
+    with pytest.raises(A.AsapError) as e:
+        A.asap_prune_step(ctx, inp, A.Params(keep_k=8, per_head_mask=True), out)
+    assert e.value.status == -5 and A.asap_launch_count(ctx) == n0
