@@ -434,6 +434,11 @@ def run_cuda(args):
         a_flops = 4.0 * batch.head_dim * pairs * batch.H
         attn = {"us": a_us, "admitted_pairs": pairs, "flops": a_flops, "TFLOPs": a_flops / a_us / 1e6,
                 "frac_of_bf16_peak": a_flops / a_us / 1e6 / peaks["bf16_tflops"], "kernel_us": ak}
+        if ak.get("attention"):       # the attention kernel alone against the measured burst peak
+            attn["roofline"] = {"kernel": "attention", "bound": "tensor", "achieved": a_flops / ak["attention"] / 1e6,
+                                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                "frac": a_flops / ak["attention"] / 1e6 / peaks["bf16_tflops"], "traffic": None,
+                                "peak_kind": peak_kind + " (burst)"}
         del v_dev, a_out, a_scr
 
     # ---- end to end from pinned host memory

@@ -186,3 +186,44 @@ def test_attention_skips_a_bad_sequence(ctx):
     r0, r1 = batch.sample_rows(0), batch.sample_rows(1)
     assert torch.all(out[r0].float() == 7.0)                    # skipped: untouched
     assert torch.equal(out[r1].cpu(), good[r1])
+
+
+def test_attention_and_consolidation_can_be_captured_into_a_cuda_graph(ctx):
+    """Both calls allocate nothing and do not synchronise: a stream capture records them, and a replay
+    reproduces the directly launched results bit for bit."""
+    batch = W.tiny(B=2, n_vis=[200, 150], text_lens=[4, 9], H=2, keep_k=40, seed=614, centres=5)
+    inp = A.make_inputs(batch, DEV)
+    p = A.Params(keep_k=40, sim_threshold=0.8)
+    step_out = A.alloc_outputs(inp, 40, fill=True)
+    A.asap_prune_step(ctx, inp, p, step_out)                           # stage-1 results to feed both calls
+    torch.cuda.synchronize()
+    v = W.draw_values(batch, 85).to(DEV)
+    st1 = [t.clone() for t in (step_out.mass, step_out.salience, step_out.keep_idx, step_out.drop_idx, step_out.mask_log)]
+    a_scr = torch.empty(A.asap_attention_scratch_bytes(batch.total, batch.D), dtype=torch.uint8, device=DEV)
+    c_scr = torch.empty(A.asap_consolidate_scratch_bytes(batch.B, 40), dtype=torch.uint8, device=DEV)
+
+    def run(att_out, cons_out, n_abs, stream=None):
+        A.asap_attention(ctx, inp, p, st1[4], v, a_scr, att_out, stream)
+        A.asap_consolidate(ctx, inp, p, st1[0], st1[1], st1[2], st1[3], c_scr, cons_out, n_abs, stream)
+
+    ref_att = torch.zeros_like(v); ref_cons = A.alloc_outputs(inp, 40, fill=True)
+    ref_abs = torch.zeros(batch.B, dtype=torch.int32, device=DEV)
+    run(ref_att, ref_cons, ref_abs)
+    torch.cuda.synchronize(); A.asap_check(ctx)
+    att = torch.zeros_like(v); cons = A.alloc_outputs(inp, 40, fill=True)
+    n_abs = torch.zeros(batch.B, dtype=torch.int32, device=DEV)
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        run(att, cons, n_abs, s)
+        s.synchronize()
+        g.capture_begin()
+        run(att, cons, n_abs, s)
+        g.capture_end()
+    att.zero_(); cons.out_hidden.zero_(); cons.keep_idx.zero_(); n_abs.zero_()
+    g.replay()
+    torch.cuda.synchronize(); A.asap_check(ctx)
+    n_out = int(ref_cons.out_cu_seqlens[-1])
+    assert torch.equal(att, ref_att) and torch.equal(n_abs, ref_abs) and int(ref_abs.sum()) > 0
+    assert torch.equal(cons.keep_idx, ref_cons.keep_idx) and torch.equal(cons.assign, ref_cons.assign)
+    assert torch.equal(cons.out_hidden[:n_out], ref_cons.out_hidden[:n_out])
