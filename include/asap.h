@@ -170,7 +170,8 @@ asap_status asap_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *
  * device memory of at least asap_consolidate_scratch_bytes(B, keep_k) bytes, 16-byte aligned
  * (the similarity matrix, keep_k * keep_k floats per sequence, and a bit matrix); nothing is
  * kept in it between calls.  Requires p->merge_enable and keep_k < max_vis (ASAP_ERR_INVALID
- * otherwise: asap_merge covers those cases) and keep_k <= 4096 (ASAP_ERR_UNSUPPORTED). */
+ * otherwise: asap_merge covers those cases) and keep_k <= 4096 (ASAP_ERR_UNSUPPORTED).  May be
+ * recorded by a stream capture. */
 size_t asap_consolidate_scratch_bytes(int32_t B, int32_t keep_k);
 asap_status asap_consolidate(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                              const float *mass, const float *salience, const int32_t *keep_idx,
@@ -189,7 +190,8 @@ asap_status asap_consolidate(asap_ctx *ctx, const asap_inputs *in, const asap_pa
  * `v` and `out` are bf16 [total_tokens, H, head_dim] device tensors, 16-byte aligned, that must
  * not overlap.  `scratch`: caller-owned device memory of at least
  * asap_attention_scratch_bytes(total_tokens, D) bytes, 16-byte aligned (the transposed values);
- * nothing is kept in it between calls.  Two launches (plus the validation kernel). */
+ * nothing is kept in it between calls.  Two launches (plus the validation kernel); may be recorded
+ * by a stream capture. */
 size_t asap_attention_scratch_bytes(int32_t total_tokens, int32_t D);
 asap_status asap_attention(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                            const float *mask_log, const void *v, void *scratch, size_t scratch_bytes,
