@@ -12,7 +12,8 @@ text, keep 64).  One JSON line is printed by rank 0:
                  (config.timed_as; --no-graph times directly launched steps, which the line also
                  reports as direct_launch)
   e2e            the same with inputs in pinned host memory: every step copies them to the
-                 device, runs the step through the C ABI and reads the shortened batch back
+                 device, runs the step through the C ABI and reads the shortened batch back (the
+                 copies of neighbouring steps overlap: two sets of buffers, three streams)
   roofline       the kernel with the largest share of the step, against the measured peak
   kernels        per-kernel device time (CUDA events recorded by the library on its stream)
   cpu_baseline   the float64 CPU oracle timed on this host's cores on a few sequences
@@ -441,43 +442,72 @@ def run_cuda(args):
                                 "peak_kind": peak_kind + " (burst)"}
         del v_dev, a_out, a_scr
 
-    # ---- end to end from pinned host memory
+    # ---- end to end from pinned host memory: every step copies its inputs to the device, runs the
+    # step through the C ABI and reads the shortened batch back; the three legs run on streams of their
+    # own over two sets of buffers, so the copies of neighbouring steps overlap (PCIe is full duplex),
+    # and the host waits for a step's results before it lets the step two later reuse their buffers
     e2e = None
     if not args.no_e2e:
         host = {n: getattr(batch, n).contiguous().pin_memory() for n in ("q", "k", "hidden", "pos_ids")}
-        dev_in = copies[0]
         n_out_rows = batch.total - units + batch.B * keep_k
-        host_out = {"out_hidden": torch.empty(n_out_rows, batch.D, dtype=torch.bfloat16).pin_memory(),
-                    "out_pos": torch.empty(n_out_rows, dtype=torch.int32).pin_memory(),
-                    "out_cu_seqlens": torch.empty(batch.B + 1, dtype=torch.int32).pin_memory(),
-                    "keep_idx": torch.empty(batch.B, keep_k, dtype=torch.int32).pin_memory()}
+        dev_in = [copies[0], copies[1 % n_copies]]
+        dev_out = [out, A.alloc_outputs(copies[0], keep_k)]
+        host_out = [{"out_hidden": torch.empty(n_out_rows, batch.D, dtype=torch.bfloat16).pin_memory(),
+                     "out_pos": torch.empty(n_out_rows, dtype=torch.int32).pin_memory(),
+                     "out_cu_seqlens": torch.empty(batch.B + 1, dtype=torch.int32).pin_memory(),
+                     "keep_idx": torch.empty(batch.B, keep_k, dtype=torch.int32).pin_memory()} for _ in range(2)]
         h2d = sum(t.numel() * t.element_size() for t in host.values())
-        d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+        d2h = sum(t.numel() * t.element_size() for t in host_out[0].values())
+        s_in, s_out = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_run = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
 
-        def e2e_step():
-            for n, t in host.items():
-                getattr(dev_in, n).copy_(t, non_blocking=True)
-            A.asap_prune_step(ctx, dev_in, params, out, stream)
-            host_out["out_hidden"].copy_(out.out_hidden[:n_out_rows], non_blocking=True)
-            host_out["out_pos"].copy_(out.out_pos[:n_out_rows], non_blocking=True)
-            host_out["out_cu_seqlens"].copy_(out.out_cu_seqlens, non_blocking=True)
-            host_out["keep_idx"].copy_(out.keep_idx, non_blocking=True)
-            stream.synchronize()            # the caller consumes the shortened batch every step
+        def e2e_steps(n, first, last):
+            first.record(s_in)
+            for i in range(n):
+                j = i & 1
+                if i >= 2:
+                    ev_out[j].synchronize()          # the caller has step i - 2's results before its buffers go round
+                with torch.cuda.stream(s_in):
+                    if i >= 2:
+                        s_in.wait_event(ev_run[j])   # step i - 2 no longer reads these inputs
+                    for name, t in host.items():
+                        getattr(dev_in[j], name).copy_(t, non_blocking=True)
+                    ev_in[j].record(s_in)
+                stream.wait_event(ev_in[j])
+                A.asap_prune_step(ctx, dev_in[j], params, dev_out[j], stream)
+                ev_run[j].record(stream)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_run[j])
+                    o = dev_out[j]
+                    host_out[j]["out_hidden"].copy_(o.out_hidden[:n_out_rows], non_blocking=True)
+                    host_out[j]["out_pos"].copy_(o.out_pos[:n_out_rows], non_blocking=True)
+                    host_out[j]["out_cu_seqlens"].copy_(o.out_cu_seqlens, non_blocking=True)
+                    host_out[j]["keep_idx"].copy_(o.keep_idx, non_blocking=True)
+                    ev_out[j].record(s_out)
+            s_out.synchronize()
+            last.record(s_out)
+            last.synchronize()
 
-        e_steps = max(3, min(args.steps, 30))
-        for _ in range(3):
-            e2e_step()
+        e_steps = max(4, min(args.steps, 30))
+        w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e2e_steps(4, w0, w1)
         R.barrier(); torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(e_steps):
-            e2e_step()
-        e1.record(stream)
+        e2e_steps(e_steps, e0, e1)
         torch.cuda.synchronize(); R.barrier()
         e_ms = R.max_over_ranks(e0.elapsed_time(e1), device)
         e2e = {"value": units_all * e_steps / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": e_steps, "ms_per_step": e_ms / e_steps}
         A.asap_check(ctx)
+        # both buffer sets carried the same batch: what came back must agree with a directly run step
+        A.asap_prune_step(ctx, dev_in[0], params, out, stream)
+        torch.cuda.synchronize()
+        for j in range(2):
+            if not (torch.equal(host_out[j]["keep_idx"], out.keep_idx.cpu()) and
+                    torch.equal(host_out[j]["out_hidden"], out.out_hidden[:n_out_rows].cpu())):
+                raise RuntimeError("end-to-end leg: the results read back differ from a directly run step")
     A.asap_free(ctx)
 
     if rank != 0:
