@@ -414,6 +414,7 @@ constexpr int SELECT_THREADS = 1024;
 __device__ __forceinline__ uint32_t score_key(float f) {
   if (f != f) return 0u;                       // NaN ranks below everything
   uint32_t u = __float_as_uint(f);
+  if (f == 0.f) u = 0u;                        // -0.0 and +0.0 are one score: they tie, the lower index wins
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 

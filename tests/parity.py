@@ -9,8 +9,11 @@ Tolerances (written here so the bar is visible in one place):
                                similarity exceeds 1e-4; inside that band the GPU's slot is
                                accepted if its oracle similarity is within 1e-4 of the best
   best_sim                     |g - o| <= 2e-4
-  merged hidden (bf16)         |g - o_f64| <= max(2e-2, 2^-7 * |o|): 2e-2 absolute, widened to one
-                               bf16 ulp for large magnitudes (a single bf16 rounding is 2^-8 |o|)
+  merged hidden (bf16)         |g - o_f64| <= max(2e-2, (2^-8 + 2^-16) * |o|): 2e-2 absolute; for magnitudes
+                               above 5.1 the bound of ONE correct bf16 rounding (half a unit in the last
+                               place is at most 2^-8 |o|) plus 2^-16 |o| for the fp32 accumulation that
+                               precedes it.  How many elements needed the relative term, and their
+                               largest error, are recorded in `stats` (merged_wide_*)
   copied rows, position ids, row maps, offsets, index padding      bit-exact
 Where the GPU made an allowed in-band choice, the oracle's downstream stages are re-evaluated
 with that choice so that later comparisons stay meaningful.
@@ -27,6 +30,42 @@ from tests.helpers import bits
 
 REL = 1e-3
 TIE = 1e-4
+MERGED_ABS = 2e-2
+MERGED_REL = 2.0 ** -8 + 2.0 ** -16
+
+
+def merged_tolerance(want):
+    """Element-wise bar of a bf16 row computed in fp32 and rounded once, against float64."""
+    return np.maximum(MERGED_ABS, np.abs(want) * MERGED_REL)
+
+
+def check_invariants(batch, b, params, out):
+    """What must hold for every sequence whatever the scores are (no oracle involved): exactly k kept
+    indices, ascending; the dropped list is the ascending complement; the shortened sequence has the
+    right length; its row map is strictly increasing and names prefix rows, kept rows, suffix rows;
+    position ids are gathered through it; prefix and suffix rows are bit-identical copies."""
+    rows = batch.sample_rows(b)
+    v0, nv = int(batch.vis_start[b]), int(batch.vis_len[b])
+    n, k = rows.stop - rows.start, params.keep_k
+    keep = out.keep_idx[b].cpu().numpy()
+    drop = out.drop_idx[b].cpu().numpy()
+    assert keep.shape[0] == k and np.all(np.diff(keep) > 0) and keep[0] >= 0 and keep[-1] < nv, f"keep_idx sample {b}"
+    assert np.array_equal(drop[:nv - k], np.setdiff1d(np.arange(nv, dtype=np.int32), keep)), f"drop_idx sample {b}"
+    assert np.all(drop[nv - k:] == -1)
+    ocu = out.out_cu_seqlens.cpu().numpy()
+    lo, hi = int(ocu[b]), int(ocu[b + 1])
+    assert hi - lo == n - nv + k, f"out_cu_seqlens sample {b}"
+    src = out.src_row[lo:hi].cpu().numpy().astype(np.int64)
+    assert np.all(np.diff(src) > 0), f"src_row not strictly increasing (sample {b})"
+    want_src = np.concatenate([np.arange(v0), v0 + keep, np.arange(v0 + nv, n)]) + rows.start
+    assert np.array_equal(src, want_src), f"src_row sample {b}"
+    assert np.array_equal(out.out_pos[lo:hi].cpu().numpy(), batch.pos_ids.numpy()[src]), f"out_pos sample {b}"
+    oh = out.out_hidden[lo:hi]
+    hid = batch.hidden[rows]
+    assert torch.equal(oh[:v0].cpu(), hid[:v0]), f"prefix rows sample {b}"
+    assert torch.equal(oh[v0 + k:].cpu(), hid[v0 + nv:]), f"suffix rows sample {b}"
+    asg = out.assign[b].cpu().numpy()
+    assert np.all(asg[nv - k:] == -1) and np.all((asg[:nv - k] >= -1) & (asg[:nv - k] < k)), f"assign sample {b}"
 
 
 def _rel_err(g, o):
@@ -134,11 +173,17 @@ def compare_sample(batch, b, params, out, rank_start=None, rank_len=None, stats=
     assert np.array_equal(oh[v0 + k:], hb[v0 + nv:]), "suffix rows must be bit-identical"
     gh = O.bf16_bits_to_f64(oh[v0:v0 + k])
     want = ref["merged"]
-    tol = np.maximum(2e-2, np.abs(want) * 2.0 ** -7)
+    tol = merged_tolerance(want)
     err = np.abs(gh - want)
     assert np.all(err <= tol), f"merged hidden sample {b}: max err {err.max():.4e} (tol {tol.flat[err.argmax()]:.3e})"
     if stats is not None:
         stats["merged_abs"] = max(stats.get("merged_abs", 0.0), float(err.max()))
+        wide = err > MERGED_ABS                     # passed only because of the relative term
+        stats["merged_wide_count"] = stats.get("merged_wide_count", 0) + int(wide.sum())
+        if wide.any():
+            stats["merged_wide_max_abs"] = max(stats.get("merged_wide_max_abs", 0.0), float(err[wide].max()))
+            stats["merged_wide_max_rel"] = max(stats.get("merged_wide_max_rel", 0.0),
+                                               float((err[wide] / np.abs(want[wide])).max()))
     # rows that received nothing must be exact copies
     if params.merge_enable and nd > 0:
         untouched = np.setdiff1d(np.arange(k), as_g[as_g >= 0])

@@ -689,7 +689,62 @@ def test_per_head_step_with_identical_heads_is_the_default_step():
     assert np.allclose(a["mask_log_heads"], np.repeat(b["mask_log"][None], H, axis=0), rtol=1e-12, atol=1e-14)
 
 
+def check_hand_per_head_merge_weight(o):
+    """Two heads whose saliences differ: the Eq. 5 weight of a token is the head mean of the per-head
+    saliences -- not one head's salience and not the salience of the head-mean mass."""
+    g = GOLD["per_head_merge_weight"]
+    qb, kb, hb = _bf16_bits(g["Q"]), _bf16_bits(g["K"]), _bf16_bits(g["hidden"])
+    q, k = o.bf16_bits_to_f64(qb), o.bf16_bits_to_f64(kb)
+    assert np.allclose(o.attention_mass_heads(q, k, 0, 3), g["s_heads"], atol=1e-15)
+    r = o.prune_sample(qb, kb, hb, np.arange(4), 0, 3, 3, 1, 1, per_head=True)
+    assert np.allclose(r["salience"], g["salience"], rtol=1e-14, atol=0)
+    assert r["keep_idx"].tolist() == g["keep"] and r["assign"].tolist() == g["assign"]
+    assert np.allclose(r["merged"], g["merged"], rtol=1e-13, atol=0)
+
+
+def test_hand_per_head_merge_weight():
+    check_hand_per_head_merge_weight(O)
+
+
+PLANTED_PER_HEAD = [
+    ("merge weight taken from head 0", "s_hat = s_hat_heads.mean(axis=0)", "s_hat = s_hat_heads[0]"),
+    ("merge weight is the salience of the head-mean mass", "s_hat = s_hat_heads.mean(axis=0)", "s_hat = salience(s, eps)"),
+]
+
+
+@pytest.mark.parametrize("label,old,new", PLANTED_PER_HEAD, ids=[p[0] for p in PLANTED_PER_HEAD])
+def test_planted_slip_in_per_head_weight_is_caught(label, old, new):
+    src = open(O.__file__).read()
+    assert src.count(old) == 1
+    mod = types.ModuleType("mutant")
+    exec(compile(src.replace(old, new), "mutant", "exec"), mod.__dict__)
+    with pytest.raises(AssertionError):
+        check_hand_per_head_merge_weight(mod)
+    # the permutation test below must notice the first slip as well (head 0 is a different head after it)
+    if "heads[0]" in new:
+        with pytest.raises(AssertionError):
+            check_per_head_permutation(mod)
+
+
+def check_per_head_permutation(o):
+    rng = np.random.default_rng(43)
+    n, H, d, v0, nv = 36, 3, 8, 3, 25
+    qb, kb = _bf16_bits(rng.standard_normal((n, H, d))), _bf16_bits(rng.standard_normal((n, H, d)))
+    hb = _bf16_bits(rng.standard_normal((n, H * d)))
+    a = o.prune_sample(qb, kb, hb, np.arange(n), v0, nv, v0, n - v0, 8, per_head=True, lambda_max=0.9)
+    perm = [2, 0, 1]
+    b = o.prune_sample(qb[:, perm], kb[:, perm], hb, np.arange(n), v0, nv, v0, n - v0, 8, per_head=True, lambda_max=0.9)
+    assert np.allclose(b["mask_log_heads"], a["mask_log_heads"][perm], rtol=1e-13, atol=1e-14)
+    assert np.allclose(b["rank_score"], a["rank_score"], rtol=1e-12, atol=1e-15)
+    # one weight per token, whatever the order of the heads: salience and merged rows do not move
+    assert np.allclose(b["salience"], a["salience"], rtol=1e-13, atol=1e-15)
+    assert np.array_equal(b["keep_idx"], a["keep_idx"]) and np.array_equal(b["assign"], a["assign"])
+    assert np.array_equal(b["out_hidden_bits"], a["out_hidden_bits"])
+    return a, qb, kb, hb
+
+
 def test_per_head_masks_differ_and_follow_a_head_permutation():
+    check_per_head_permutation(O)
     rng = np.random.default_rng(43)
     n, H, d, v0, nv = 36, 3, 8, 3, 25
     qb, kb = _bf16_bits(rng.standard_normal((n, H, d))), _bf16_bits(rng.standard_normal((n, H, d)))

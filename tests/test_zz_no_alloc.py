@@ -23,6 +23,9 @@ def _scores(B, nvs, mv, seed, ties):
     for b in range(B):
         r = torch.randn(nvs[b], generator=g)
         s[b, :nvs[b]] = torch.round(r * 3) / 3 if ties else r     # ties exercise the lower-index rule
+    if ties:                      # -0.0 and +0.0 are one score: among them the lower index wins too
+        s[1, 0:40:2] = -0.0
+        s[1, 1:40:2] = 0.0
     return s.to(DEV)
 
 
