@@ -1,4 +1,5 @@
-"""Theoretical FLOPs of the LLM backbone attributable to the image tokens (App. A of the paper).
+"""Theoretical FLOPs of the LLM backbone attributable to the image tokens (App. A of the paper), and the
+key / value cache storage of a pruning schedule (Sec. 5.5, Table 4).
 
 Host-side accounting only; nothing here touches the GPU or the prune step.  One decoder layer
 that sees v image tokens costs 4 v d^2 + 2 v^2 d + 3 v d m (attention projections, attention
@@ -32,3 +33,18 @@ def single_prune_stages(total_layers: int, prune_layer: int, v0: int, keep: int)
     0 .. prune_layer see v0 image tokens, the rest see `keep`."""
     first = prune_layer + 1
     return [(first, v0), (total_layers - first, keep)]
+
+
+def kv_cache_bytes(stages: Sequence[Tuple[int, int]], d: int, bytes_per_element: int = 2) -> int:
+    """Key / value cache storage of a prefill (Sec. 5.5, Table 4, column "Storage"): every layer keeps
+    one key row and one value row of width d per token it saw.  `stages` lists (number of layers,
+    tokens of the whole sequence seen by those layers), as in schedule_flops."""
+    return sum(layers * tokens * 2 * d * bytes_per_element for layers, tokens in stages)
+
+
+def kv_storage_bytes(rows_before: int, rows_after: int, layers: int, d: int, bytes_per_element: int = 2) -> dict:
+    """What compacting the cached keys and values of `layers` layers from rows_before to rows_after
+    rows saves (the layers up to the pruning layer, which cached every token before the prune step)."""
+    before = kv_cache_bytes([(layers, rows_before)], d, bytes_per_element)
+    after = kv_cache_bytes([(layers, rows_after)], d, bytes_per_element)
+    return {"layers": layers, "bytes_before": before, "bytes_after": after, "bytes_saved": before - after}

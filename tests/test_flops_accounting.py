@@ -34,3 +34,23 @@ def test_schedule_and_ratio():
     assert F.layer_flops(192, d, m) / F.layer_flops(576, d, m) < r < 1.0
     # the quadratic term: halving the tokens more than halves the attention part
     assert F.layer_flops(288, d, m) * 2 < F.layer_flops(576, d, m)
+
+
+@pytest.mark.parametrize("row", GOLD["kv_storage"]["rows"], ids=lambda r: f"{r['tokens']} tokens")
+def test_printed_kv_storage_is_reproduced(row):
+    g = GOLD["kv_storage"]
+    got = F.kv_cache_bytes([(g["layers"], row["tokens"])], g["d"], g["bytes_per_element"]) / 1e6
+    assert abs(got - row["mb"]) < 5e-3, (got, row)
+
+
+def test_kv_storage_of_a_schedule_and_of_a_compaction():
+    g = GOLD["kv_storage"]
+    d, L = g["d"], g["layers"]
+    per_token_layer = 2 * d * 2
+    stages = [(3, 613), (29, 229)]                      # prune 576 -> 192 image tokens after layer index 2
+    assert F.kv_cache_bytes(stages, d) == (3 * 613 + 29 * 229) * per_token_layer
+    # no single prune after an integer layer gives the pruned rows the paper prints (see the fixture)
+    singles = [F.kv_cache_bytes([(k, 613), (L - k, 229)], d) / 1e6 for k in range(L + 1)]
+    assert all(min(abs(s - mb) for s in singles) > 0.5 for mb in g["not_reproduced_mb"][:2])
+    s = F.kv_storage_bytes(613, 229, 3, d)
+    assert s["bytes_before"] - s["bytes_after"] == s["bytes_saved"] == 3 * (613 - 229) * per_token_layer

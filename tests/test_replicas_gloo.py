@@ -76,3 +76,17 @@ def test_shards_partition_the_batch(n, w):
 def test_aggregate_throughput_uses_the_slowest_rank():
     assert R.aggregate_throughput([100, 100], [1.0, 2.0]) == 100.0
     assert R.aggregate_throughput([9216] * 8, [0.001] * 8) == pytest.approx(8 * 9216 / 0.001)
+
+
+def test_bench_spawns_its_own_ranks_without_a_launcher():
+    """`bench.py --gpus 2` started with no launcher environment starts the two ranks itself; here they
+    run the host-only rendezvous check over gloo (join, barrier, the two reductions of the benchmark)."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "rendezvous-check"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, res.stdout                       # rank 0 alone prints
+    got = json.loads(lines[0])
+    assert got == {"impl": "rendezvous-check", "n_gpus": 2, "slowest": 2.0, "total": 200.0}
