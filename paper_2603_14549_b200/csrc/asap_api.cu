@@ -299,7 +299,8 @@ asap_status launch_select(asap_ctx *ctx, const asap_inputs *in, const asap_param
 
 // Step 4a: kept rows gathered, cosine similarity and assignment, CSR of the assignment.
 asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
-                               const int32_t *keep_idx, const asap_outputs *out, cudaStream_t st) {
+                               const int32_t *keep_idx, const int32_t *drop_idx, const asap_outputs *out,
+                               cudaStream_t st) {
   const int B = in->B, D = in->D, k = p->keep_k;
   if (merging(in, p)) {
     mark(ctx, "kept_gather", st);
@@ -307,13 +308,12 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
         static_cast<const __nv_bfloat16 *>(in->hidden), ctx->desc, D, k, keep_idx, ctx->kept_rows, ctx->kept_inv);
     ASAP_TRY(after_launch(ctx, "kept_gather"));
 
-    const int n_nt = (k + 255) / 256;
-    const int n_tile = (((k + n_nt - 1) / n_nt) + 15) & ~15;
-    const int stage_bytes = 2 * (SIM_A_BYTES + n_tile * 128);   // two adjacent 64-column blocks per stage
+    int n_nt = (k + 255) / 256;
+    int n_tile = (((k + n_nt - 1) / n_nt) + 15) & ~15;
     // Small problems leave most SMs without a row tile: slice the hidden dimension over several
     // blocks (at most 8, a divisor of the number of 128-column steps, scratch permitting), up to
     // two blocks per SM.
-    const int max_mt = (in->max_vis + 127) / 128;
+    const int max_mt = (in->max_vis - k + 127) / 128;    // row tiles of 128 dropped tokens
     const int n_kb = D / 128;
     // The slice count minimises a simple cost: streaming a row tile takes about 1 us per 128-column
     // step of the slice, and the last slice adds up keep_k * slices partial values per row at about
@@ -335,11 +335,28 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     // block of the rows and of every slot tile).
     // Taken only while three such stages still fit (up to 384 slots): with two, the shorter copies
     // cost more than the second read of the rows (measured: 320 slots 87 -> 77 us, 510 slots 91 -> 96 us).
-    const bool wide = n_nt >= 2 && n_nt * n_tile <= 512 && 3 * (SIM_A_BYTES + n_nt * n_tile * 128) <= 192 * 1024;
+    bool wide = n_nt >= 2 && n_nt * n_tile <= 512 && 3 * (SIM_A_BYTES + n_nt * n_tile * 128) <= 192 * 1024;
+    // More slots than that, and enough row tiles that the hidden dimension is not sliced: the slot tiles are
+    // dealt to several blocks per row tile (groups of at most 384 slots = one or two tiles), each a single
+    // pass in the layout above; the last block of a row tile combines the groups' best slots.  Several
+    // passes inside one block would read the dropped rows from memory once per pass: the rows that all
+    // resident blocks hold between two passes do not fit L2.
+    int groups = 1;
+    if (!wide && n_nt >= 2 && splits == 1 && D % 64 == 0 && (size_t)B * max_mt <= ctx->cap_tiles) {
+      int g = (k + 383) / 384;
+      const int per_group = (k + g - 1) / g;
+      const int tiles_g = per_group > 256 ? 2 : 1;
+      const int tile_g = (((per_group + tiles_g - 1) / tiles_g) + 15) & ~15;
+      g = (k + tiles_g * tile_g - 1) / (tiles_g * tile_g);
+      if ((size_t)B * max_mt * g * 256 * sizeof(float) <= ctx->sim_part_bytes) {
+        groups = g; n_nt = tiles_g; n_tile = tile_g; wide = true;
+      }
+    }
+    const int stage_bytes = 2 * (SIM_A_BYTES + n_tile * 128);   // two adjacent 64-column blocks per stage
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < (wide ? n_nt * n_tile : 2 * n_tile)) tmem_cols <<= 1;
     const int stage_bytes_used = wide ? SIM_A_BYTES + n_nt * n_tile * 128 : stage_bytes;
-    const long long ctas = (long long)max_mt * B * splits;
+    const long long ctas = (long long)max_mt * B * splits * groups;
     const bool two_per_sm = !wide && ctas > ctx->num_sms && ctas <= 2LL * ctx->num_sms && tmem_cols <= 256 &&
                             2 * stage_bytes <= 96 * 1024;
     // at most 192 KB of tiles: the block then fits the 196 KB shared-memory carve-out, which leaves
@@ -350,6 +367,7 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     if ((size_t)(SIM_THREADS / 32 + 1) * k * sizeof(int) > (size_t)stages * stage_bytes_used)
       return fail(ctx, ASAP_ERR_UNSUPPORTED, "keep_k = %d is too large for the merge path", k);
     CUtensorMap map_h, map_kept;
+    // (the row operand is gathered by ordinary asynchronous copies; the map of `hidden` is only prefetched)
     if (!make_map(ctx, &map_h, in->hidden, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
         !make_map(ctx, &map_kept, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, (uint32_t)n_tile))
       return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for hidden / kept rows");
@@ -357,15 +375,16 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = n_tile;
     sa.n_nt = n_nt; sa.stages = stages; sa.splits = splits; sa.max_mt = max_mt; sa.tmem_cols = tmem_cols;
     sa.wide = wide ? 1 : 0;
+    sa.groups = groups;
     sa.threshold = p->sim_threshold;
-    sa.role = ctx->role; sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
+    sa.drop_idx = drop_idx; sa.hidden = static_cast<const __nv_bfloat16 *>(in->hidden); sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
     sa.best_sim = out->best_sim; sa.seg = ctx->seg; sa.members = ctx->members; sa.counters = ctx->cnt_sim;
     sa.tile_counters = ctx->cnt_tiles; sa.part = ctx->sim_part;
     sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
     sa.smat = nullptr;
     sa.status = ctx->status;
     mark(ctx, "sim", st);
-    launch_pdl(sim_kernel, dim3(dim3(max_mt, B, splits)), dim3(SIM_THREADS), smem, st, map_h, map_kept, sa);
+    launch_pdl(sim_kernel, dim3(dim3(max_mt * groups, B, splits)), dim3(SIM_THREADS), smem, st, map_h, map_kept, sa);
     ASAP_TRY(after_launch(ctx, "sim"));
   }
   return ASAP_OK;
@@ -399,7 +418,7 @@ asap_status launch_merge_back(asap_ctx *ctx, const asap_inputs *in, const asap_p
 asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                          const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
                          const asap_outputs *out, cudaStream_t st) {
-  ASAP_TRY(launch_merge_front(ctx, in, p, keep_idx, out, st));
+  ASAP_TRY(launch_merge_front(ctx, in, p, keep_idx, drop_idx, out, st));
   return launch_merge_back(ctx, in, p, salience, keep_idx, drop_idx, out, st);
 }
 
@@ -450,8 +469,9 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = n_tile;
   sa.n_nt = n_nt; sa.stages = stages; sa.splits = splits; sa.max_mt = max_mt; sa.tmem_cols = tmem_cols;
   sa.wide = 0;
+  sa.groups = 1;
   sa.threshold = p->sim_threshold;
-  sa.role = ctx->role; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
+  sa.drop_idx = nullptr; sa.hidden = nullptr; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
   sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr; sa.tile_counters = ctx->cnt_tiles;
   sa.part = ctx->sim_part; sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
   sa.smat = smat; sa.status = ctx->status;
@@ -724,7 +744,7 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
   if (main_status == ASAP_OK && cudaStreamWaitEvent(st, ctx->ev_desc, 0) != cudaSuccess)
     main_status = fail(ctx, ASAP_ERR_CUDA, "wait for the descriptors");
   if (main_status == ASAP_OK) main_status = launch_select(ctx, in, p, out->rank_score, out, true, true, st);
-  if (main_status == ASAP_OK) main_status = launch_merge_front(ctx, in, p, out->keep_idx, out, st);
+  if (main_status == ASAP_OK) main_status = launch_merge_front(ctx, in, p, out->keep_idx, out->drop_idx, out, st);
   // the side stream always rejoins, also after an error, so that `stream` stays ordered behind it
   e = cudaStreamWaitEvent(st, ctx->ev_join, 0);
   if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "join with the side stream: %s", cudaGetErrorString(e));

@@ -150,6 +150,24 @@ __device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const void *tmap,
       ::"r"(smem_dst), "l"(tmap), "r"(bar), "r"(x), "r"(y)
       : "memory");
 }
+// Asynchronous 16-byte copies global -> shared issued by ordinary threads (used where the rows of a
+// tile are scattered and no tiled copy describes them).  They complete in groups; after
+// cp_async_wait<N>() all but the N most recent groups of the calling thread have landed.  Their
+// writes belong to the generic proxy: the thread that issues the MMAs runs fence_proxy_async() after it
+// has seen the copies' barrier complete and before it issues the MMAs that read the data.
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void *src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+// The mbarrier gets one arrival from this thread once all its earlier cp_async16 copies have landed
+// (the arrival is counted against the barrier's expected count; it does not block the thread).
+__device__ __forceinline__ void cp_async_arrive_on(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const void *tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }

@@ -471,11 +471,15 @@ head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
 // =======================================================================================
 // sim_kernel
 //
-// One block per (128 visual rows, sample, slice of the hidden dimension).  D = V_tile Kept^T
-// with M = 128 visual rows, N = n_tile kept slots per accumulator, K = this block's slice of
-// the hidden size in steps of 64.  While the first accumulator is being built the epilogue
-// warps also read every row tile from shared memory and add up the squares (the row norms of
-// Sec. 4.2's cosine similarity), so the visual rows are read from memory once.
+// One block per (128 dropped rows, sample, slice of the hidden dimension).  D = Drop_tile Kept^T
+// with M = 128 dropped rows, N = n_tile kept slots per accumulator, K = this block's slice of
+// the hidden size in steps of 64.  The dropped rows are fetched where they lie in `hidden` by four
+// gather warps (16-byte asynchronous copies, written in the 128-byte-swizzled layout the tiled
+// copies produce; a gather copy of four rows per instruction through the tensor-map unit was
+// measured at one instruction per ~74 clk and SM, a tenth of what the tile needs), so only rows
+// whose result is used are multiplied.  While the first
+// accumulator is being built the epilogue warps also read every row tile from shared memory and
+// add up the squares (the row norms of Sec. 4.2's cosine similarity).
 //   one slice:      the epilogue scales column s by 1/||kept_s||, keeps the running maximum
 //                   and the first slot attaining it, and writes, for rows that were dropped,
 //                   the slot (or -1 if the cosine similarity is not above the threshold) and
@@ -483,18 +487,28 @@ head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
 //   several slices: (small problems, to fill the machine) every block stores its partial dot
 //                   products and partial squared norms; the block that finishes last for the
 //                   row tile adds the slices in slice order and does the same epilogue.
-// Rows that were kept, or lie past the image span, are computed but not written.
-// The block that finishes a sample's last row tile groups the dropped tokens by destination.
+// Rows past the last dropped token (the ragged tail of the last tile) repeat that token and are
+// not written.  The block that finishes a sample's last row tile groups the dropped tokens by
+// destination.
 //   one pass:       (a.wide, when all kept slots fit the 512 tensor-memory columns) the accumulators of
 //                   all slot tiles are live at once and a stage is one 64-column block of the rows
 //                   plus the matching block of EVERY slot tile, so the visual rows are read from
 //                   memory once instead of once per slot tile.
+//   slot groups:    (a.groups > 1, one-pass layout, blockIdx.x = row tile * groups + group) more kept slots than tensor memory
+//                   holds at once: every block takes one group of slot tiles in ONE pass over the hidden
+//                   dimension and publishes its rows' best (value, slot); the block that finishes a row
+//                   tile last takes the maximum over the groups (lowest slot among equals).  The blocks
+//                   of a row tile are neighbours in launch order and stream the same rows at the same
+//                   time, so the rows come from memory once and from L2 afterwards -- several passes in
+//                   one block read them from memory every time, because the rows of all resident
+//                   blocks together do not fit L2.
 //   matrix mode:    (a.smat set) the row operand is the dense kept-row array too, and
 //                   the epilogue writes the whole keep_k x keep_k cosine matrix of the sample,
 //                   S[p][q] = <h_p, h_q> * (1/||h_p|| * 1/||h_q||), for the routing inside the
-//                   kept set; `tmap_h` is then a map of the kept rows with a 128-row box.
+//                   kept set; `tmap_h` is then a map of the kept rows with a 128-row box (plain
+//                   tiled copies, no gather).
 // =======================================================================================
-constexpr int SIM_THREADS = 192;
+constexpr int SIM_THREADS = 320;            // copy warp, MMA warp, four epilogue warps, four gather warps
 constexpr int SIM_A_BYTES = 128 * 128;           // 128 rows x 64 bf16
 constexpr int SIM_BOOK_BYTES = 2048;
 constexpr uint32_t SIM_TMEM_COLS = 512;
@@ -504,9 +518,11 @@ struct SimArgs {
   const SampleDesc *desc;
   int D, max_vis, keep_k, n_tile, n_nt, stages, splits, max_mt;
   int wide;                  // 1: one pass, all slot tiles' accumulators live at once
+  int groups;                // > 1: slot tiles dealt to `groups` blocks per row tile (n_nt counts one group's tiles)
   uint32_t tmem_cols;        // power of two >= 2 * n_tile: two accumulators
   float threshold;
-  const int32_t *role;       // [B, max_vis]
+  const int32_t *drop_idx;   // [B, max_vis-keep_k] dropped tokens, ascending (row operand of the main mode)
+  const __nv_bfloat16 *hidden;   // [tokens, D] (main mode: the gather warps read the dropped rows from here)
   const float *kept_inv;     // [B*keep_k]   1/||kept row||, 0 for a zero row
   int32_t *assign;           // [B, max_vis-keep_k]
   float *best_sim;           // [B, max_vis-keep_k] or nullptr
@@ -539,9 +555,16 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
            SimArgs a) {
   pdl_enter();
   extern __shared__ uint8_t smem_raw[];
-  const int mt = blockIdx.x, b = blockIdx.y, z = blockIdx.z;
+  // the groups of a row tile are neighbours in launch order (blockIdx.x = row tile * groups + group)
+  const int mt = blockIdx.x / a.groups, b = blockIdx.y;
+  const int z = blockIdx.z;                              // slice of the hidden dimension
+  const int gz = blockIdx.x - mt * a.groups;             // group of slot tiles
+  const int tile0 = gz * a.n_nt;                         // first slot tile of this block
   const SampleDesc d = a.desc[b];
-  if (!d.valid || mt * 128 >= (a.smat ? a.keep_k : d.nv)) return;
+  if (!d.valid) return;
+  const int nd = d.nv - a.keep_k;                        // dropped tokens of this sample
+  const int n_rows = a.smat ? a.keep_k : nd;             // rows of the row operand
+  if (mt * 128 >= max(n_rows, 1)) return;
   if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SIM_TIMEOUT) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -552,10 +575,15 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   const int b_bytes = a.n_tile * 128;
   const int stage_bytes = a.wide ? SIM_A_BYTES + a.n_nt * b_bytes : 2 * (SIM_A_BYTES + b_bytes);
   SimBook *bk = reinterpret_cast<SimBook *>(base_ptr + (size_t)a.stages * stage_bytes);
+  if (n_rows <= 0) {
+    // nothing was dropped in this sample: only the (empty) grouping has to be written
+    if (z == 0 && gz == 0) csr_block(d, b, a.max_vis, a.keep_k, a.assign, a.seg, a.members, reinterpret_cast<int *>(base_ptr), bk->scan);
+    return;
+  }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.stages; ++s) {
-      mbar_init(smem_u32(&bk->full[s]), 1);
+      mbar_init(smem_u32(&bk->full[s]), a.smat ? 1 : 129);  // the copy warp's announcement (+ every gather thread)
       mbar_init(smem_u32(&bk->empty[s]), 5);      // the MMAs that read the stage + four epilogue warps
     }
     for (int i = 0; i < 2; ++i) {
@@ -581,34 +609,37 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   const int total_it = a.wide ? n_kb : a.n_nt * n_kb;
 
   if (warp == 0) {
+    // ---- copy warp: the kept-row tiles (and, in matrix mode, the row operand) by tiled copies
     if (lane == 0) {
       tma_prefetch_desc(&tmap_h);
       tma_prefetch_desc(&tmap_kept);
+      const bool gather = a.smat == nullptr;
       const int row_b = b * a.keep_k;
-      const int row_a = a.smat ? row_b + mt * 128 : d.row0 + d.v0 + mt * 128;
+      const int row_a = row_b + mt * 128;                // matrix mode: rows of the dense kept array
+      const int tx_bytes = gather ? stage_bytes - (a.wide ? 1 : 2) * SIM_A_BYTES : stage_bytes;
       const int rot = (mt * 5 + b * 3) % n_kb;
       int issued = 0;
       for (int it = 0; it < total_it; ++it) {
         // every block walks its k-blocks from a different starting point, so that at any moment
         // the blocks read different 128-byte columns of the rows and spread over the memory channels
         const int s = it % a.stages, nt = it / n_kb, kb = kb0 + (it - nt * n_kb + rot) % n_kb;
+        const uint32_t full = smem_u32(&bk->full[s]);
         if (it >= a.stages) mbar_wait(smem_u32(&bk->empty[s]), ((it / a.stages) - 1) & 1, wc);
         if (bk->abort_flag) break;
         const uint32_t dst = base + s * stage_bytes;
-        mbar_expect_tx(smem_u32(&bk->full[s]), stage_bytes);
+        mbar_expect_tx(full, tx_bytes);
         if (a.wide) {
-          tma_load_2d(dst, &tmap_h, smem_u32(&bk->full[s]), kb * 64, row_a);
+          if (!gather) tma_load_2d(dst, &tmap_h, full, kb * 64, row_a);
           for (int t = 0; t < a.n_nt; ++t)
-            tma_load_2d(dst + SIM_A_BYTES + t * b_bytes, &tmap_kept, smem_u32(&bk->full[s]), kb * 64,
-                        row_b + t * a.n_tile);
-          issued = it + 1;
-          continue;
+            tma_load_2d(dst + SIM_A_BYTES + t * b_bytes, &tmap_kept, full, kb * 64, row_b + (tile0 + t) * a.n_tile);
+        } else {
+          if (!gather) {
+            tma_load_2d(dst, &tmap_h, full, kb * 128, row_a);
+            tma_load_2d(dst + SIM_A_BYTES, &tmap_h, full, kb * 128 + 64, row_a);
+          }
+          tma_load_2d(dst + 2 * SIM_A_BYTES, &tmap_kept, full, kb * 128, row_b + nt * a.n_tile);
+          tma_load_2d(dst + 2 * SIM_A_BYTES + b_bytes, &tmap_kept, full, kb * 128 + 64, row_b + nt * a.n_tile);
         }
-        tma_load_2d(dst, &tmap_h, smem_u32(&bk->full[s]), kb * 128, row_a);
-        tma_load_2d(dst + SIM_A_BYTES, &tmap_h, smem_u32(&bk->full[s]), kb * 128 + 64, row_a);
-        tma_load_2d(dst + 2 * SIM_A_BYTES, &tmap_kept, smem_u32(&bk->full[s]), kb * 128, row_b + nt * a.n_tile);
-        tma_load_2d(dst + 2 * SIM_A_BYTES + b_bytes, &tmap_kept, smem_u32(&bk->full[s]), kb * 128 + 64,
-                    row_b + nt * a.n_tile);
         issued = it + 1;
       }
       // drain: the last fill of every stage must have landed before the block leaves
@@ -619,6 +650,51 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         }
       }
     }
+  } else if (warp >= 6) {
+    // ---- gather warps (main mode): warp g fetches rows 32 g .. 32 g + 31 of the tile, i.e. the hidden
+    // rows of 32 dropped tokens, one stage's columns at a time.  A warp instruction covers whole rows
+    // (2 rows x 256 bytes, or 4 rows x 128 bytes in the one-pass layout), each lane one 16-byte chunk,
+    // written where the tiled copies would put it: row r of a 64-column block is 128 bytes at
+    // r * 128, its chunk c at position c ^ (r & 7).  Every lane's copies of a stage arrive on the stage's
+    // barrier by themselves when they have landed, so the warps only ever wait for a free stage.
+    if (a.smat == nullptr) {
+      const int g = warp - 6;
+      const int cpr = a.wide ? 8 : 16;                   // 16-byte chunks per row and stage
+      const int c = lane & (cpr - 1), rsub = lane / cpr, rpi = 32 / cpr, n_i = 32 / rpi;
+      const int32_t *drop_b = a.drop_idx + (size_t)b * (a.max_vis - a.keep_k);
+      const uint8_t *hid = reinterpret_cast<const uint8_t *>(a.hidden);
+      const size_t pitch = (size_t)a.D * 2;
+      size_t src_off[16];
+      uint32_t dst_off[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int r = g * 32 + (i < n_i ? i : 0) * rpi + rsub;
+        const int dp = min(mt * 128 + r, nd - 1);        // the ragged tail repeats the last dropped token
+        const int row = d.row0 + d.v0 + min(max(__ldg(drop_b + dp), 0), d.nv - 1);
+        src_off[i] = (size_t)row * pitch + (size_t)c * 16;
+        dst_off[i] = (uint32_t)((c >> 3) * SIM_A_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+      }
+      const int stage_cols_bytes = a.wide ? 128 : 256;
+      const int rot = (mt * 5 + b * 3) % n_kb;
+      for (int it = 0; it < total_it; ++it) {
+        const int s = it % a.stages, nt = it / n_kb, kb = kb0 + (it - nt * n_kb + rot) % n_kb;
+        int go = 1;
+        if (lane == 0) {
+          if (it >= a.stages) mbar_wait(smem_u32(&bk->empty[s]), ((it / a.stages) - 1) & 1, wc);
+          go = bk->abort_flag ? 0 : 1;
+        }
+        go = __shfl_sync(0xffffffffu, go, 0);
+        if (!go) break;
+        const uint32_t dst = base + s * stage_bytes;
+        const uint8_t *src = hid + (size_t)kb * stage_cols_bytes;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          if (i < n_i) cp_async16(dst + dst_off[i], src + src_off[i]);
+        cp_async_arrive_on(smem_u32(&bk->full[s]));       // this lane's share of the stage, once it has landed
+      }
+      cp_async_commit();
+      cp_async_wait<0>();                                 // nothing of this thread's is in flight when the block leaves
+    }
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_bf16(128, a.n_tile);
@@ -627,6 +703,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         for (int kb = 0; kb < n_kb; ++kb) {
           const int s = kb % a.stages;
           mbar_wait(smem_u32(&bk->full[s]), (kb / a.stages) & 1, wc);
+          fence_proxy_async();       // the gathered rows were written by ordinary asynchronous copies
           tc_fence_after();
           if (!bk->abort_flag) {
             const uint32_t sa = base + s * stage_bytes, sb = sa + SIM_A_BYTES;
@@ -648,6 +725,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const int s = it % a.stages;
           mbar_wait(smem_u32(&bk->full[s]), (it / a.stages) & 1, wc);
+          fence_proxy_async();
           tc_fence_after();
           if (!bk->abort_flag) {
             const uint32_t sa = base + s * stage_bytes, sb = sa + 2 * SIM_A_BYTES;
@@ -667,7 +745,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   } else {
     const int quarter = warp & 3;
     const int lrow = quarter * 32 + lane;
-    const int v = mt * 128 + lrow;                       // visual index of this thread's row
+    const int v = mt * 128 + lrow;                       // this thread's row: dropped position (kept slot in matrix mode)
     const float *kinv = a.kept_inv + (size_t)b * a.keep_k;
     // ---- squared norm of this thread's row, from the row tiles of the first accumulator's pass.
     // Row r of a tile is 128 bytes; its 16-byte chunk c sits at chunk position c ^ (r & 7).
@@ -710,8 +788,8 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) +
                              (a.wide ? nt * a.n_tile : buf * (a.tmem_cols >> 1));
-      const int slot0 = nt * a.n_tile;
-      const int ncol = min(a.n_tile, a.keep_k - slot0);   // kept slots in this accumulator
+      const int slot0 = (tile0 + nt) * a.n_tile;
+      const int ncol = min(a.n_tile, a.keep_k - slot0);   // kept slots in this accumulator (none in a group's ragged end)
 #pragma unroll 1
       for (int c = 0; c < ncol; c += 16) {
         uint32_t r[16];
@@ -803,18 +881,40 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         }
       }
     }
-    if (a.smat) finalize = false;
-    if (finalize && v < d.nv && !bk->abort_flag) {
-      const int role = a.role[(size_t)b * a.max_vis + v];
-      if (role < 0) {
-        const int dp = -role - 1;
-        const bool zero_row = !(ss_tot >= 1e-24f);      // ||h|| < 1e-12: similarity 0 to every slot
-        const float sim = zero_row ? 0.f : best * rsqrtf(ss_tot);
-        const int slot = zero_row ? 0 : best_slot;
-        const size_t o = (size_t)b * (a.max_vis - a.keep_k) + dp;
-        a.assign[o] = (sim > a.threshold) ? slot : -1;
-        if (a.best_sim) a.best_sim[o] = sim;
+    if (a.groups > 1) {
+      // publish this group's best (value, slot); the last group to arrive for the row tile combines them
+      const size_t tile = ((size_t)b * a.max_mt + mt) * a.groups;
+      a.part[(tile + gz) * 256 + lrow] = best;
+      reinterpret_cast<int *>(a.part)[(tile + gz) * 256 + 128 + lrow] = best_slot;
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (warp == 2 && lane == 0) {
+        unsigned int *cnt = a.tile_counters + (size_t)b * a.max_mt + mt;
+        const unsigned int old = atomicAdd(cnt, 1u);
+        bk->is_last = (old == (unsigned int)(a.groups - 1));
+        if (bk->is_last) *cnt = 0u;
       }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      finalize = bk->is_last != 0;
+      if (finalize) {
+        __threadfence();
+        best = -INFINITY;
+        best_slot = 0;
+        for (int g2 = 0; g2 < a.groups; ++g2) {           // ascending slots: the first maximum stays
+          const float val = __ldcg(a.part + (tile + g2) * 256 + lrow);
+          const int slot = __ldcg(reinterpret_cast<const int *>(a.part) + (tile + g2) * 256 + 128 + lrow);
+          if (val > best) { best = val; best_slot = slot; }
+        }
+      }
+    }
+    if (a.smat) finalize = false;
+    if (finalize && v < nd && !bk->abort_flag) {
+      const bool zero_row = !(ss_tot >= 1e-24f);        // ||h|| < 1e-12: similarity 0 to every slot
+      const float sim = zero_row ? 0.f : best * rsqrtf(ss_tot);
+      const int slot = zero_row ? 0 : best_slot;
+      const size_t o = (size_t)b * (a.max_vis - a.keep_k) + v;
+      a.assign[o] = (sim > a.threshold) ? slot : -1;
+      if (a.best_sim) a.best_sim[o] = sim;
     }
     if (warp == 2 && lane == 0) bk->is_last = finalize ? 1 : 0;
     __threadfence();
@@ -826,12 +926,12 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     tmem_dealloc(tmem_base, a.tmem_cols);
   }
   if (a.smat) return;
-  if (!bk->is_last && a.splits > 1) return;     // a slice that did not finalize its row tile
+  if (!bk->is_last && (a.splits > 1 || a.groups > 1)) return;     // a slice / group that did not finalize its row tile
   __syncthreads();
   // the block that finishes the sample's last row tile groups the dropped tokens by destination
   if (threadIdx.x == 0) {
     __threadfence();
-    const unsigned int n_mt = (unsigned int)((d.nv + 127) / 128);
+    const unsigned int n_mt = (unsigned int)((nd + 127) / 128);
     const unsigned int old = atomicAdd(a.counters + b, 1u);
     bk->is_last = (old == n_mt - 1u);
     if (bk->is_last) a.counters[b] = 0u;

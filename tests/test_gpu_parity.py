@@ -104,6 +104,16 @@ def test_identity_when_k_equals_visual_count(ctx):
     assert torch.equal(out.out_pos.cpu(), batch.pos_ids)
 
 
+def test_one_sequence_keeps_everything_while_another_merges(ctx):
+    """keep_k equals the first sequence's visual count (nothing dropped there, its rows are copies) while
+    the second one drops and merges 80 tokens."""
+    batch = W.tiny(B=2, n_vis=[150, 230], text_lens=[9, 21], H=2, keep_k=150, seed=109, centres=9)
+    inp, out = run_step(ctx, batch, A.Params(keep_k=150))
+    n0 = int(batch.cu_seqlens[1])
+    assert torch.equal(out.out_hidden[:n0].cpu(), batch.hidden[:n0])
+    assert int((out.assign[0] >= 0).sum()) == 0 and int((out.assign[1] >= 0).sum()) == 80
+
+
 def test_mask_off_merge_off_is_plain_topk_gather(ctx):
     batch = W.tiny(B=2, n_vis=[190, 133], text_lens=[12, 31], H=2, keep_k=24, seed=106)
     inp, out = run_step(ctx, batch, A.Params(keep_k=24, mask_enable=False, merge_enable=False))
