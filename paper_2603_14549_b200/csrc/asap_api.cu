@@ -313,7 +313,7 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     // Small problems leave most SMs without a row tile: slice the hidden dimension over several
     // blocks (at most 8, a divisor of the number of 128-column steps, scratch permitting), up to
     // two blocks per SM.
-    const int max_mt = (in->max_vis - k + 127) / 128;    // row tiles of 128 dropped tokens
+    int max_mt = (in->max_vis + 127) / 128;              // row tiles when every visual row is multiplied
     const int n_kb = D / 128;
     // The slice count minimises a simple cost: streaming a row tile takes about 1 us per 128-column
     // step of the slice, and the last slice adds up keep_k * slices partial values per row at about
@@ -335,6 +335,12 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     // block of the rows and of every slot tile).
     // Taken only while three such stages still fit (up to 384 slots): with two, the shorter copies
     // cost more than the second read of the rows (measured: 320 slots 87 -> 77 us, 510 slots 91 -> 96 us).
+    // The row operand: every visual row by tiled copies (a fifth to a half of the products are then thrown
+    // away), or the dropped rows alone, gathered (half the bytes per clock, four more warps, one block per
+    // SM).  Gathering is taken for batches large enough not to be sliced, from a fifth of the rows kept.
+    const bool gather_rows = splits == 1 && (long long)k * 5 >= (long long)in->max_vis &&
+                             (long long)max_mt * B > ctx->num_sms;
+    if (gather_rows) max_mt = (in->max_vis - k + 127) / 128;
     bool wide = n_nt >= 2 && n_nt * n_tile <= 512 && 3 * (SIM_A_BYTES + n_nt * n_tile * 128) <= 192 * 1024;
     // More slots than that, and enough row tiles that the hidden dimension is not sliced: the slot tiles are
     // dealt to several blocks per row tile (groups of at most 384 slots = one or two tiles), each a single
@@ -342,7 +348,7 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     // passes inside one block would read the dropped rows from memory once per pass: the rows that all
     // resident blocks hold between two passes do not fit L2.
     int groups = 1;
-    if (!wide && n_nt >= 2 && splits == 1 && D % 64 == 0 && (size_t)B * max_mt <= ctx->cap_tiles) {
+    if (gather_rows && !wide && n_nt >= 2 && D % 64 == 0 && (size_t)B * max_mt <= ctx->cap_tiles) {
       int g = (k + 383) / 384;
       const int per_group = (k + g - 1) / g;
       const int tiles_g = per_group > 256 ? 2 : 1;
@@ -364,10 +370,10 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     int stages = ((two_per_sm ? 96 : 192) * 1024) / stage_bytes_used;
     if (stages > SIM_MAX_STAGES) stages = SIM_MAX_STAGES;
     const size_t smem = (size_t)stages * stage_bytes_used + SIM_BOOK_BYTES + 1024;
-    if ((size_t)(SIM_THREADS / 32 + 1) * k * sizeof(int) > (size_t)stages * stage_bytes_used)
+    const int sim_threads = gather_rows ? SIM_THREADS : SIM_THREADS_TILED;
+    if ((size_t)(sim_threads / 32 + 1) * k * sizeof(int) > (size_t)stages * stage_bytes_used)
       return fail(ctx, ASAP_ERR_UNSUPPORTED, "keep_k = %d is too large for the merge path", k);
     CUtensorMap map_h, map_kept;
-    // (the row operand is gathered by ordinary asynchronous copies; the map of `hidden` is only prefetched)
     if (!make_map(ctx, &map_h, in->hidden, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
         !make_map(ctx, &map_kept, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, (uint32_t)n_tile))
       return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for hidden / kept rows");
@@ -377,14 +383,18 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     sa.wide = wide ? 1 : 0;
     sa.groups = groups;
     sa.threshold = p->sim_threshold;
-    sa.drop_idx = drop_idx; sa.hidden = static_cast<const __nv_bfloat16 *>(in->hidden); sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
+    sa.drop_idx = gather_rows ? drop_idx : nullptr; sa.role = ctx->role;
+    sa.hidden = static_cast<const __nv_bfloat16 *>(in->hidden); sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
     sa.best_sim = out->best_sim; sa.seg = ctx->seg; sa.members = ctx->members; sa.counters = ctx->cnt_sim;
     sa.tile_counters = ctx->cnt_tiles; sa.part = ctx->sim_part;
     sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
     sa.smat = nullptr;
     sa.status = ctx->status;
     mark(ctx, "sim", st);
-    launch_pdl(sim_kernel, dim3(dim3(max_mt * groups, B, splits)), dim3(SIM_THREADS), smem, st, map_h, map_kept, sa);
+    if (gather_rows)
+      launch_pdl(sim_kernel<true>, dim3(max_mt * groups, B, splits), dim3(SIM_THREADS), smem, st, map_h, map_kept, sa);
+    else
+      launch_pdl(sim_kernel<false>, dim3(max_mt * groups, B, splits), dim3(SIM_THREADS_TILED), smem, st, map_h, map_kept, sa);
     ASAP_TRY(after_launch(ctx, "sim"));
   }
   return ASAP_OK;
@@ -471,12 +481,12 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   sa.wide = 0;
   sa.groups = 1;
   sa.threshold = p->sim_threshold;
-  sa.drop_idx = nullptr; sa.hidden = nullptr; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
+  sa.drop_idx = nullptr; sa.role = nullptr; sa.hidden = nullptr; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
   sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr; sa.tile_counters = ctx->cnt_tiles;
   sa.part = ctx->sim_part; sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
   sa.smat = smat; sa.status = ctx->status;
   mark(ctx, "sim_kept", st);
-  launch_pdl(sim_kernel, dim3(max_mt, B, splits), dim3(SIM_THREADS), smem, st, map_a, map_b, sa);
+  launch_pdl(sim_kernel<false>, dim3(max_mt, B, splits), dim3(SIM_THREADS_TILED), smem, st, map_a, map_b, sa);
   ASAP_TRY(after_launch(ctx, "sim_kept"));
 
   RouteArgs ra;
@@ -587,7 +597,8 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
   // kernels whose dynamic shared memory exceeds the 48 KB default
   if (e == cudaSuccess) e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_BYTES);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM_BYTES);

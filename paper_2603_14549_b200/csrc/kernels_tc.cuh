@@ -471,13 +471,18 @@ head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
 // =======================================================================================
 // sim_kernel
 //
-// One block per (128 dropped rows, sample, slice of the hidden dimension).  D = Drop_tile Kept^T
-// with M = 128 dropped rows, N = n_tile kept slots per accumulator, K = this block's slice of
-// the hidden size in steps of 64.  The dropped rows are fetched where they lie in `hidden` by four
-// gather warps (16-byte asynchronous copies, written in the 128-byte-swizzled layout the tiled
-// copies produce; a gather copy of four rows per instruction through the tensor-map unit was
-// measured at one instruction per ~74 clk and SM, a tenth of what the tile needs), so only rows
-// whose result is used are multiplied.  While the first
+// One block per (128 rows, sample, slice of the hidden dimension).  D = Row_tile Kept^T
+// with M = 128 rows (see "row operand" below), N = n_tile kept slots per accumulator, K = this block's slice of
+// the hidden size in steps of 64.
+//   row operand:    either the dropped rows alone, fetched where they lie in `hidden` by the gather
+//                   warps (16-byte asynchronous copies, written in the 128-byte-swizzled layout the
+//                   tiled copies produce), so that only rows whose result is used are multiplied; or
+//                   every visual row by plain tiled copies, the kept rows' results being thrown away.
+//                   The gather path moves at most ~23 bytes per clock and SM (the load/store unit's
+//                   requests in flight; a gather copy of four rows per instruction through the
+//                   tensor-map unit managed a third of that), the tiled path twice as much, so the host
+//                   gathers only when the kept rows are a large share of the span.
+// While the first
 // accumulator is being built the epilogue warps also read every row tile from shared memory and
 // add up the squares (the row norms of Sec. 4.2's cosine similarity).
 //   one slice:      the epilogue scales column s by 1/||kept_s||, keeps the running maximum
@@ -508,7 +513,11 @@ head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
 //                   kept set; `tmap_h` is then a map of the kept rows with a 128-row box (plain
 //                   tiled copies, no gather).
 // =======================================================================================
-constexpr int SIM_THREADS = 320;            // copy warp, MMA warp, four epilogue warps, four gather warps
+#ifndef SIM_GWARPS_N
+#define SIM_GWARPS_N 4
+#endif
+constexpr int SIM_GWARPS = SIM_GWARPS_N;                // gather warps
+constexpr int SIM_THREADS = 192 + 32 * SIM_GWARPS;      // copy warp, MMA warp, four epilogue warps, the gather warps
 constexpr int SIM_A_BYTES = 128 * 128;           // 128 rows x 64 bf16
 constexpr int SIM_BOOK_BYTES = 2048;
 constexpr uint32_t SIM_TMEM_COLS = 512;
@@ -521,8 +530,10 @@ struct SimArgs {
   int groups;                // > 1: slot tiles dealt to `groups` blocks per row tile (n_nt counts one group's tiles)
   uint32_t tmem_cols;        // power of two >= 2 * n_tile: two accumulators
   float threshold;
-  const int32_t *drop_idx;   // [B, max_vis-keep_k] dropped tokens, ascending (row operand of the main mode)
-  const __nv_bfloat16 *hidden;   // [tokens, D] (main mode: the gather warps read the dropped rows from here)
+  const int32_t *drop_idx;   // [B, max_vis-keep_k] dropped tokens, ascending: the row operand is gathered from them;
+                             // nullptr: the row operand is every visual row (tiled copies), kept rows' results unused
+  const int32_t *role;       // [B, max_vis] kept slot / -(dropped position + 1) of every visual token (all-rows form)
+  const __nv_bfloat16 *hidden;   // [tokens, D] (the gather warps read the dropped rows from here)
   const float *kept_inv;     // [B*keep_k]   1/||kept row||, 0 for a zero row
   int32_t *assign;           // [B, max_vis-keep_k]
   float *best_sim;           // [B, max_vis-keep_k] or nullptr
@@ -542,6 +553,7 @@ struct SimBook {
   int abort_flag;
   int is_last;
   int scan[33];
+  int rows[128];             // packed row of each of the tile's dropped tokens (main mode)
 };
 
 static_assert(sizeof(SimBook) <= SIM_BOOK_BYTES, "similarity kernel bookkeeping exceeds its shared-memory slot");
@@ -550,7 +562,10 @@ __device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t n) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n) : "memory");
 }
 
-__global__ void __launch_bounds__(SIM_THREADS, 1)
+constexpr int SIM_THREADS_TILED = 192;                  // without gather warps: two such blocks fit an SM
+
+template <bool GATHER>
+__global__ void __launch_bounds__(GATHER ? SIM_THREADS : SIM_THREADS_TILED, 1)
 sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_kept,
            SimArgs a) {
   pdl_enter();
@@ -563,7 +578,8 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   const SampleDesc d = a.desc[b];
   if (!d.valid) return;
   const int nd = d.nv - a.keep_k;                        // dropped tokens of this sample
-  const int n_rows = a.smat ? a.keep_k : nd;             // rows of the row operand
+  constexpr bool gather = GATHER;                        // a.drop_idx given, not matrix mode
+  const int n_rows = a.smat ? a.keep_k : (gather ? nd : d.nv);   // rows of the row operand
   if (mt * 128 >= max(n_rows, 1)) return;
   if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SIM_TIMEOUT) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -583,7 +599,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.stages; ++s) {
-      mbar_init(smem_u32(&bk->full[s]), a.smat ? 1 : 129);  // the copy warp's announcement (+ every gather thread)
+      mbar_init(smem_u32(&bk->full[s]), GATHER ? 1 + 32 * SIM_GWARPS : 1);  // the copy warp's announcement (+ every gather thread)
       mbar_init(smem_u32(&bk->empty[s]), 5);      // the MMAs that read the stage + four epilogue warps
     }
     for (int i = 0; i < 2; ++i) {
@@ -613,9 +629,9 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     if (lane == 0) {
       tma_prefetch_desc(&tmap_h);
       tma_prefetch_desc(&tmap_kept);
-      const bool gather = a.smat == nullptr;
       const int row_b = b * a.keep_k;
-      const int row_a = row_b + mt * 128;                // matrix mode: rows of the dense kept array
+      // tiled row operand: rows of the dense kept array (matrix mode) or of the image span
+      const int row_a = a.smat ? row_b + mt * 128 : d.row0 + d.v0 + mt * 128;
       const int tx_bytes = gather ? stage_bytes - (a.wide ? 1 : 2) * SIM_A_BYTES : stage_bytes;
       const int rot = (mt * 5 + b * 3) % n_kb;
       int issued = 0;
@@ -651,29 +667,28 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       }
     }
   } else if (warp >= 6) {
-    // ---- gather warps (main mode): warp g fetches rows 32 g .. 32 g + 31 of the tile, i.e. the hidden
-    // rows of 32 dropped tokens, one stage's columns at a time.  A warp instruction covers whole rows
+    // ---- gather warps (main mode): warp g fetches its share of the tile's rows (128 / SIM_GWARPS hidden rows
+    // of dropped tokens), one stage's columns at a time.  A warp instruction covers whole rows
     // (2 rows x 256 bytes, or 4 rows x 128 bytes in the one-pass layout), each lane one 16-byte chunk,
     // written where the tiled copies would put it: row r of a 64-column block is 128 bytes at
     // r * 128, its chunk c at position c ^ (r & 7).  Every lane's copies of a stage arrive on the stage's
-    // barrier by themselves when they have landed, so the warps only ever wait for a free stage.
-    if (a.smat == nullptr) {
+    // barrier by themselves when they have landed, so the warps only ever wait for a free stage.  Few
+    // threads with many copies each: every thread costs the barrier one arrival per stage, and 128
+    // arrivals per stage were measured to hold the whole pipeline back.
+    if (gather) {
       const int g = warp - 6;
+      constexpr int RW = 128 / SIM_GWARPS;                // rows of the tile per gather warp
       const int cpr = a.wide ? 8 : 16;                   // 16-byte chunks per row and stage
-      const int c = lane & (cpr - 1), rsub = lane / cpr, rpi = 32 / cpr, n_i = 32 / rpi;
+      const int c = lane & (cpr - 1), rsub = lane / cpr, rpi = 32 / cpr, n_i = RW / rpi;
       const int32_t *drop_b = a.drop_idx + (size_t)b * (a.max_vis - a.keep_k);
-      const uint8_t *hid = reinterpret_cast<const uint8_t *>(a.hidden);
-      const size_t pitch = (size_t)a.D * 2;
-      size_t src_off[16];
-      uint32_t dst_off[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int r = g * 32 + (i < n_i ? i : 0) * rpi + rsub;
+      for (int r = g * RW + lane; r < (g + 1) * RW; r += 32) {
         const int dp = min(mt * 128 + r, nd - 1);        // the ragged tail repeats the last dropped token
-        const int row = d.row0 + d.v0 + min(max(__ldg(drop_b + dp), 0), d.nv - 1);
-        src_off[i] = (size_t)row * pitch + (size_t)c * 16;
-        dst_off[i] = (uint32_t)((c >> 3) * SIM_A_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+        bk->rows[r] = d.row0 + d.v0 + min(max(__ldg(drop_b + dp), 0), d.nv - 1);
       }
+      __syncwarp();
+      const uint8_t *hid = reinterpret_cast<const uint8_t *>(a.hidden) + (size_t)c * 16;
+      const size_t pitch = (size_t)a.D * 2;
+      const uint32_t dst_c = (uint32_t)((c >> 3) * SIM_A_BYTES);
       const int stage_cols_bytes = a.wide ? 128 : 256;
       const int rot = (mt * 5 + b * 3) % n_kb;
       for (int it = 0; it < total_it; ++it) {
@@ -685,11 +700,13 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         }
         go = __shfl_sync(0xffffffffu, go, 0);
         if (!go) break;
-        const uint32_t dst = base + s * stage_bytes;
+        const uint32_t dst = base + s * stage_bytes + dst_c;
         const uint8_t *src = hid + (size_t)kb * stage_cols_bytes;
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-          if (i < n_i) cp_async16(dst + dst_off[i], src + src_off[i]);
+#pragma unroll 8
+        for (int i = 0; i < n_i; ++i) {
+          const int r = g * RW + i * rpi + rsub;
+          cp_async16(dst + r * 128 + (((c & 7) ^ (r & 7)) << 4), src + (size_t)bk->rows[r] * pitch);
+        }
         cp_async_arrive_on(smem_u32(&bk->full[s]));       // this lane's share of the stage, once it has landed
       }
       cp_async_commit();
@@ -908,11 +925,17 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       }
     }
     if (a.smat) finalize = false;
-    if (finalize && v < nd && !bk->abort_flag) {
+    // the dropped position of this thread's row: the row index itself, or looked up for a visual row
+    int dp = -1;
+    if (finalize && v < n_rows) {
+      if (gather) dp = v;
+      else { const int role = a.role[(size_t)b * a.max_vis + v]; dp = role < 0 ? -role - 1 : -1; }
+    }
+    if (dp >= 0 && dp < nd && !bk->abort_flag) {
       const bool zero_row = !(ss_tot >= 1e-24f);        // ||h|| < 1e-12: similarity 0 to every slot
       const float sim = zero_row ? 0.f : best * rsqrtf(ss_tot);
       const int slot = zero_row ? 0 : best_slot;
-      const size_t o = (size_t)b * (a.max_vis - a.keep_k) + v;
+      const size_t o = (size_t)b * (a.max_vis - a.keep_k) + dp;
       a.assign[o] = (sim > a.threshold) ? slot : -1;
       if (a.best_sim) a.best_sim[o] = sim;
     }
@@ -931,7 +954,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   // the block that finishes the sample's last row tile groups the dropped tokens by destination
   if (threadIdx.x == 0) {
     __threadfence();
-    const unsigned int n_mt = (unsigned int)((nd + 127) / 128);
+    const unsigned int n_mt = (unsigned int)((n_rows + 127) / 128);
     const unsigned int old = atomicAdd(a.counters + b, 1u);
     bk->is_last = (old == n_mt - 1u);
     if (bk->is_last) a.counters[b] = 0u;
