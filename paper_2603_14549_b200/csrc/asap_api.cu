@@ -42,7 +42,7 @@ struct asap_ctx {
   float *qsum_partial = nullptr, *qbar = nullptr, *score_partial = nullptr, *inv_norm = nullptr,
         *kept_inv = nullptr;
   unsigned int *cnt_qsum = nullptr, *cnt_mass = nullptr, *cnt_score = nullptr, *cnt_sim = nullptr,
-               *cnt_tiles = nullptr;
+               *cnt_tiles = nullptr, *cnt_work = nullptr;
   float *sim_part = nullptr;        // partial dot products / squared norms of a sliced similarity GEMM
   size_t sim_part_bytes = 0, cap_tiles = 0;
   int32_t *role = nullptr, *seg = nullptr, *members = nullptr;
@@ -267,7 +267,7 @@ asap_status launch_rank(asap_ctx *ctx, const asap_inputs *in, const asap_params 
   sa.mask_log = p->per_head_mask ? out->mask_log_heads : out->mask_log;
   sa.mask_b_stride = p->per_head_mask ? in->H * in->max_vis : in->max_vis;
   sa.mask_h_stride = p->per_head_mask ? in->max_vis : 0;
-  sa.partial = ctx->score_partial; sa.status = ctx->status;
+  sa.partial = ctx->score_partial; sa.work = ctx->cnt_work; sa.status = ctx->status;
   mark(ctx, "score", st);
   const int items = B * in->H;
   launch_pdl(score_kernel, dim3(items < ctx->num_sms ? items : ctx->num_sms), dim3(SC_THREADS), SC_SMEM_BYTES, st,
@@ -560,7 +560,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   const size_t o_spart = carve(Hc * T * sizeof(float));
   const size_t o_inv = carve(T * sizeof(float));
   const size_t o_kinv = carve(max_keep_rows * sizeof(float));
-  const size_t o_cnt = carve((Bc * col_blocks + 3 * Bc) * sizeof(unsigned int));
+  const size_t o_cnt = carve((Bc * col_blocks + 3 * Bc + 2) * sizeof(unsigned int));
   const size_t o_role = carve(T * sizeof(int32_t));
   const size_t o_seg = carve((max_keep_rows + Bc) * sizeof(int32_t));
   const size_t o_mem = carve(T * sizeof(int32_t));
@@ -585,6 +585,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   ctx->cnt_mass = ctx->cnt_qsum + Bc * col_blocks;
   ctx->cnt_score = ctx->cnt_mass + Bc;
   ctx->cnt_sim = ctx->cnt_score + Bc;
+  ctx->cnt_work = ctx->cnt_sim + Bc;
   ctx->role = reinterpret_cast<int32_t *>(ctx->arena + o_role);
   ctx->seg = reinterpret_cast<int32_t *>(ctx->arena + o_seg);
   ctx->members = reinterpret_cast<int32_t *>(ctx->arena + o_mem);
@@ -592,7 +593,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   ctx->cnt_tiles = reinterpret_cast<unsigned int *>(ctx->arena + o_tiles);
   ctx->sim_part = reinterpret_cast<float *>(ctx->arena + o_simpart);
   ctx->status = reinterpret_cast<uint32_t *>(ctx->arena + o_status);
-  e = cudaMemset(ctx->arena + o_cnt, 0, (Bc * col_blocks + 3 * Bc) * sizeof(unsigned int));
+  e = cudaMemset(ctx->arena + o_cnt, 0, (Bc * col_blocks + 3 * Bc + 2) * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMemset(ctx->arena + o_tiles, 0, ctx->cap_tiles * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
   // kernels whose dynamic shared memory exceeds the 48 KB default

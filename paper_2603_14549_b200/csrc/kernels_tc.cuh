@@ -33,17 +33,22 @@ __device__ __forceinline__ void group_bar_sync(int group) {
 // =======================================================================================
 // score_kernel
 //
-// Persistent blocks; a work item is one (sample b, head h) and blocks take items round robin.
-// For each tile of up to 128 ranking rows of the item:
-//   pass 1  D = Q_rows K_tile^T   (M = 128 rows,  N = 128 keys): thread-per-row running
-//           max / sum over all admitted keys  ->  off_i = max_i + log2(sum_i)   (log2 units)
-//   pass 2  D = K_tile Q_rows^T   (M = 128 keys,  N = rows):     thread-per-key sum over rows
-//           of exp2(logit + mask - off_i), i.e. of the Eq. 4 probabilities A[i, j]
+// Persistent blocks; a work item is one (sample b, head h); blocks draw items from a global
+// counter (the ranking rows per sample differ by up to 8x, so a fixed deal leaves blocks idle).
+// The ranking rows of an item are taken 256 at a time (a row pair: two row tiles of 128).  For
+// each row pair, every key tile is brought to shared memory once per pass and serves both row tiles:
+//   pass 1  D = Q_rows K_tile^T   (M = 128 rows, N = 128 keys, one accumulator per row tile):
+//           thread-per-row running max / sum over all admitted keys -> off_i = max_i + log2(sum_i)
+//   pass 2  D = K_tile Q_rows^T   (M = 128 keys, N = all rows of the pair, up to 256): thread-per-key
+//           sum over rows of exp2(logit + mask - off_i), i.e. of the Eq. 4 probabilities A[i, j]
 // Key tiles stream through a shared-memory ring in one linear order (pass 1 ascending, pass 2
-// over the tiles that hold visual keys, coming back from L2), the query tile is double
-// buffered, and so are the accumulators in tensor memory; the producer and the MMA issuer run
-// ahead across passes, row tiles and items, so the only warps that ever wait are the four
-// epilogue warps' consumers.
+// over the tiles that hold visual keys, coming back from L2); tensor memory holds two halves of 256
+// columns that alternate between consecutive operations, so the MMA issuer runs one operation ahead
+// of the epilogue warps.
+// Epilogue: two groups of four warps.  Pass 1 with two row tiles: group g owns row tile g of every
+// key tile.  Pass 1 with one row tile, and pass 2: the groups take alternate operations.  Every
+// epilogue warp passes every operation's barriers (waits for the accumulator, releases it), whether
+// it has work on it or not, so the barrier counts never depend on the shape of the item.
 // Additive mask (Eq. 3), logits in log2 units: 0 for key j <= row position p; m_j*log2(e) for
 // j > p when both are in the image span (mask enabled); -inf otherwise.
 // The per-head sums over ranking rows go to `partial`; head_sum_kernel adds them in head order.
@@ -53,13 +58,16 @@ constexpr int SC_EPI_THREADS = 256;
 constexpr int SC_STAGES = 4;
 constexpr int SC_HALF_BYTES = 128 * 128;        // 128 rows x 64 bf16
 constexpr int SC_TILE_BYTES = 2 * SC_HALF_BYTES;
-constexpr int SC_SMEM_MAIN = (2 + SC_STAGES) * SC_TILE_BYTES;
+constexpr int SC_Q_HALF_BYTES = 256 * 128;      // 256 rows x 64 bf16: one 64-column half of a row pair
+constexpr int SC_Q_BYTES = 2 * SC_Q_HALF_BYTES;
+constexpr int SC_SMEM_MAIN = SC_Q_BYTES + SC_STAGES * SC_TILE_BYTES;
 // Total dynamic shared memory stays at 195 KB: with the 1 KB the system reserves per block that
 // is the 196 KB carve-out, which leaves the SM 32 KB of L1 for the memory-bound kernels that run
 // beside this one; one byte more selects the 228 KB carve-out and costs them about 10 us.
 constexpr int SC_BOOK_BYTES = 3072;
 constexpr int SC_SMEM_BYTES = SC_SMEM_MAIN + SC_BOOK_BYTES;
-constexpr uint32_t SC_TMEM_COLS = 512;     // four accumulators of 128 columns
+constexpr uint32_t SC_TMEM_COLS = 512;     // two halves of 256 columns
+constexpr int SC_ITEM_SLOTS = 4;
 
 struct ScoreArgs {
   PrepareArgs pa;             // every block derives its descriptors itself: the kernel does not wait
@@ -69,29 +77,36 @@ struct ScoreArgs {
   const float *mask_log;      // [B, max_vis] m_j (natural log), or [B, H, max_vis] with a mask per head
   int mask_b_stride, mask_h_stride;   // max_vis, 0   or   H * max_vis, max_vis
   float *partial;             // [B, H, max_vis] per-head sums over ranking rows
+  unsigned int *work;         // [2] next item / blocks that have finished; both zero between launches
   uint32_t *status;
 };
 
 struct ScoreBook {             // bookkeeping block placed after the tiles in shared memory
-  uint64_t full[SC_STAGES], empty[SC_STAGES], q_full[2], q_empty[2], acc_full[4], acc_empty[4];
-  float off[128];              // per ranking row: max + log2(sum), +inf for rows past the tile
-  float soft[2][128];          // per epilogue group, per key of its current tile: m_j*log2(e) or -inf
-  float pm[128], pl[128];      // group 1's running (max, sum) per row at the end of pass 1
+  uint64_t full[SC_STAGES], empty[SC_STAGES], q_full, q_empty, acc_full[2], acc_empty[2];
+  uint64_t item_full[SC_ITEM_SLOTS], item_empty[SC_ITEM_SLOTS], mma_done;
+  int item_q[SC_ITEM_SLOTS];   // items drawn by the producer, -1 = no more
+  alignas(16) float off[256];  // per ranking row of the pair: max + log2(sum), +inf for rows past its end
+                               // (with one row tile, off[128..255] carries group 1's partial sums)
+  alignas(16) float soft[2][128];   // per epilogue group, per key of its current tile: m_j*log2(e) or -inf
+                               // (soft[1] also carries group 1's partial maxima at the end of pass 1)
   uint32_t tmem_base;
   int abort_flag;
 };
 
 static_assert(sizeof(ScoreBook) <= SC_BOOK_BYTES, "score kernel bookkeeping exceeds its shared-memory slot");
 
-struct RowTile {
-  int R0, nrows, n_kt, t_lo, t_hi, n_p2;
+struct RowPair {
+  int R0, nrows, nrt, n2, n_kt, t_lo, t_hi, n_p2;
   bool use_soft;
 };
 
-__device__ __forceinline__ RowTile score_row_tile(const SampleDesc &d, int rt, int mask_enable) {
-  RowTile r;
-  r.R0 = d.r0 + rt * 128;
-  r.nrows = min(128, d.nr - rt * 128);
+// Row pair rp of a sample's ranking rows: rows R0 .. R0 + nrows - 1 (sequence-relative positions).
+__device__ __forceinline__ RowPair score_row_pair(const SampleDesc &d, int rp, int mask_enable) {
+  RowPair r;
+  r.R0 = d.r0 + rp * 256;
+  r.nrows = min(256, d.nr - rp * 256);
+  r.nrt = (r.nrows + 127) >> 7;
+  r.n2 = (r.nrows + 15) & ~15;
   const int p_max = r.R0 + r.nrows - 1;
   r.use_soft = mask_enable && (r.R0 < d.v0 + d.nv) && (p_max >= d.v0);
   int jmax = p_max;
@@ -118,8 +133,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     if (threadIdx.x == 0) atomicOr(a.status, STATUS_SCORE_TIMEOUT);
     return;
   }
-  const uint32_t q_smem = base;                          // two query tiles
-  const uint32_t k_smem = base + 2 * SC_TILE_BYTES;      // ring of key tiles
+  const uint32_t q_smem = base;                          // the row pair's queries
+  const uint32_t k_smem = base + SC_Q_BYTES;             // ring of key tiles
   ScoreBook *bk = reinterpret_cast<ScoreBook *>(base_ptr + SC_SMEM_MAIN);
 
   if (threadIdx.x == 0) {
@@ -127,14 +142,17 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       mbar_init(smem_u32(&bk->full[s]), 1);
       mbar_init(smem_u32(&bk->empty[s]), 1);
     }
+    mbar_init(smem_u32(&bk->q_full), 1);
+    mbar_init(smem_u32(&bk->q_empty), 1);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&bk->q_full[i]), 1);
-      mbar_init(smem_u32(&bk->q_empty[i]), 1);
-    }
-    for (int i = 0; i < 4; ++i) {
       mbar_init(smem_u32(&bk->acc_full[i]), 1);
-      mbar_init(smem_u32(&bk->acc_empty[i]), 4);
+      mbar_init(smem_u32(&bk->acc_empty[i]), 8);          // every epilogue warp
     }
+    for (int i = 0; i < SC_ITEM_SLOTS; ++i) {
+      mbar_init(smem_u32(&bk->item_full[i]), 1);
+      mbar_init(smem_u32(&bk->item_empty[i]), 9);         // the MMA issuer + every epilogue warp
+    }
+    mbar_init(smem_u32(&bk->mma_done), 1);
     bk->abort_flag = 0;
     fence_barrier_init();
   }
@@ -151,27 +169,35 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   __syncthreads();
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ producer: items, queries, key tiles
     if (lane == 0) {
       tma_prefetch_desc(&tmap_q);
       tma_prefetch_desc(&tmap_k);
-      int kc = 0, qc = 0;                       // key tiles / query tiles issued so far
+      int kc = 0, qc = 0, ic = 0;               // key tiles / row pairs / items so far
       int k_issued = 0, q_issued = 0;           // copies actually issued (an abort is sticky, so
                                                 // these are prefixes of the two sequences)
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+      while (true) {
+        const int slot = ic % SC_ITEM_SLOTS;
+        if (ic >= SC_ITEM_SLOTS) mbar_wait(smem_u32(&bk->item_empty[slot]), ((ic / SC_ITEM_SLOTS) - 1) & 1, wc);
+        int item = bk->abort_flag ? n_items : (int)atomicAdd(a.work, 1u);
+        if (item >= n_items) item = -1;
+        bk->item_q[slot] = item;
+        mbar_arrive(smem_u32(&bk->item_full[slot]));      // release: the slot's content is visible to the waiters
+        ++ic;
+        if (item < 0) break;
         const int b = item / a.H, h = item - b * a.H;
         const SampleDesc d = make_desc(a.pa, b);
         if (!d.valid) continue;
-        const int n_rt = (d.nr + 127) / 128;
-        for (int rt = 0; rt < n_rt; ++rt, ++qc) {
-          const RowTile T = score_row_tile(d, rt, a.mask_enable);
-          const int qb = qc & 1;
-          if (qc >= 2) mbar_wait(smem_u32(&bk->q_empty[qb]), ((qc >> 1) - 1) & 1, wc);
+        const int n_rp = (d.nr + 255) / 256;
+        for (int rp = 0; rp < n_rp; ++rp, ++qc) {
+          const RowPair T = score_row_pair(d, rp, a.mask_enable);
+          if (qc >= 1) mbar_wait(smem_u32(&bk->q_empty), (qc - 1) & 1, wc);
           if (!bk->abort_flag) {
-            const uint32_t dst = q_smem + qb * SC_TILE_BYTES;
-            mbar_expect_tx(smem_u32(&bk->q_full[qb]), SC_TILE_BYTES);
-            tma_load_2d(dst, &tmap_q, smem_u32(&bk->q_full[qb]), h * 128, d.row0 + T.R0);
-            tma_load_2d(dst + SC_HALF_BYTES, &tmap_q, smem_u32(&bk->q_full[qb]), h * 128 + 64, d.row0 + T.R0);
+            mbar_expect_tx(smem_u32(&bk->q_full), T.nrt * SC_TILE_BYTES);
+            for (int hf = 0; hf < 2; ++hf)
+              for (int rt = 0; rt < T.nrt; ++rt)
+                tma_load_2d(q_smem + hf * SC_Q_HALF_BYTES + rt * SC_HALF_BYTES, &tmap_q, smem_u32(&bk->q_full),
+                            h * 128 + hf * 64, d.row0 + T.R0 + rt * 128);
             q_issued = qc + 1;
           }
           for (int u = 0; u < T.n_kt + T.n_p2; ++u, ++kc) {
@@ -193,58 +219,69 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         const int fills = k_issued > s ? (k_issued - s + SC_STAGES - 1) / SC_STAGES : 0;
         if (fills > 0) mbar_wait_drain(smem_u32(&bk->full[s]), (fills - 1) & 1, TC_WAIT_LIMIT);
       }
-      for (int i = 0; i < 2; ++i) {
-        const int fills = q_issued > i ? (q_issued - i + 1) / 2 : 0;
-        if (fills > 0) mbar_wait_drain(smem_u32(&bk->q_full[i]), (fills - 1) & 1, TC_WAIT_LIMIT);
-      }
+      if (q_issued > 0) mbar_wait_drain(smem_u32(&bk->q_full), (q_issued - 1) & 1, TC_WAIT_LIMIT);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      int kc = 0, qc = 0, g = 0;
+      int kc = 0, qc = 0, g = 0, ic = 0;
+      bool issued_any = false;
       const uint32_t idesc1 = umma_idesc_bf16(128, 128);
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+      while (true) {
+        const int slot = ic % SC_ITEM_SLOTS;
+        mbar_wait(smem_u32(&bk->item_full[slot]), (ic / SC_ITEM_SLOTS) & 1, wc);
+        const int item = bk->abort_flag ? -1 : bk->item_q[slot];
+        mbar_arrive(smem_u32(&bk->item_empty[slot]));
+        ++ic;
+        if (item < 0) break;
         const int b = item / a.H;
         const SampleDesc d = make_desc(a.pa, b);
         if (!d.valid) continue;
-        const int n_rt = (d.nr + 127) / 128;
-        for (int rt = 0; rt < n_rt; ++rt, ++qc) {
-          const RowTile T = score_row_tile(d, rt, a.mask_enable);
-          const int n2 = (T.nrows + 15) & ~15;
-          const uint32_t idesc2 = umma_idesc_bf16(128, n2);
-          const int qb = qc & 1;
-          const uint32_t qs = q_smem + qb * SC_TILE_BYTES;
-          mbar_wait(smem_u32(&bk->q_full[qb]), (qc >> 1) & 1, wc);
+        const int n_rp = (d.nr + 255) / 256;
+        for (int rp = 0; rp < n_rp; ++rp, ++qc) {
+          const RowPair T = score_row_pair(d, rp, a.mask_enable);
+          const uint32_t idesc2 = umma_idesc_bf16(128, T.n2);
+          mbar_wait(smem_u32(&bk->q_full), qc & 1, wc);
           for (int u = 0; u < T.n_kt + T.n_p2; ++u, ++kc, ++g) {
             const bool pass1 = u < T.n_kt;
-            const int s = kc % SC_STAGES, buf = g & 3;
-            if (g >= 4) mbar_wait(smem_u32(&bk->acc_empty[buf]), ((g >> 2) - 1) & 1, wc);
+            const int s = kc % SC_STAGES, hh = g & 1;
+            if (g >= 2) mbar_wait(smem_u32(&bk->acc_empty[hh]), ((g >> 1) - 1) & 1, wc);
             mbar_wait(smem_u32(&bk->full[s]), (kc / SC_STAGES) & 1, wc);
             tc_fence_after();
             if (!bk->abort_flag) {
               const uint32_t ks = k_smem + s * SC_TILE_BYTES;
-              const uint32_t dcol = tmem_base + buf * 128;
+              const uint32_t dcol = tmem_base + hh * 256;
+              if (pass1) {
+                for (int rt = 0; rt < T.nrt; ++rt)
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk) {
-                const uint32_t o = (kk >> 2) * SC_HALF_BYTES + (kk & 3) * 32;
-                const uint64_t dq = umma_desc_sw128(qs + o), dk = umma_desc_sw128(ks + o);
-                if (pass1) tc_mma_bf16(dcol, dq, dk, idesc1, kk > 0);
-                else       tc_mma_bf16(dcol, dk, dq, idesc2, kk > 0);
+                  for (int kk = 0; kk < 8; ++kk)
+                    tc_mma_bf16(dcol + rt * 128,
+                                umma_desc_sw128(q_smem + (kk >> 2) * SC_Q_HALF_BYTES + rt * SC_HALF_BYTES + (kk & 3) * 32),
+                                umma_desc_sw128(ks + (kk >> 2) * SC_HALF_BYTES + (kk & 3) * 32), idesc1, kk > 0);
+              } else {
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                  tc_mma_bf16(dcol, umma_desc_sw128(ks + (kk >> 2) * SC_HALF_BYTES + (kk & 3) * 32),
+                              umma_desc_sw128(q_smem + (kk >> 2) * SC_Q_HALF_BYTES + (kk & 3) * 32), idesc2, kk > 0);
               }
               tc_commit(smem_u32(&bk->empty[s]));
-              tc_commit(smem_u32(&bk->acc_full[buf]));
+              tc_commit(smem_u32(&bk->acc_full[hh]));
+              issued_any = true;
             }
           }
-          if (!bk->abort_flag) tc_commit(smem_u32(&bk->q_empty[qb]));
+          if (!bk->abort_flag) tc_commit(smem_u32(&bk->q_empty));
         }
+      }
+      // every MMA this thread issued has completed before tensor memory is given back: after an abort the
+      // epilogue warps no longer wait for the accumulators, so nothing else would hold the block until then
+      if (issued_any) {
+        tc_commit(smem_u32(&bk->mma_done));
+        mbar_wait_drain(smem_u32(&bk->mma_done), 0, TC_WAIT_LIMIT);
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue (2 groups x 4 warps)
-    // Group w owns accumulators w and w + 2, i.e. every second operation of the linear sequence
-    // (operation g uses accumulator g mod 4), so the MMA issuer can run two operations ahead; the
-    // two groups share the four sub-partitions, so one group's exponentials overlap the other's
-    // tensor-memory loads.  Warp q of a group reads tensor-memory lanes 32q .. 32q+31.
+    // Warp q of a group reads tensor-memory lanes 32q .. 32q+31.
     const int group = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int lrow = quarter * 32 + lane;          // tensor-memory lane owned by this thread
@@ -252,53 +289,80 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     const float scale = a.scale_log2;
     const uint32_t tlane0 = tmem_base + ((uint32_t)(quarter * 32) << 16);
     float *soft = bk->soft[group];
-    int g = 0;
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    float *pm = bk->soft[1], *pl = bk->off + 128;  // group 1's (max, sum) when both groups share one row tile
+    int g = 0, ic = 0;
+    while (true) {
+      const int slot = ic % SC_ITEM_SLOTS;
+      mbar_wait(smem_u32(&bk->item_full[slot]), (ic / SC_ITEM_SLOTS) & 1, wc);
+      const int item = bk->abort_flag ? -1 : bk->item_q[slot];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bk->item_empty[slot]));
+      ++ic;
+      if (item < 0) break;
       const int b = item / a.H, h = item - b * a.H;
       const SampleDesc d = make_desc(a.pa, b);
       if (!d.valid) continue;
-      const int n_rt = (d.nr + 127) / 128;
+      const int n_rp = (d.nr + 255) / 256;
       float *part = a.partial + ((size_t)b * a.H + h) * a.max_vis;
       const float *mlog = a.mask_log + (size_t)b * a.mask_b_stride + (size_t)h * a.mask_h_stride;
       const int v_end = d.v0 + d.nv;
       {
-        // visual keys beyond the tiles the first row tile visits in pass 2 (possible only when
+        // visual keys beyond the tiles the first row pair visits in pass 2 (possible only when
         // ranking rows lie before the end of the image span) start from zero; the epilogue-wide
         // barrier that ends every pass 1 orders these stores before any later add
-        const RowTile T0 = score_row_tile(d, 0, a.mask_enable);
+        const RowPair T0 = score_row_pair(d, 0, a.mask_enable);
         const int first = T0.n_p2 > 0 ? max((T0.t_hi + 1) * 128 - d.v0, 0) : 0;
         for (int j = first + et; j < d.nv; j += SC_EPI_THREADS) part[j] = 0.f;
       }
-      for (int rt = 0; rt < n_rt; ++rt) {
-        const RowTile T = score_row_tile(d, rt, a.mask_enable);
-        // ---------------- pass 1: thread = ranking row, this group's share of the key tiles
-        const bool row_ok = lrow < T.nrows;
-        const bool warp_rows = quarter * 32 < T.nrows;
-        const int p_i = T.R0 + lrow;
+      for (int rp = 0; rp < n_rp; ++rp) {
+        const RowPair T = score_row_pair(d, rp, a.mask_enable);
+        // ---------------- pass 1: thread = ranking row.  Two row tiles: group g owns tile g of every key
+        // tile; one row tile: the groups take alternate key tiles
+        const bool two = T.nrt == 2;
+        const int my_row = (two ? group * 128 : 0) + lrow;             // row of the pair
+        const bool row_ok = my_row < T.nrows;
+        const bool warp_rows = (two ? group * 128 : 0) + quarter * 32 < T.nrows;
+        const int p_i = T.R0 + my_row;
         const bool row_vis = T.use_soft && p_i >= d.v0 && p_i < v_end;
         float m = -INFINITY, l = 0.f;
         for (int t = 0; t < T.n_kt; ++t, ++g) {
-          if ((g & 1) != group) continue;
+          const int hh = g & 1;
+          const bool mine = two || hh == group;
           const int j0 = t * 128;
-          const bool fast = (j0 + 127 <= T.R0);
-          const bool stage_soft = T.use_soft && !fast;
+          const bool fast = (j0 + 127 <= T.R0 + (two ? group * 128 : 0));
+          const bool stage_soft = mine && T.use_soft && !fast;
           if (stage_soft) {
             const int j = j0 + lrow;
             soft[lrow] = (j >= d.v0 && j < v_end) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
             group_bar_sync(group);
           }
-          const int buf = g & 3;
-          const uint32_t tlane = tlane0 + buf * 128;
-          mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 2) & 1, wc);
+          const uint32_t tlane = tlane0 + hh * 256 + (two ? group * 128 : 0);
+          mbar_wait(smem_u32(&bk->acc_full[hh]), (g >> 1) & 1, wc);
           tc_fence_after();
-          if (warp_rows) {
+          if (mine && warp_rows && !bk->abort_flag) {
 #pragma unroll 1
             for (int c = 0; c < 128; c += 64) {
               uint32_t r[64];
               tmem_ld32p(tlane + c, r);
               tmem_ld32p(tlane + c + 32, r + 32);
               tmem_wait_ld();
-              if (fast) {
+              bool summed = false;
+              if (fast && m > -INFINITY) {
+                // every key admitted, no mask, and the row already has a reference maximum: add
+                // exp2(dot * scale - m) without looking for a new maximum (a stale reference only scales
+                // the sum; off_i = m + log2(l) comes out the same).  Should a term outgrow fp32's range
+                // the chunk is done again below, with its true maximum as the new reference.
+                float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int e = 0; e < 64; ++e) sm[e & 7] += fast_exp2(fmaf(__uint_as_float(r[e]), scale, -m));
+                const float cs = ((sm[0] + sm[1]) + (sm[2] + sm[3])) + ((sm[4] + sm[5]) + (sm[6] + sm[7]));
+                if (cs < 1e30f) {
+                  if (row_ok) l += cs;
+                  summed = true;
+                }
+              }
+              if (summed) {
+              } else if (fast) {
                 // every key admitted, no mask: max on the raw dot products (scale > 0), then
                 // exp2(dot * scale - max) into eight independent partial sums
                 float mx[8];
@@ -354,42 +418,47 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           }
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
+          if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[hh]));
           if (stage_soft) group_bar_sync(group);   // soft[] is rewritten by this group's next masked tile
         }
-        // the two groups saw disjoint key tiles: merge their (max, sum) per row, then
-        // off_i = max_i + log2(sum_i), so that exp2(x - off_i) = exp2(x - max_i) / sum_i
-        if (group == 1) { bk->pm[lrow] = m; bk->pl[lrow] = l; }
-        epi_bar_sync();
-        if (group == 0) {
-          const float m1 = bk->pm[lrow], l1 = bk->pl[lrow];
-          const float mm = fmaxf(m, m1);
-          float ll = 0.f;
-          if (m > -INFINITY) ll += l * fast_exp2(m - mm);
-          if (m1 > -INFINITY) ll += l1 * fast_exp2(m1 - mm);
-          bk->off[lrow] = row_ok ? (mm + __log2f(ll)) : INFINITY;
+        // off_i = max_i + log2(sum_i), so that exp2(x - off_i) = exp2(x - max_i) / sum_i.  With one row
+        // tile the two groups saw disjoint key tiles: their (max, sum) per row are merged first
+        if (two) {
+          bk->off[my_row] = row_ok ? (m + __log2f(l)) : INFINITY;
+          epi_bar_sync();
+        } else {
+          epi_bar_sync();                           // group 0 is past its last use of soft[1] and off[128..]
+          if (group == 1) { pm[lrow] = m; pl[lrow] = l; }
+          epi_bar_sync();
+          if (group == 0) {
+            const float m1 = pm[lrow], l1 = pl[lrow];
+            const float mm = fmaxf(m, m1);
+            float ll = 0.f;
+            if (m > -INFINITY) ll += l * fast_exp2(m - mm);
+            if (m1 > -INFINITY) ll += l1 * fast_exp2(m1 - mm);
+            bk->off[lrow] = row_ok ? (mm + __log2f(ll)) : INFINITY;
+          }
+          epi_bar_sync();
         }
-        epi_bar_sync();
-        // ---------------- pass 2: thread = key, this group's share of the visual key tiles
-        const int n2 = (T.nrows + 15) & ~15;
+        // ---------------- pass 2: thread = key; the groups take alternate visual key tiles
         for (int u = 0; u < T.n_p2; ++u, ++g) {
-          if ((g & 1) != group) continue;
+          const int hh = g & 1;
+          const bool mine = hh == group;
           const int t = T.t_hi - u, j0 = t * 128;
           const int j = j0 + lrow;
           const bool key_ok = j >= d.v0 && j < v_end;
           const bool fast = (j0 + 127 <= T.R0);
           const bool warp_keys = (j0 + quarter * 32 + 31 >= d.v0) && (j0 + quarter * 32 < v_end);
-          const float soft_j = (T.use_soft && key_ok) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
-          const int buf = g & 3;
-          const uint32_t tlane = tlane0 + buf * 128;
-          mbar_wait(smem_u32(&bk->acc_full[buf]), (g >> 2) & 1, wc);
+          const float soft_j = (mine && T.use_soft && key_ok) ? __ldg(mlog + (j - d.v0)) * LOG2E_F : -INFINITY;
+          const uint32_t tlane = tlane0 + hh * 256;
+          mbar_wait(smem_u32(&bk->acc_full[hh]), (g >> 1) & 1, wc);
           tc_fence_after();
-          if (warp_keys) {
+          if (mine && warp_keys && !bk->abort_flag) {
             float sm[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
-            for (int c = 0; c < n2; c += 32) {
+            for (int c = 0; c < T.n2; c += 32) {
               uint32_t r[32];
-              const bool full = c + 32 <= n2;       // n2 is a multiple of 16: the last chunk may be half
+              const bool full = c + 32 <= T.n2;       // n2 is a multiple of 16: the last chunk may be half
               if (full) tmem_ld32p(tlane + c, r);
               else {
                 tmem_ld16p(tlane + c, r);
@@ -397,18 +466,20 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 for (int e = 16; e < 32; ++e) r[e] = 0u;
               }
               tmem_wait_ld();
-              // rows past the tile have off = +inf, so their terms vanish
+              // rows past the pair's end have off = +inf (every entry up to the next multiple of 128 is
+              // written), so their terms vanish; four offsets per shared-memory load
+              float o32[32];
+#pragma unroll
+              for (int e = 0; e < 32; e += 4)
+                *reinterpret_cast<float4 *>(o32 + e) = *reinterpret_cast<const float4 *>(bk->off + c + e);
               if (fast) {
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                  const float o = (full || e < 16) ? bk->off[c + e] : INFINITY;
-                  sm[e & 7] += fast_exp2(fmaf(__uint_as_float(r[e]), scale, -o));
-                }
+                for (int e = 0; e < 32; ++e) sm[e & 7] += fast_exp2(fmaf(__uint_as_float(r[e]), scale, -o32[e]));
               } else {
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                   const int p = T.R0 + c + e;
-                  const float o = (full || e < 16) ? bk->off[c + e] : INFINITY;
+                  const float o = o32[e];
                   const float above = (p >= d.v0 && p < v_end) ? soft_j : -INFINITY;
                   const float add = (j <= p) ? 0.f : above;
                   sm[e & 7] += fast_exp2(fmaf(__uint_as_float(r[e]), scale, add) - o);
@@ -417,16 +488,16 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             }
             if (key_ok) {
               const float sum = ((sm[0] + sm[1]) + (sm[2] + sm[3])) + ((sm[4] + sm[5]) + (sm[6] + sm[7]));
-              // the first row tile initialises the slots it covers; later row tiles add
-              if (rt == 0) part[j - d.v0] = sum;
+              // the first row pair initialises the slots it covers; later row pairs add
+              if (rp == 0) part[j - d.v0] = sum;
               else part[j - d.v0] += sum;
             }
           }
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[buf]));
+          if (lane == 0) mbar_arrive(smem_u32(&bk->acc_empty[hh]));
         }
-        epi_bar_sync();   // off[] is rewritten by the next row tile
+        epi_bar_sync();   // off[] is rewritten by the next row pair; its sums are visible to the next pair's adds
       }
     }
     __threadfence();
@@ -438,6 +509,16 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, SC_TMEM_COLS);
+  }
+  // the block that leaves last puts the work counters back to zero for the next launch (every block
+  // has drawn its last item by then: a block only gets here after a draw past the end)
+  if (threadIdx.x == 0) {
+    const unsigned int done = atomicAdd(a.work + 1, 1u);
+    if (done == gridDim.x - 1) {
+      a.work[0] = 0u;
+      a.work[1] = 0u;
+      __threadfence();
+    }
   }
 }
 

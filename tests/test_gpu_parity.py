@@ -59,6 +59,18 @@ def test_many_row_tiles_and_three_slot_tiles(ctx):
     run_step(ctx, batch, A.Params(keep_k=600), samples=[0, 1, 14])
 
 
+def test_a_late_dominant_key_moves_the_softmax_reference(ctx):
+    """One visual key far into the sequence is scaled so that its logits exceed every earlier logit of a
+    ranking row by hundreds of nats (or fall that far below, for rows whose dot product is negative).  A
+    running sum kept relative to an early maximum would overflow there: the row's reference has to move,
+    and the probabilities of all other keys have to come out as (correctly) vanishing."""
+    batch = W.tiny(B=2, n_vis=[400, 330], text_lens=[40, 150], H=2, keep_k=50, seed=110, centres=8)
+    for b, where in ((0, 300), (1, 200)):
+        row = int(batch.cu_seqlens[b]) + int(batch.vis_start[b]) + where
+        batch.k[row] = (batch.k[row].float() * 300.0).to(torch.bfloat16)
+    run_step(ctx, batch, A.Params(keep_k=50))
+
+
 def test_text_longer_than_one_row_tile(ctx):
     batch = W.tiny(B=2, n_vis=[200, 140], text_lens=[150, 129], H=2, keep_k=40, seed=102, centres=8)
     run_step(ctx, batch, A.Params(keep_k=40))
