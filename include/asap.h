@@ -31,8 +31,12 @@
  *     arrays live on the device; the first kernel of each call checks them (spans inside the
  *     sequence, vis_len within [min_vis, max_vis], ascending cu_seqlens, ...) and records a
  *     violation in a device status word that asap_check reads.  A kernel never traps or
- *     spins without bound; every wait in the tensor-core kernels has an iteration limit after
- *     which the status word is set and the block leaves.
+ *     spins without bound; every wait in the tensor-core kernels has a limit (about a second)
+ *     after which a time-out bit is set in the status word and the block leaves, once the copies
+ *     and tensor-core operations it has in flight have completed.  A time-out bit is sticky: every
+ *     result enqueued on the context since it was set is invalid (later tensor-core kernels see the
+ *     bit and leave at once), and the context resumes normal work only after asap_check has
+ *     reported and cleared the word.
  *   - bf16 tensors are row-major with the stated shapes and no padding.
  *   - A context serves one stream at a time: two calls on the same context that overlap on
  *     the GPU race on its scratch memory.
@@ -265,7 +269,16 @@ asap_status asap_select_static(const asap_inputs *in, const asap_params *p, cons
 typedef struct {
   char name[32];     /* kernel name: "qsum", "mass_salience", "score", "select", "sim", ... */
   uint64_t launches; /* launches timed since profiling was enabled */
-  double total_ms;   /* sum over those launches of (next event - this kernel's event) */
+  double total_ms;   /* Diagnostics for the bounded waits of the tensor-core kernels (conventions above; the paper has no
+ * counterpart).  The next call of an entry point on this context -- and only that call -- runs with
+ * `cycles` clock cycles as the limit of every wait, instead of about a second.  With a limit of a few
+ * cycles a healthy run gives up at its first wait that is not satisfied at once: the call returns
+ * normally, its results are invalid, and asap_check reports ASAP_ERR_DEVICE with the kernel's
+ * time-out bit.  This is how the give-up path is exercised without making anything hang.  cycles must
+ * be positive. */
+asap_status asap_debug_wait_limit(asap_ctx *ctx, long long cycles);
+
+/* sum over those launches of (next event - this kernel's event) */
 } asap_kernel_time;
 asap_status asap_profile(asap_ctx *ctx, int enable);
 

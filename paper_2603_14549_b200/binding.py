@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "ASAP_OK", -1: "ASAP_ERR_INVALID", -2: "ASAP_ERR_ALIGN", -3: 
                 -4: "ASAP_ERR_CUDA", -5: "ASAP_ERR_UNSUPPORTED", -6: "ASAP_ERR_DEVICE"}
 
 EXPORTS = ("asap_init", "asap_score", "asap_select", "asap_merge", "asap_prune_step", "asap_check",
-           "asap_last_error", "asap_launch_count", "asap_free", "asap_profile", "asap_profile_read", "asap_select_static", "asap_compact_kv",
+           "asap_last_error", "asap_launch_count", "asap_free", "asap_profile", "asap_profile_read", "asap_debug_wait_limit", "asap_select_static", "asap_compact_kv",
            "asap_consolidate", "asap_consolidate_scratch_bytes", "asap_attention", "asap_attention_scratch_bytes")
 
 
@@ -111,6 +111,8 @@ def load_library() -> C.CDLL:
     lib.asap_launch_count.argtypes = [C.c_void_p]
     lib.asap_profile.restype = C.c_int
     lib.asap_profile.argtypes = [C.c_void_p, C.c_int]
+    lib.asap_debug_wait_limit.restype = C.c_int
+    lib.asap_debug_wait_limit.argtypes = [C.c_void_p, C.c_longlong]
     lib.asap_profile_read.restype = C.c_int
     lib.asap_profile_read.argtypes = [C.c_void_p, C.POINTER(CKernelTime), C.c_int]
     lib.asap_free.restype = None
@@ -332,6 +334,10 @@ def asap_launch_count(ctx) -> int:
 def asap_last_error(ctx) -> str:
     text = load_library().asap_last_error(ctx)
     return text.decode() if text else ""
+
+
+def asap_debug_wait_limit(ctx, cycles: int) -> None:
+    _raise(ctx, load_library().asap_debug_wait_limit(ctx, int(cycles)))
 
 
 def asap_profile(ctx, enable: bool) -> None:

@@ -52,6 +52,8 @@ struct asap_ctx {
   cudaStream_t side = nullptr;            // second stream for the mass kernels of asap_prune_step
   cudaEvent_t ev_fork = nullptr, ev_desc = nullptr, ev_join = nullptr;
   uint64_t launches = 0;
+  long long wait_limit = TC_WAIT_LIMIT;   // clock cycles a wait of the tensor-core kernels may take (asap_debug_wait_limit)
+  size_t counters_off = 0, counters_bytes = 0, tiles_off = 0, tiles_bytes = 0;   // the kernels' hand-shake counters in the arena
   char err[512] = "";
   // per-kernel timing (asap_profile): one event before every launch, one at the end of a call
   bool prof_on = false;
@@ -189,6 +191,7 @@ asap_status after_launch(asap_ctx *ctx, const char *what) {
 
 asap_status finish(asap_ctx *ctx, asap_status result, cudaStream_t st) {
   mark(ctx, nullptr, st);
+  ctx->wait_limit = TC_WAIT_LIMIT;      // a limit set by asap_debug_wait_limit holds for one call
   return result;
 }
 
@@ -267,7 +270,7 @@ asap_status launch_rank(asap_ctx *ctx, const asap_inputs *in, const asap_params 
   sa.mask_log = p->per_head_mask ? out->mask_log_heads : out->mask_log;
   sa.mask_b_stride = p->per_head_mask ? in->H * in->max_vis : in->max_vis;
   sa.mask_h_stride = p->per_head_mask ? in->max_vis : 0;
-  sa.partial = ctx->score_partial; sa.work = ctx->cnt_work; sa.status = ctx->status;
+  sa.partial = ctx->score_partial; sa.work = ctx->cnt_work; sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
   mark(ctx, "score", st);
   const int items = B * in->H;
   launch_pdl(score_kernel, dim3(items < ctx->num_sms ? items : ctx->num_sms), dim3(SC_THREADS), SC_SMEM_BYTES, st,
@@ -389,7 +392,7 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     sa.tile_counters = ctx->cnt_tiles; sa.part = ctx->sim_part;
     sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
     sa.smat = nullptr;
-    sa.status = ctx->status;
+    sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
     mark(ctx, "sim", st);
     if (gather_rows)
       launch_pdl(sim_kernel<true>, dim3(max_mt * groups, B, splits), dim3(SIM_THREADS), smem, st, map_h, map_kept, sa);
@@ -484,7 +487,7 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   sa.drop_idx = nullptr; sa.role = nullptr; sa.hidden = nullptr; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
   sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr; sa.tile_counters = ctx->cnt_tiles;
   sa.part = ctx->sim_part; sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
-  sa.smat = smat; sa.status = ctx->status;
+  sa.smat = smat; sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
   mark(ctx, "sim_kept", st);
   launch_pdl(sim_kernel<false>, dim3(max_mt, B, splits), dim3(SIM_THREADS_TILED), smem, st, map_a, map_b, sa);
   ASAP_TRY(after_launch(ctx, "sim_kept"));
@@ -581,6 +584,8 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   ctx->score_partial = reinterpret_cast<float *>(ctx->arena + o_spart);
   ctx->inv_norm = reinterpret_cast<float *>(ctx->arena + o_inv);
   ctx->kept_inv = reinterpret_cast<float *>(ctx->arena + o_kinv);
+  ctx->counters_off = o_cnt; ctx->counters_bytes = (Bc * col_blocks + 3 * Bc + 2) * sizeof(unsigned int);
+  ctx->tiles_off = o_tiles; ctx->tiles_bytes = ctx->cap_tiles * sizeof(unsigned int);
   ctx->cnt_qsum = reinterpret_cast<unsigned int *>(ctx->arena + o_cnt);
   ctx->cnt_mass = ctx->cnt_qsum + Bc * col_blocks;
   ctx->cnt_score = ctx->cnt_mass + Bc;
@@ -690,6 +695,7 @@ asap_status asap_attention(asap_ctx *ctx, const asap_inputs *in, const asap_para
   aa.desc = ctx->desc; aa.H = in->H; aa.D = D; aa.max_vis = in->max_vis; aa.mask_enable = p->mask_enable ? 1 : 0;
   aa.scale_log2 = 1.4426950408889634f / sqrtf((float)in->head_dim);
   aa.mask_log = mask_log; aa.out = static_cast<__nv_bfloat16 *>(out); aa.status = ctx->status;
+  aa.wait_limit = ctx->wait_limit;
   aa.mask_b_stride = p->per_head_mask ? in->H * in->max_vis : in->max_vis;
   aa.mask_h_stride = p->per_head_mask ? in->max_vis : 0;
   mark(ctx, "attention", st);
@@ -801,6 +807,11 @@ asap_status asap_check(asap_ctx *ctx, void *stream) {
   if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "asap_check: %s", cudaGetErrorString(e));
   if (word == 0) { ctx->err[0] = 0; return ASAP_OK; }
   cudaMemsetAsync(ctx->status, 0, sizeof(uint32_t), st);
+  if (word & (STATUS_SCORE_TIMEOUT | STATUS_SIM_TIMEOUT | STATUS_ATTN_TIMEOUT)) {
+    // blocks that gave up did not finish the hand-shakes that leave the counters at zero
+    cudaMemsetAsync(ctx->arena + ctx->counters_off, 0, ctx->counters_bytes, st);
+    cudaMemsetAsync(ctx->arena + ctx->tiles_off, 0, ctx->tiles_bytes, st);
+  }
   cudaStreamSynchronize(st);
   return fail(ctx, ASAP_ERR_DEVICE, "device status 0x%x:%s%s%s%s%s", word,
               (word & STATUS_BAD_SAMPLE) ? " a per-sample span failed validation (sample skipped);" : "",
@@ -808,6 +819,13 @@ asap_status asap_check(asap_ctx *ctx, void *stream) {
               (word & STATUS_SCORE_TIMEOUT) ? " a wait timed out in the score kernel;" : "",
               (word & STATUS_SIM_TIMEOUT) ? " a wait timed out in the similarity kernel;" : "",
               (word & STATUS_ATTN_TIMEOUT) ? " a wait timed out in the attention kernel;" : "");
+}
+
+asap_status asap_debug_wait_limit(asap_ctx *ctx, long long cycles) {
+  if (!ctx) return fail(nullptr, ASAP_ERR_INVALID, "null context");
+  if (cycles <= 0) return fail(ctx, ASAP_ERR_INVALID, "asap_debug_wait_limit: cycles must be positive");
+  ctx->wait_limit = cycles;
+  return ASAP_OK;
 }
 
 asap_status asap_profile(asap_ctx *ctx, int enable) {

@@ -115,16 +115,15 @@ struct WaitCtx {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx &w) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  uint32_t spins = 0;
   while (true) {
+    // (a try_wait that fails has itself waited for a while inside the hardware, so looking at the
+    // flag and the clock after every one costs nothing that matters)
     if (mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 63u) == 0u) {
-      if (*w.abort_flag) return false;
-      if (clock64() - t0 > w.limit) {
-        *w.abort_flag = 1;
-        atomicOr(w.status, w.status_bit);
-        return false;
-      }
+    if (*w.abort_flag) return false;
+    if (clock64() - t0 > w.limit) {
+      *w.abort_flag = 1;
+      atomicOr(w.status, w.status_bit);
+      return false;
     }
   }
 }

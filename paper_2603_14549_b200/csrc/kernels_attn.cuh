@@ -85,10 +85,11 @@ struct AttnArgs {
   int mask_b_stride, mask_h_stride;   // max_vis, 0   or   H * max_vis, max_vis
   __nv_bfloat16 *out;          // [tokens, H, 128]
   uint32_t *status;
+  long long wait_limit;        // clock cycles a wait may take before the block gives up
 };
 
 struct AttnBook {
-  uint64_t full[AT_STAGES], empty[AT_STAGES], q_full, s_full[2], p_ready[2], pv_done[2];
+  uint64_t full[AT_STAGES], empty[AT_STAGES], q_full, s_full[2], p_ready[2], pv_done[2], mma_done;
   uint32_t tmem_base;
   int abort_flag;
   alignas(16) float m_tile[2][128];   // [row tile][key]: Eq. 3's addend for the keys of the current tile
@@ -146,6 +147,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
       mbar_init(smem_u32(&bk->s_full[g]), 1);
       mbar_init(smem_u32(&bk->p_ready[g]), 256);
       mbar_init(smem_u32(&bk->pv_done[g]), 1);
+      if (g == 0) mbar_init(smem_u32(&bk->mma_done), 1);
     }
     bk->abort_flag = 0;
     fence_barrier_init();
@@ -181,7 +183,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bk->tmem_base;
-  WaitCtx wc{&bk->abort_flag, a.status, STATUS_ATTN_TIMEOUT, AT_WAIT_LIMIT};
+  WaitCtx wc{&bk->abort_flag, a.status, STATUS_ATTN_TIMEOUT, a.wait_limit};
 
   if (warp == 0) {
     if (lane == 0) {
@@ -250,6 +252,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         }
         if (!bk->abort_flag) tc_commit(smem_u32(&bk->empty[s]));
       }
+      // every MMA this thread issued has completed before tensor memory is given back: after an abort the
+      // softmax warps no longer wait for S or P V, so nothing else would hold the block until then
+      tc_commit(smem_u32(&bk->mma_done));
+      mbar_wait_drain(smem_u32(&bk->mma_done), 0, AT_WAIT_LIMIT);
     }
   } else {
     // Two threads per query row: warps w and w + 4 of a group own the same 32 rows (tensor-memory

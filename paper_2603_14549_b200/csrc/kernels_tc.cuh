@@ -79,6 +79,7 @@ struct ScoreArgs {
   float *partial;             // [B, H, max_vis] per-head sums over ranking rows
   unsigned int *work;         // [2] next item / blocks that have finished; both zero between launches
   uint32_t *status;
+  long long wait_limit;       // clock cycles a wait may take before the block gives up
 };
 
 struct ScoreBook {             // bookkeeping block placed after the tiles in shared memory
@@ -164,7 +165,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bk->tmem_base;
-  WaitCtx wc{&bk->abort_flag, a.status, STATUS_SCORE_TIMEOUT, TC_WAIT_LIMIT};
+  WaitCtx wc{&bk->abort_flag, a.status, STATUS_SCORE_TIMEOUT, a.wait_limit};
   if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SCORE_TIMEOUT) bk->abort_flag = 1;   // benign race: same value
   __syncthreads();
 
@@ -178,7 +179,12 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                                                 // these are prefixes of the two sequences)
       while (true) {
         const int slot = ic % SC_ITEM_SLOTS;
-        if (ic >= SC_ITEM_SLOTS) mbar_wait(smem_u32(&bk->item_empty[slot]), ((ic / SC_ITEM_SLOTS) - 1) & 1, wc);
+        // The item queue keeps working after an abort (its waits ignore the flag and are bounded on their
+        // own): every consumer must see the same sequence of items, ending with -1, or the epilogue warps'
+        // named barriers would no longer match.  After an abort that sequence ends at once.
+        if (ic >= SC_ITEM_SLOTS &&
+            !mbar_wait_drain(smem_u32(&bk->item_empty[slot]), ((ic / SC_ITEM_SLOTS) - 1) & 1, TC_WAIT_LIMIT))
+          break;
         int item = bk->abort_flag ? n_items : (int)atomicAdd(a.work, 1u);
         if (item >= n_items) item = -1;
         bk->item_q[slot] = item;
@@ -229,8 +235,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       const uint32_t idesc1 = umma_idesc_bf16(128, 128);
       while (true) {
         const int slot = ic % SC_ITEM_SLOTS;
-        mbar_wait(smem_u32(&bk->item_full[slot]), (ic / SC_ITEM_SLOTS) & 1, wc);
-        const int item = bk->abort_flag ? -1 : bk->item_q[slot];
+        const bool got = mbar_wait_drain(smem_u32(&bk->item_full[slot]), (ic / SC_ITEM_SLOTS) & 1, TC_WAIT_LIMIT);
+        const int item = got ? bk->item_q[slot] : -1;
         mbar_arrive(smem_u32(&bk->item_empty[slot]));
         ++ic;
         if (item < 0) break;
@@ -293,8 +299,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     int g = 0, ic = 0;
     while (true) {
       const int slot = ic % SC_ITEM_SLOTS;
-      mbar_wait(smem_u32(&bk->item_full[slot]), (ic / SC_ITEM_SLOTS) & 1, wc);
-      const int item = bk->abort_flag ? -1 : bk->item_q[slot];
+      const bool got = mbar_wait_drain(smem_u32(&bk->item_full[slot]), (ic / SC_ITEM_SLOTS) & 1, TC_WAIT_LIMIT);
+      const int item = got ? bk->item_q[slot] : -1;
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bk->item_empty[slot]));
       ++ic;
@@ -626,10 +632,11 @@ struct SimArgs {
   float *ss_part;            // [B, max_mt, splits, 128]         partial squared norms
   float *smat;               // [B, keep_k, keep_k] or nullptr: matrix mode
   uint32_t *status;
+  long long wait_limit;      // clock cycles a wait may take before the block gives up
 };
 
 struct SimBook {
-  uint64_t full[SIM_MAX_STAGES], empty[SIM_MAX_STAGES], acc_full[2], acc_empty[2];
+  uint64_t full[SIM_MAX_STAGES], empty[SIM_MAX_STAGES], acc_full[2], acc_empty[2], mma_done;
   uint32_t tmem_base;
   int abort_flag;
   int is_last;
@@ -687,6 +694,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       mbar_init(smem_u32(&bk->acc_full[i]), 1);
       mbar_init(smem_u32(&bk->acc_empty[i]), 4);
     }
+    mbar_init(smem_u32(&bk->mma_done), 1);
     bk->abort_flag = 0;
     bk->is_last = 0;
     fence_barrier_init();
@@ -699,7 +707,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bk->tmem_base;
-  WaitCtx wc{&bk->abort_flag, a.status, STATUS_SIM_TIMEOUT, TC_WAIT_LIMIT};
+  WaitCtx wc{&bk->abort_flag, a.status, STATUS_SIM_TIMEOUT, a.wait_limit};
   // steps of this slice: 128 columns each, or 64 in the one-pass layout
   const int n_kb = a.wide ? (a.D / 64) / a.splits : (a.D / 128) / a.splits;
   const int kb0 = z * n_kb;
@@ -743,7 +751,9 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       for (int s = 0; s < a.stages; ++s) {
         if (issued > s) {
           const int last = ((issued - 1 - s) / a.stages) * a.stages + s;
-          mbar_wait_drain(smem_u32(&bk->full[s]), (last / a.stages) & 1, TC_WAIT_LIMIT);
+          // after an abort the gather warps may not have handed their part of the stage over, so the
+          // barrier may never complete: the tiled copies themselves land within microseconds
+          mbar_wait_drain(smem_u32(&bk->full[s]), (last / a.stages) & 1, bk->abort_flag ? 400000LL : TC_WAIT_LIMIT);
         }
       }
     }
@@ -839,6 +849,10 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         }
         if (!bk->abort_flag) tc_commit(smem_u32(&bk->acc_full[buf]));
       }
+      // every MMA this thread issued has completed before tensor memory is given back: after an abort the
+      // epilogue warps no longer wait for the accumulators, so nothing else would hold the block until then
+      tc_commit(smem_u32(&bk->mma_done));
+      mbar_wait_drain(smem_u32(&bk->mma_done), 0, TC_WAIT_LIMIT);
     }
   } else {
     const int quarter = warp & 3;
