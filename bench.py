@@ -460,7 +460,7 @@ def run_cuda(args):
     peaks, peak_kind = load_peaks()
 
     seed = R.replica_seed(W.BASE_SEED + int(args.workload[1]) - 1, rank)
-    batch = W.config(args.workload, seed=seed)
+    batch = W.config(args.workload, B=args.sequences, seed=seed)
     keep_k = batch.keep_k
     stream = torch.cuda.Stream(device=device)     # a stream of our own: the legacy stream cannot be captured
     torch.cuda.set_stream(stream)
@@ -546,9 +546,44 @@ def run_cuda(args):
               "GBs": kv_bytes / kv_us / 1e3, "frac_of_hbm_peak": kv_bytes / kv_us / 1e3 / peaks["hbm_gbs"],
               "roofline": {"kernel": "gather_rows", "bound": "hbm", "achieved": kv_bytes / kv_us / 1e3,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": kv_bytes / kv_us / 1e3 / peaks["hbm_gbs"],
-                           "traffic": load_traffic(args.workload).get("gather_rows"), "peak_kind": peak_kind},
+                           "traffic": (load_traffic(args.workload).get("gather_rows_per_tensor") or 0) * n_t or None,
+                           "peak_kind": peak_kind},
               "storage": F.kv_storage_bytes(batch.total, n_out, args.kv_layers, batch.D)}
         del kv_src, kv_dst
+
+    # ---- the three stages called one by one (asap_score / asap_select / asap_merge, and the score with one
+    # mask per head): the kernels only these entry points launch (head_sum, prepare, role_map, mass_heads)
+    staged = None
+    if solo and args.staged_iters > 0:
+        out_h = A.alloc_outputs(copies[0], keep_k, per_head=True) if batch.H % 2 == 0 else None
+        p_h = dataclasses.replace(params, per_head_mask=True)
+        sal, kidx, didx, rsc = (x.clone() for x in (out.salience, out.keep_idx, out.drop_idx, out.rank_score))
+
+        def staged_call(i):
+            c = copies[i % n_copies]
+            A.asap_score(ctx, c, params, out, stream)
+            A.asap_select(ctx, c, params, rsc, out, stream)
+            A.asap_merge(ctx, c, params, sal, kidx, didx, out, stream)
+            if out_h is not None:
+                A.asap_score(ctx, c, p_h, out_h, stream)
+        for i in range(2):
+            staged_call(i)
+        torch.cuda.synchronize()
+        A.asap_check(ctx)
+        A.asap_profile(ctx, True)
+        for i in range(args.staged_iters):
+            staged_call(i)
+        torch.cuda.synchronize()
+        sk = {name: ms / max(n, 1) * 1e3 for name, (n, ms) in A.asap_profile_read(ctx).items()}
+        A.asap_profile(ctx, False)
+        hs_bytes = sum(batch.H * int(v) * 4 + int(v) * 4 for v in batch.vis_len)
+        mh_bytes = sum(int(v) * batch.D * 2 + 2 * batch.H * int(v) * 4 for v in batch.vis_len)
+        staged = {"calls": "asap_score, asap_select, asap_merge, asap_score(per_head_mask)", "kernel_us": sk,
+                  "head_sum_GBs": hs_bytes / sk["head_sum"] / 1e3 if sk.get("head_sum") else None,
+                  "mass_heads_GBs": mh_bytes / sk["mass_heads"] / 1e3 if sk.get("mass_heads") else None}
+        A.asap_prune_step(ctx, copies[0], params, out, stream)     # the later legs use the step's own results
+        torch.cuda.synchronize()
+        del out_h
 
     # ---- stage 2 as Sec. 4.2 words it (routing inside the kept set, refill by attention mass), timed
     # apart from the step on the step's own stage-1 results
@@ -734,7 +769,9 @@ def run_cuda(args):
         "metric": METRIC, "value": units_all / step_s, "unit": UNIT, "n_gpus": size, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}", "sequences_per_gpu": batch.B,
+        "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}" +
+                               (f" -- PREFIX of {batch.B} sequences" if args.sequences else ""),
+                   "sequences_per_gpu": batch.B,
                    "visual_tokens_per_gpu": units, "keep_k": keep_k, "ranking_rows": "image span + text span" if rank_visual else "text span",
                    "l2": (f"inputs rotate over {n_copies} device copies ({n_copies * S.in_bytes / 2**20:.0f} MiB) "
                           f"so no step finds its inputs in the {L2_BYTES // 2**20} MiB L2"),
@@ -744,7 +781,7 @@ def run_cuda(args):
                        "p90": per_step[(len(per_step) * 9) // 10] * 1e3, "samples": len(per_step)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": t["launches"], "roofline": roofline, "kernels": kernels,
         "sustained": sustained, "other_workloads": others,
-        "cpu_baseline": cpu, "kv_compaction": kv, "consolidate_within_kept": cons, "masked_attention": attn, "direct_launch": direct,
+        "cpu_baseline": cpu, "kv_compaction": kv, "staged_entry_points": staged, "consolidate_within_kept": cons, "masked_attention": attn, "direct_launch": direct,
     }
     print(json.dumps(line))
     R.shutdown()
@@ -798,6 +835,8 @@ def main():
     ap.add_argument("--workload", default="c4", choices=sorted(WORKLOADS))
     ap.add_argument("--rank-rows", default="text", choices=["text", "visual+text"],
                     help="query rows whose Eq. 4 probabilities rank the visual keys (default: the text span)")
+    ap.add_argument("--sequences", type=int, default=None,
+                    help="only the first N sequences of the workload (profiling captures; the line's config says so)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=12, help="timed end-to-end steps (at most --steps)")
     ap.add_argument("--kv-layers", type=int, default=3,
@@ -807,6 +846,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time directly launched steps instead of graph replays")
     ap.add_argument("--direct-steps", type=int, default=50,
                     help="also time this many directly launched steps when the headline is a graph replay (0 = skip)")
+    ap.add_argument("--staged-iters", type=int, default=5,
+                    help="also call asap_score / asap_select / asap_merge one by one this many times (0 = skip)")
     ap.add_argument("--consolidate-iters", type=int, default=20, help="timed asap_consolidate calls (0 = skip)")
     ap.add_argument("--attention-iters", type=int, default=5,
                     help="also time asap_attention (the layer's attention under the SG-BiMask) this many times (0 = skip)")

@@ -417,13 +417,18 @@ asap_status launch_merge_back(asap_ctx *ctx, const asap_inputs *in, const asap_p
   ma.out_pos = out->out_pos; ma.src_row = out->src_row;
   const int copy_rows = in->max_seq - in->min_vis;   // prefix + suffix rows of the longest sequence, at most
   const dim3 grid(k + (copy_rows + MERGE_COPY_ROWS - 1) / MERGE_COPY_ROWS, B);
-  const int nv = (D / 8 + MERGE_THREADS - 1) / MERGE_THREADS;
+  // Block width: 256 threads unless a wider block covers the row's 16-byte vectors with fewer idle lanes
+  // (D = 5120: 640 vectors = 2 x 320 instead of 2.5 x 256).
+  const int vecs = D / 8;
+  int threads = MERGE_THREADS;
+  if (vecs % MERGE_MAX_THREADS == 0 && vecs % MERGE_THREADS != 0) threads = MERGE_MAX_THREADS;
+  const int nv = (vecs + threads - 1) / threads;
   mark(ctx, "merge_compact", st);
   switch (nv) {
-    case 1: launch_pdl(merge_compact_kernel<1>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
-    case 2: launch_pdl(merge_compact_kernel<2>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
-    case 3: launch_pdl(merge_compact_kernel<3>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
-    default: launch_pdl(merge_compact_kernel<4>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
+    case 1: launch_pdl(merge_compact_kernel<1>, dim3(grid), dim3(threads), 0, st, ma); break;
+    case 2: launch_pdl(merge_compact_kernel<2>, dim3(grid), dim3(threads), 0, st, ma); break;
+    case 3: launch_pdl(merge_compact_kernel<3>, dim3(grid), dim3(threads), 0, st, ma); break;
+    default: launch_pdl(merge_compact_kernel<4>, dim3(grid), dim3(threads), 0, st, ma); break;
   }
   return after_launch(ctx, "merge_compact");
 }

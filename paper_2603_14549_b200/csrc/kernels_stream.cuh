@@ -1120,7 +1120,8 @@ route_kernel(RouteArgs a) {
 //   blockIdx.x >= keep_k : each warp copies one prefix / suffix row.
 // Every output row also gets its gathered position id and its source row (hand-off of Fig. 3).
 // =======================================================================================
-constexpr int MERGE_THREADS = 256;
+constexpr int MERGE_THREADS = 256;                    // default block; the launch may pick a width that divides the row
+constexpr int MERGE_MAX_THREADS = 320;
 constexpr int MERGE_COPY_ROWS = MERGE_THREADS / 32;   // copy rows per block
 constexpr int MERGE_LIST = 256;                        // members listed per pass
 constexpr int MERGE_BATCH = 4;                         // member rows in flight per thread
@@ -1137,8 +1138,8 @@ struct MergeArgs {
   int32_t *out_pos, *src_row;
 };
 
-template <int NV>   // 16-byte vectors per thread: D <= NV * 256 * 8
-__global__ void __launch_bounds__(MERGE_THREADS)
+template <int NV>   // 16-byte vectors per thread: D <= NV * blockDim.x * 8
+__global__ void __launch_bounds__(MERGE_MAX_THREADS)
 merge_compact_kernel(MergeArgs a) {
   pdl_enter();
   __shared__ int s_j[MERGE_LIST];
@@ -1152,7 +1153,7 @@ merge_compact_kernel(MergeArgs a) {
     // ---------------------------------------------------------------- copy rows, one per warp
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int c = ((int)blockIdx.x - k) * MERGE_COPY_ROWS + warp;     // index among prefix + suffix rows
-    if (c >= d.n - d.nv) return;
+    if (warp >= MERGE_COPY_ROWS || c >= d.n - d.nv) return;
     const int srow = c < d.v0 ? c : c + d.nv;
     const int orow = d.out_row0 + (c < d.v0 ? c : c + k);
     const size_t grow = (size_t)(d.row0 + srow);
@@ -1193,13 +1194,13 @@ merge_compact_kernel(MergeArgs a) {
   uint4 self[NV];
 #pragma unroll
   for (int u = 0; u < NV; ++u) {
-    const int v = threadIdx.x + u * MERGE_THREADS;
+    const int v = threadIdx.x + u * blockDim.x;
     if (v < nvec) self[u] = __ldg(src + v);
   }
   if (m_hi <= m_lo) {
 #pragma unroll
     for (int u = 0; u < NV; ++u) {
-      const int v = threadIdx.x + u * MERGE_THREADS;
+      const int v = threadIdx.x + u * blockDim.x;
       if (v < nvec) dst[v] = self[u];
     }
     return;
@@ -1235,7 +1236,7 @@ merge_compact_kernel(MergeArgs a) {
           const uint4 *msrc = reinterpret_cast<const uint4 *>(vis0 + (size_t)s_j[m0 + t] * a.D);
 #pragma unroll
           for (int u = 0; u < NV; ++u) {
-            const int v = threadIdx.x + u * MERGE_THREADS;
+            const int v = threadIdx.x + u * blockDim.x;
             if (v < nvec) x[t][u] = __ldg(msrc + v);
           }
         }
@@ -1259,14 +1260,14 @@ merge_compact_kernel(MergeArgs a) {
   if (den <= a.eps) {
 #pragma unroll
     for (int u = 0; u < NV; ++u) {
-      const int v = threadIdx.x + u * MERGE_THREADS;
+      const int v = threadIdx.x + u * blockDim.x;
       if (v < nvec) dst[v] = self[u];
     }
   } else {
     const float inv = 1.0f / den;
 #pragma unroll
     for (int u = 0; u < NV; ++u) {
-      const int v = threadIdx.x + u * MERGE_THREADS;
+      const int v = threadIdx.x + u * blockDim.x;
       if (v < nvec) {
         uint4 o;
         o.x = pack2_rn(acc[u][0] * inv, acc[u][1] * inv);
