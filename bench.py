@@ -92,7 +92,7 @@ def algorithmic(batch, keep_k, rank_visual=False):
     every operand it consumes read once, every result written once (bf16 = 2 bytes)."""
     D = batch.D
     out = {name: {"bytes": 0, "flops": 0} for name in
-           ("qsum", "mass_salience", "score", "head_sum", "select", "kept_gather", "sim", "merge_compact",
+           ("qsum", "mass_salience", "salience", "score", "head_sum", "select", "kept_gather", "sim", "merge_compact",
             "prepare", "role_map")}
     for b in range(batch.B):
         n = int(batch.cu_seqlens[b + 1] - batch.cu_seqlens[b])
@@ -103,6 +103,7 @@ def algorithmic(batch, keep_k, rank_visual=False):
         out["qsum"]["flops"] += nv * D
         out["mass_salience"]["bytes"] += nv * row + nv * 12
         out["mass_salience"]["flops"] += 2 * nv * D
+        out["salience"]["bytes"] += batch.H * nv * 4 + nv * 12      # per-head masses in, mass / salience / mask out
         # ranking rows = text span: queries once, every key they may attend to once
         out["score"]["bytes"] += tl * row + (t0 + tl) * row + nv * 4
         out["score"]["flops"] += 2 * tl * (t0 + (tl + 1) // 2) * D

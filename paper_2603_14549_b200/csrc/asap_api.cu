@@ -5,6 +5,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -43,6 +44,8 @@ struct asap_ctx {
         *kept_inv = nullptr;
   unsigned int *cnt_qsum = nullptr, *cnt_mass = nullptr, *cnt_score = nullptr, *cnt_sim = nullptr,
                *cnt_tiles = nullptr, *cnt_work = nullptr;
+  float *mass_partial = nullptr;    // [B, H, max_vis] per-head attention masses written by the score kernel
+  long long fuse_mass_min_tokens = 50000;   // B * max_vis from which the attention mass rides in the score kernel
   float *sim_part = nullptr;        // partial dot products / squared norms of a sliced similarity GEMM
   size_t sim_part_bytes = 0, cap_tiles = 0;
   int32_t *role = nullptr, *seg = nullptr, *members = nullptr;
@@ -258,7 +261,7 @@ asap_status launch_mass(asap_ctx *ctx, const asap_inputs *in, const asap_params 
 
 // Steps 1c-2: Eq. 4 probabilities of the ranking rows, summed per head; optionally the head sum.
 asap_status launch_rank(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const asap_outputs *out,
-                        bool with_head_sum, cudaStream_t st) {
+                        bool with_head_sum, cudaStream_t st, bool with_mass = false) {
   const int D = in->D, B = in->B;
   CUtensorMap map_q, map_k;
   if (!make_map(ctx, &map_q, in->q, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
@@ -270,6 +273,7 @@ asap_status launch_rank(asap_ctx *ctx, const asap_inputs *in, const asap_params 
   sa.mask_log = p->per_head_mask ? out->mask_log_heads : out->mask_log;
   sa.mask_b_stride = p->per_head_mask ? in->H * in->max_vis : in->max_vis;
   sa.mask_h_stride = p->per_head_mask ? in->max_vis : 0;
+  sa.qbar = with_mass ? ctx->qbar : nullptr; sa.mass_heads = ctx->mass_partial; sa.D = D;
   sa.partial = ctx->score_partial; sa.work = ctx->cnt_work; sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
   mark(ctx, "score", st);
   const int items = B * in->H;
@@ -417,18 +421,13 @@ asap_status launch_merge_back(asap_ctx *ctx, const asap_inputs *in, const asap_p
   ma.out_pos = out->out_pos; ma.src_row = out->src_row;
   const int copy_rows = in->max_seq - in->min_vis;   // prefix + suffix rows of the longest sequence, at most
   const dim3 grid(k + (copy_rows + MERGE_COPY_ROWS - 1) / MERGE_COPY_ROWS, B);
-  // Block width: 256 threads unless a wider block covers the row's 16-byte vectors with fewer idle lanes
-  // (D = 5120: 640 vectors = 2 x 320 instead of 2.5 x 256).
-  const int vecs = D / 8;
-  int threads = MERGE_THREADS;
-  if (vecs % MERGE_MAX_THREADS == 0 && vecs % MERGE_THREADS != 0) threads = MERGE_MAX_THREADS;
-  const int nv = (vecs + threads - 1) / threads;
+  const int nv = (D / 8 + MERGE_THREADS - 1) / MERGE_THREADS;
   mark(ctx, "merge_compact", st);
   switch (nv) {
-    case 1: launch_pdl(merge_compact_kernel<1>, dim3(grid), dim3(threads), 0, st, ma); break;
-    case 2: launch_pdl(merge_compact_kernel<2>, dim3(grid), dim3(threads), 0, st, ma); break;
-    case 3: launch_pdl(merge_compact_kernel<3>, dim3(grid), dim3(threads), 0, st, ma); break;
-    default: launch_pdl(merge_compact_kernel<4>, dim3(grid), dim3(threads), 0, st, ma); break;
+    case 1: launch_pdl(merge_compact_kernel<1>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
+    case 2: launch_pdl(merge_compact_kernel<2>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
+    case 3: launch_pdl(merge_compact_kernel<3>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
+    default: launch_pdl(merge_compact_kernel<4>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
   }
   return after_launch(ctx, "merge_compact");
 }
@@ -566,6 +565,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   const size_t o_qpart = carve(ctx->cap_chunks * Dc * sizeof(float));
   const size_t o_qbar = carve(Bc * Dc * sizeof(float));
   const size_t o_spart = carve(Hc * T * sizeof(float));
+  const size_t o_mpart = carve(Hc * T * sizeof(float));
   const size_t o_inv = carve(T * sizeof(float));
   const size_t o_kinv = carve(max_keep_rows * sizeof(float));
   const size_t o_cnt = carve((Bc * col_blocks + 3 * Bc + 2) * sizeof(unsigned int));
@@ -587,6 +587,8 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   ctx->qsum_partial = reinterpret_cast<float *>(ctx->arena + o_qpart);
   ctx->qbar = reinterpret_cast<float *>(ctx->arena + o_qbar);
   ctx->score_partial = reinterpret_cast<float *>(ctx->arena + o_spart);
+  ctx->mass_partial = reinterpret_cast<float *>(ctx->arena + o_mpart);
+  if (const char *env = getenv("ASAP_FUSE_MASS_MIN_TOKENS")) ctx->fuse_mass_min_tokens = atoll(env);
   ctx->inv_norm = reinterpret_cast<float *>(ctx->arena + o_inv);
   ctx->kept_inv = reinterpret_cast<float *>(ctx->arena + o_kinv);
   ctx->counters_off = o_cnt; ctx->counters_bytes = (Bc * col_blocks + 3 * Bc + 2) * sizeof(unsigned int);
@@ -743,7 +745,28 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
   // mass kernels then run on the context's side stream next to the score kernel, and rejoin before
   // the merge, which is the first consumer of the salience.  With caller-given ranking rows (which may
   // be visual) and while per-kernel timing is on, everything runs in order on `stream`.
-  const bool overlap = in->rank_start == nullptr && !ctx->prof_on && ctx->side != nullptr && !p->per_head_mask;
+  const bool text_rows = in->rank_start == nullptr && !p->per_head_mask;
+  if (text_rows && (long long)in->B * in->max_vis >= ctx->fuse_mass_min_tokens) {
+    // Large batches: the mass kernels no longer hide beside the score kernel (both are bound by the same
+    // memory system), so Eq. 1's key side is taken from the key tiles the score kernel streams anyway:
+    // query sum (carrying the validation) -> score kernel with two more columns per key tile -> Eq. 2-3.
+    PrepareArgs pa = prepare_args(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity);
+    pa.write_desc = 1;
+    const int max_chunks = (in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS;
+    mark(ctx, "qsum", st);
+    launch_pdl(qsum_kernel, dim3(max_chunks, (in->D + QSUM_COLS - 1) / QSUM_COLS, in->B), dim3(QSUM_THREADS), 0, st,
+               static_cast<const __nv_bfloat16 *>(in->q), pa, in->D, max_chunks, ctx->qsum_partial, ctx->qbar, ctx->cnt_qsum);
+    ASAP_TRY(after_launch(ctx, "qsum"));
+    ASAP_TRY(launch_rank(ctx, in, p, out, false, st, true));
+    mark(ctx, "salience", st);
+    launch_pdl(salience_from_heads_kernel, dim3(in->B), dim3(SAL_THREADS), 0, st, ctx->desc, in->H, in->max_vis,
+               1.0f / ((float)in->H * sqrtf((float)in->head_dim)), p->lambda_max, p->eps, ctx->mass_partial, out->mass,
+               out->salience, out->mask_log, out->rank_score);
+    ASAP_TRY(after_launch(ctx, "salience"));
+    ASAP_TRY(launch_select(ctx, in, p, out->rank_score, out, true, true, st));
+    return finish(ctx, launch_merge(ctx, in, p, out->salience, out->keep_idx, out->drop_idx, out, st), st);
+  }
+  const bool overlap = text_rows && !ctx->prof_on && ctx->side != nullptr;
   if (!overlap) {
     ASAP_TRY(launch_mass(ctx, in, p, out, true, out->out_cu_seqlens, out->out_rows_capacity, st));
     ASAP_TRY(launch_rank(ctx, in, p, out, false, st));

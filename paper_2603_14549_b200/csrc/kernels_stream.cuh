@@ -2,6 +2,7 @@
 //   prepare        device-side validation, per-sample descriptors, output row offsets
 //   qsum           sum of the visual query rows                       (Eq. 1, summed over i first)
 //   mass_salience  s_j, then s_hat_j and m_j                          (Eq. 1, Eq. 2, Eq. 3)
+//   salience_from_heads  the same from per-head masses the score kernel produced
 //   select         stable radix top-k of the ranking scores           (Fig. 3)
 //   role_map       kept slot / dropped position of every visual token
 //   kept_gather    kept rows gathered for the similarity GEMM, with their inverse norms (Sec. 4.2)
@@ -274,6 +275,72 @@ mass_salience_kernel(const __nv_bfloat16 *__restrict__ k, const SampleDesc *__re
   for (int j = threadIdx.x; j < max_vis; j += MASS_THREADS) {
     if (j < d.nv) {
       const float sh = (__ldcg(mass_b + j) - lo) * inv;
+      sal_b[j] = sh;
+      msk_b[j] = logf(fmaxf(lambda_max * sh, eps));
+    } else {
+      mass_b[j] = 0.f; sal_b[j] = 0.f; msk_b[j] = 0.f;
+    }
+  }
+}
+
+// =======================================================================================
+// salience_from_heads: the tail of Eq. 1 and Eq. 2-3 when the per-head masses qbar^h . k_j^h were
+// produced elsewhere (by the score kernel, from the key tiles it streams anyway).  One block per
+// sample: s_j = scale * sum_h heads[b, h, j] (heads in order), then the min-max normalisation and
+// the mask vector over the image span; padding past the span is zeroed as mass_salience does.
+// =======================================================================================
+constexpr int SAL_THREADS = 1024;
+
+__global__ void __launch_bounds__(SAL_THREADS)
+salience_from_heads_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis, float scale, float lambda_max,
+                           float eps, const float *__restrict__ heads /*[B, H, max_vis]*/, float *__restrict__ mass,
+                           float *__restrict__ salience, float *__restrict__ mask_log, float *__restrict__ rank_score) {
+  pdl_enter();
+  __shared__ float s_red[2 * (SAL_THREADS / 32)];
+  const int b = blockIdx.x;
+  const SampleDesc d = desc[b];
+  float *mass_b = mass + (size_t)b * max_vis, *sal_b = salience + (size_t)b * max_vis, *msk_b = mask_log + (size_t)b * max_vis;
+  if (!d.valid) {
+    for (int j = threadIdx.x; j < max_vis; j += SAL_THREADS) {
+      mass_b[j] = 0.f; sal_b[j] = 0.f; msk_b[j] = 0.f;
+      rank_score[(size_t)b * max_vis + j] = 0.f;       // the score and selection kernels skip the sample
+    }
+    return;
+  }
+  const float *hb = heads + (size_t)b * H * max_vis;
+  float lo = INFINITY, hi = -INFINITY;
+  for (int j = threadIdx.x; j < d.nv; j += SAL_THREADS) {
+    float tot = 0.f;
+    int hh = 0;
+    for (; hh + 8 <= H; hh += 8) {            // eight loads in flight
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = __ldcg(hb + (size_t)(hh + e) * max_vis + j);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) tot += v[e];
+    }
+    for (; hh < H; ++hh) tot += __ldcg(hb + (size_t)hh * max_vis + j);
+    tot *= scale;
+    mass_b[j] = tot;
+    lo = fminf(lo, tot); hi = fmaxf(hi, tot);
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+  }
+  if (lane == 0) { s_red[warp] = lo; s_red[SAL_THREADS / 32 + warp] = hi; }
+  __syncthreads();
+  lo = s_red[0]; hi = s_red[SAL_THREADS / 32];
+#pragma unroll
+  for (int w = 1; w < SAL_THREADS / 32; ++w) {
+    lo = fminf(lo, s_red[w]); hi = fmaxf(hi, s_red[SAL_THREADS / 32 + w]);
+  }
+  const float inv = 1.0f / ((hi - lo) + eps);
+  for (int j = threadIdx.x; j < max_vis; j += SAL_THREADS) {
+    if (j < d.nv) {
+      const float sh = (mass_b[j] - lo) * inv;      // this thread's own store above
       sal_b[j] = sh;
       msk_b[j] = logf(fmaxf(lambda_max * sh, eps));
     } else {
@@ -1120,8 +1187,7 @@ route_kernel(RouteArgs a) {
 //   blockIdx.x >= keep_k : each warp copies one prefix / suffix row.
 // Every output row also gets its gathered position id and its source row (hand-off of Fig. 3).
 // =======================================================================================
-constexpr int MERGE_THREADS = 256;                    // default block; the launch may pick a width that divides the row
-constexpr int MERGE_MAX_THREADS = 320;
+constexpr int MERGE_THREADS = 256;
 constexpr int MERGE_COPY_ROWS = MERGE_THREADS / 32;   // copy rows per block
 constexpr int MERGE_LIST = 256;                        // members listed per pass
 constexpr int MERGE_BATCH = 4;                         // member rows in flight per thread
@@ -1138,9 +1204,12 @@ struct MergeArgs {
   int32_t *out_pos, *src_row;
 };
 
-template <int NV>   // 16-byte vectors per thread: D <= NV * blockDim.x * 8
-__global__ void __launch_bounds__(MERGE_MAX_THREADS)
+// NV: 16-byte vectors per thread (D <= NV * 256 * 8); wide rows keep fewer member rows in flight per thread
+// so that three blocks still fit the register file of an SM.
+template <int NV>
+__global__ void __launch_bounds__(MERGE_THREADS, NV >= 4 ? 2 : 3)
 merge_compact_kernel(MergeArgs a) {
+  constexpr int BATCH = NV >= 3 ? 2 : MERGE_BATCH;
   pdl_enter();
   __shared__ int s_j[MERGE_LIST];
   __shared__ float s_w[MERGE_LIST];
@@ -1153,7 +1222,7 @@ merge_compact_kernel(MergeArgs a) {
     // ---------------------------------------------------------------- copy rows, one per warp
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int c = ((int)blockIdx.x - k) * MERGE_COPY_ROWS + warp;     // index among prefix + suffix rows
-    if (warp >= MERGE_COPY_ROWS || c >= d.n - d.nv) return;
+    if (c >= d.n - d.nv) return;
     const int srow = c < d.v0 ? c : c + d.nv;
     const int orow = d.out_row0 + (c < d.v0 ? c : c + k);
     const size_t grow = (size_t)(d.row0 + srow);
@@ -1194,13 +1263,13 @@ merge_compact_kernel(MergeArgs a) {
   uint4 self[NV];
 #pragma unroll
   for (int u = 0; u < NV; ++u) {
-    const int v = threadIdx.x + u * blockDim.x;
+    const int v = threadIdx.x + u * MERGE_THREADS;
     if (v < nvec) self[u] = __ldg(src + v);
   }
   if (m_hi <= m_lo) {
 #pragma unroll
     for (int u = 0; u < NV; ++u) {
-      const int v = threadIdx.x + u * blockDim.x;
+      const int v = threadIdx.x + u * MERGE_THREADS;
       if (v < nvec) dst[v] = self[u];
     }
     return;
@@ -1228,21 +1297,21 @@ merge_compact_kernel(MergeArgs a) {
       s_w[threadIdx.x] = sal_b[j];
     }
     __syncthreads();
-    for (int m0 = 0; m0 < cnt; m0 += MERGE_BATCH) {
-      uint4 x[MERGE_BATCH][NV];
+    for (int m0 = 0; m0 < cnt; m0 += BATCH) {
+      uint4 x[BATCH][NV];
 #pragma unroll
-      for (int t = 0; t < MERGE_BATCH; ++t) {
+      for (int t = 0; t < BATCH; ++t) {
         if (m0 + t < cnt) {
           const uint4 *msrc = reinterpret_cast<const uint4 *>(vis0 + (size_t)s_j[m0 + t] * a.D);
 #pragma unroll
           for (int u = 0; u < NV; ++u) {
-            const int v = threadIdx.x + u * blockDim.x;
+            const int v = threadIdx.x + u * MERGE_THREADS;
             if (v < nvec) x[t][u] = __ldg(msrc + v);
           }
         }
       }
 #pragma unroll
-      for (int t = 0; t < MERGE_BATCH; ++t) {
+      for (int t = 0; t < BATCH; ++t) {
         if (m0 + t < cnt) {
           const float w = s_w[m0 + t];
           den += w;
@@ -1260,14 +1329,14 @@ merge_compact_kernel(MergeArgs a) {
   if (den <= a.eps) {
 #pragma unroll
     for (int u = 0; u < NV; ++u) {
-      const int v = threadIdx.x + u * blockDim.x;
+      const int v = threadIdx.x + u * MERGE_THREADS;
       if (v < nvec) dst[v] = self[u];
     }
   } else {
     const float inv = 1.0f / den;
 #pragma unroll
     for (int u = 0; u < NV; ++u) {
-      const int v = threadIdx.x + u * blockDim.x;
+      const int v = threadIdx.x + u * MERGE_THREADS;
       if (v < nvec) {
         uint4 o;
         o.x = pack2_rn(acc[u][0] * inv, acc[u][1] * inv);

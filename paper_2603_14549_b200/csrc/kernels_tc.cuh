@@ -52,6 +52,13 @@ __device__ __forceinline__ void group_bar_sync(int group) {
 // Additive mask (Eq. 3), logits in log2 units: 0 for key j <= row position p; m_j*log2(e) for
 // j > p when both are in the image span (mask enabled); -inf otherwise.
 // The per-head sums over ranking rows go to `partial`; head_sum_kernel adds them in head order.
+// Attention mass on the way (a.qbar given; ranking rows after the image span): Eq. 1 with the sum over
+// the queries taken first is qbar^h . k_j^h, and pass 2 already multiplies every visual key tile by the
+// row pair's queries.  The summed query rides along as three more "query rows" (its bf16 value, the bf16
+// value of what that rounding lost, and again: 24 bits of mantissa together, all that fp32 holds),
+// written behind the pair's rows in shared memory, so the first row pair's pass-2 accumulators get three
+// more columns whose sum is the key's mass for this head.  Row pairs then hold at most 240 rows (the
+// accumulator grows by the 16 columns an MMA's width moves in).
 // =======================================================================================
 constexpr int SC_THREADS = 320;          // producer warp, MMA warp, 2 x 4 epilogue warps
 constexpr int SC_EPI_THREADS = 256;
@@ -77,6 +84,10 @@ struct ScoreArgs {
   const float *mask_log;      // [B, max_vis] m_j (natural log), or [B, H, max_vis] with a mask per head
   int mask_b_stride, mask_h_stride;   // max_vis, 0   or   H * max_vis, max_vis
   float *partial;             // [B, H, max_vis] per-head sums over ranking rows
+  const float *qbar;          // [B, D] sum of the visual queries (Eq. 1, queries first), or nullptr.  Given: the
+                              // kernel also writes mass_heads (the attention mass per head), see below
+  float *mass_heads;          // [B, H, max_vis] qbar^h . k_j^h for every visual key j (unscaled)
+  int D;
   unsigned int *work;         // [2] next item / blocks that have finished; both zero between launches
   uint32_t *status;
   long long wait_limit;       // clock cycles a wait may take before the block gives up
@@ -84,7 +95,7 @@ struct ScoreArgs {
 
 struct ScoreBook {             // bookkeeping block placed after the tiles in shared memory
   uint64_t full[SC_STAGES], empty[SC_STAGES], q_full, q_empty, acc_full[2], acc_empty[2];
-  uint64_t item_full[SC_ITEM_SLOTS], item_empty[SC_ITEM_SLOTS], mma_done;
+  uint64_t item_full[SC_ITEM_SLOTS], item_empty[SC_ITEM_SLOTS], mma_done, qbar_ready;
   int item_q[SC_ITEM_SLOTS];   // items drawn by the producer, -1 = no more
   alignas(16) float off[256];  // per ranking row of the pair: max + log2(sum), +inf for rows past its end
                                // (with one row tile, off[128..255] carries group 1's partial sums)
@@ -102,10 +113,10 @@ struct RowPair {
 };
 
 // Row pair rp of a sample's ranking rows: rows R0 .. R0 + nrows - 1 (sequence-relative positions).
-__device__ __forceinline__ RowPair score_row_pair(const SampleDesc &d, int rp, int mask_enable) {
+__device__ __forceinline__ RowPair score_row_pair(const SampleDesc &d, int rp, int mask_enable, int pair_rows) {
   RowPair r;
-  r.R0 = d.r0 + rp * 256;
-  r.nrows = min(256, d.nr - rp * 256);
+  r.R0 = d.r0 + rp * pair_rows;
+  r.nrows = min(pair_rows, d.nr - rp * pair_rows);
   r.nrt = (r.nrows + 127) >> 7;
   r.n2 = (r.nrows + 15) & ~15;
   const int p_max = r.R0 + r.nrows - 1;
@@ -126,6 +137,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_items = a.B * a.H;
+  const bool with_mass = a.qbar != nullptr;
+  const int pair_rows = with_mass ? 240 : 256;           // ranking rows per row pair
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -154,6 +167,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       mbar_init(smem_u32(&bk->item_empty[i]), 9);         // the MMA issuer + every epilogue warp
     }
     mbar_init(smem_u32(&bk->mma_done), 1);
+    mbar_init(smem_u32(&bk->qbar_ready), 1);
     bk->abort_flag = 0;
     fence_barrier_init();
   }
@@ -194,9 +208,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         const int b = item / a.H, h = item - b * a.H;
         const SampleDesc d = make_desc(a.pa, b);
         if (!d.valid) continue;
-        const int n_rp = (d.nr + 255) / 256;
+        const int n_rp = (d.nr + pair_rows - 1) / pair_rows;
         for (int rp = 0; rp < n_rp; ++rp, ++qc) {
-          const RowPair T = score_row_pair(d, rp, a.mask_enable);
+          const RowPair T = score_row_pair(d, rp, a.mask_enable, pair_rows);
           if (qc >= 1) mbar_wait(smem_u32(&bk->q_empty), (qc - 1) & 1, wc);
           if (!bk->abort_flag) {
             mbar_expect_tx(smem_u32(&bk->q_full), T.nrt * SC_TILE_BYTES);
@@ -230,7 +244,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      int kc = 0, qc = 0, g = 0, ic = 0;
+      int kc = 0, qc = 0, g = 0, ic = 0, mc = 0;      // mc: items whose summed-query rows were waited for
       bool issued_any = false;
       const uint32_t idesc1 = umma_idesc_bf16(128, 128);
       while (true) {
@@ -243,13 +257,18 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         const int b = item / a.H;
         const SampleDesc d = make_desc(a.pa, b);
         if (!d.valid) continue;
-        const int n_rp = (d.nr + 255) / 256;
+        const int n_rp = (d.nr + pair_rows - 1) / pair_rows;
         for (int rp = 0; rp < n_rp; ++rp, ++qc) {
-          const RowPair T = score_row_pair(d, rp, a.mask_enable);
-          const uint32_t idesc2 = umma_idesc_bf16(128, T.n2);
+          const RowPair T = score_row_pair(d, rp, a.mask_enable, pair_rows);
+          const bool mass_here = with_mass && rp == 0;       // three more columns (16 with padding): the summed query
+          const uint32_t idesc2 = umma_idesc_bf16(128, T.n2 + (mass_here ? 16 : 0));
           mbar_wait(smem_u32(&bk->q_full), qc & 1, wc);
           for (int u = 0; u < T.n_kt + T.n_p2; ++u, ++kc, ++g) {
             const bool pass1 = u < T.n_kt;
+            if (mass_here && u == T.n_kt) {                  // an epilogue warp has written the summed-query rows
+              mbar_wait(smem_u32(&bk->qbar_ready), mc & 1, wc);
+              ++mc;
+            }
             const int s = kc % SC_STAGES, hh = g & 1;
             if (g >= 2) mbar_wait(smem_u32(&bk->acc_empty[hh]), ((g >> 1) - 1) & 1, wc);
             mbar_wait(smem_u32(&bk->full[s]), (kc / SC_STAGES) & 1, wc);
@@ -275,6 +294,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
               issued_any = true;
             }
           }
+          if (mass_here && T.n_p2 == 0) {                    // (no visual key tile: keep the barrier's phases in step)
+            mbar_wait(smem_u32(&bk->qbar_ready), mc & 1, wc);
+            ++mc;
+          }
           if (!bk->abort_flag) tc_commit(smem_u32(&bk->q_empty));
         }
       }
@@ -296,7 +319,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     const uint32_t tlane0 = tmem_base + ((uint32_t)(quarter * 32) << 16);
     float *soft = bk->soft[group];
     float *pm = bk->soft[1], *pl = bk->off + 128;  // group 1's (max, sum) when both groups share one row tile
-    int g = 0, ic = 0;
+    int g = 0, ic = 0, qc = 0;
     while (true) {
       const int slot = ic % SC_ITEM_SLOTS;
       const bool got = mbar_wait_drain(smem_u32(&bk->item_full[slot]), (ic / SC_ITEM_SLOTS) & 1, TC_WAIT_LIMIT);
@@ -308,7 +331,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       const int b = item / a.H, h = item - b * a.H;
       const SampleDesc d = make_desc(a.pa, b);
       if (!d.valid) continue;
-      const int n_rp = (d.nr + 255) / 256;
+      const int n_rp = (d.nr + pair_rows - 1) / pair_rows;
       float *part = a.partial + ((size_t)b * a.H + h) * a.max_vis;
       const float *mlog = a.mask_log + (size_t)b * a.mask_b_stride + (size_t)h * a.mask_h_stride;
       const int v_end = d.v0 + d.nv;
@@ -316,12 +339,48 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         // visual keys beyond the tiles the first row pair visits in pass 2 (possible only when
         // ranking rows lie before the end of the image span) start from zero; the epilogue-wide
         // barrier that ends every pass 1 orders these stores before any later add
-        const RowPair T0 = score_row_pair(d, 0, a.mask_enable);
+        const RowPair T0 = score_row_pair(d, 0, a.mask_enable, pair_rows);
         const int first = T0.n_p2 > 0 ? max((T0.t_hi + 1) * 128 - d.v0, 0) : 0;
         for (int j = first + et; j < d.nv; j += SC_EPI_THREADS) part[j] = 0.f;
       }
-      for (int rp = 0; rp < n_rp; ++rp) {
-        const RowPair T = score_row_pair(d, rp, a.mask_enable);
+      for (int rp = 0; rp < n_rp; ++rp, ++qc) {
+        const RowPair T = score_row_pair(d, rp, a.mask_enable, pair_rows);
+        if (with_mass && rp == 0 && warp == 2) {
+          // The summed query of this head as rows n2 .. n2 + 2 of the pair's query tile: 3 rows x 16 chunks
+          // of 16 bytes at their swizzled places (row r of a 64-column half is 128 bytes at
+          // r * 128, chunk c at c ^ (r & 7)), once the tiled copy of the queries has landed.
+          mbar_wait(smem_u32(&bk->q_full), qc & 1, wc);
+          const int c16 = lane & 15;
+          const float *src = a.qbar + (size_t)b * a.D + h * 128 + c16 * 8;
+          uint32_t w[3][4];                                 // the value as three bf16 pieces: 24 bits of mantissa, all of fp32's
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float x[2] = {__ldcg(src + 2 * e), __ldcg(src + 2 * e + 1)}, piece[3][2];
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+              float rest = x[t];
+#pragma unroll
+              for (int k = 0; k < 3; ++k) {
+                piece[k][t] = __bfloat162float(__float2bfloat16_rn(rest));
+                rest -= piece[k][t];
+              }
+            }
+#pragma unroll
+            for (int k = 0; k < 3; ++k) w[k][e] = pack2_rn(piece[k][0], piece[k][1]);
+          }
+          // lanes 0-15 write the first piece's row and the third's, lanes 16-31 the second's
+#pragma unroll
+          for (int k = 0; k < 3; ++k) {
+            if ((k == 1) == (lane >= 16)) {
+              const int row = T.n2 + k;
+              uint8_t *dst = base_ptr + (c16 >> 3) * SC_Q_HALF_BYTES + row * 128 + (((c16 & 7) ^ (row & 7)) << 4);
+              *reinterpret_cast<uint4 *>(dst) = make_uint4(w[k][0], w[k][1], w[k][2], w[k][3]);
+            }
+          }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bk->qbar_ready));
+        }
         // ---------------- pass 1: thread = ranking row.  Two row tiles: group g owns tile g of every key
         // tile; one row tile: the groups take alternate key tiles
         const bool two = T.nrt == 2;
@@ -497,6 +556,15 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
               // the first row pair initialises the slots it covers; later row pairs add
               if (rp == 0) part[j - d.v0] = sum;
               else part[j - d.v0] += sum;
+            }
+            if (with_mass && rp == 0) {
+              // columns n2 .. n2 + 2: the three pieces of the summed query against this key
+              uint32_t r[16];
+              tmem_ld16(tlane + T.n2, r);
+              tmem_wait_ld();
+              if (key_ok)
+                a.mass_heads[((size_t)b * a.H + h) * a.max_vis + (j - d.v0)] =
+                    (__uint_as_float(r[0]) + __uint_as_float(r[1])) + __uint_as_float(r[2]);
             }
           }
           tc_fence_before();
