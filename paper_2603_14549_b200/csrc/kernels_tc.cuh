@@ -636,7 +636,7 @@ head_sum_kernel(const SampleDesc *__restrict__ desc, int H, int max_vis,
 //                   The gather path moves at most ~23 bytes per clock and SM (the load/store unit's
 //                   requests in flight; a gather copy of four rows per instruction through the
 //                   tensor-map unit managed a third of that), the tiled path twice as much, so the host
-//                   gathers only when the kept rows are a large share of the span.
+//                   gathers only when the kept rows are a large share of the span (two fifths or more).
 // While the first
 // accumulator is being built the epilogue warps also read every row tile from shared memory and
 // add up the squares (the row norms of Sec. 4.2's cosine similarity).
