@@ -225,11 +225,15 @@ asap_status asap_compact_kv(asap_ctx *ctx, const int32_t *src_row, const int32_t
                             const void *const *src, void *const *dst, void *stream);
 
 /* Reads the device status word (one 4-byte copy after synchronising `stream`).  ASAP_OK, or
- * ASAP_ERR_DEVICE with the reason in asap_last_error; the word is cleared. */
+ * ASAP_ERR_DEVICE with the reason in asap_last_error; the word is cleared.  After a time-out bit
+ * (a bounded wait ran out in a tensor-core kernel) every result enqueued on the context since
+ * the bit was set is invalid, and the call also puts the kernels' hand-shake counters back to
+ * zero; the context is ready for normal work when it returns. */
 asap_status asap_check(asap_ctx *ctx, void *stream);
 
 /* Text of the last error recorded on this context (empty string if none).  Valid until the
- * next call on the context.  asap_last_error(NULL) describes a failed asap_init. */
+ * next call on the context.  asap_last_error(NULL) describes a failed asap_init or
+ * asap_select_static; that text lives in one buffer shared by all threads of the process. */
 const char *asap_last_error(const asap_ctx *ctx);
 
 /* Step 3 once more, for callers that cannot allocate device memory.  (The paper has no
@@ -256,7 +260,13 @@ const char *asap_last_error(const asap_ctx *ctx);
  * memory limit; make that first call outside any stream capture.  All calls on a device share
  * the one array, which keeps what the previous call left: the call clears the status word
  * itself and overwrites the rest, but two calls that overlap on the GPU (different streams,
- * different threads) race on it.  Errors are reported through asap_last_error(NULL). */
+ * different threads) race on it.  Errors are reported through asap_last_error(NULL), one text
+ * buffer for the whole process: read it from the thread that made the failing call, before another
+ * thread calls asap_init or this function.  With device_status == NULL a sequence that fails the
+ * device-side validation is still skipped (its outputs are all -1) but nothing the caller can
+ * read records that: pass a status word if the per-sequence arrays are not trusted.  The first
+ * call on a device also pays for what any first CUDA call pays (context creation, loading of the
+ * library's device code), which the driver does with allocations of its own. */
 asap_status asap_select_static(const asap_inputs *in, const asap_params *p, const float *rank_score,
                                int32_t *keep_idx, int32_t *drop_idx, uint32_t *device_status,
                                void *stream);

@@ -11,7 +11,9 @@ widened exactly to float64 before any arithmetic.
 Parity status of each function (what pins it, see tests/test_oracle_pins.py):
   attention_mass        pinned  (closed form via the summed query; hand-worked fixture)
   attention_mass_heads  pinned  (its head mean is attention_mass; one head = attention_mass; the
-                                 per-head step with identical heads equals the default step)
+                                 per-head step with identical heads equals the default step; a hand-worked
+                                 two-head case fixes the per-head masses and the Eq. 5 weight of the
+                                 per-head step -- the head mean of the per-head saliences)
   salience / mask_log   pinned  (hand-worked fixture; extremes; affine invariance)
   mask_matrix           pinned  (hand-enumerated 5x5 fixture; causal limit)
   attention_probs /

@@ -46,8 +46,12 @@ def test_static_select_matches_select_on_two_calls_in_a_row():
             keep = torch.full((B, k), -7, dtype=torch.int32, device=DEV)
             drop = torch.full((B, mv - k), -7, dtype=torch.int32, device=DEV)
             status = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info(0)[0]
             A.asap_select_static(inp, p, scores, keep, drop, status)
             torch.cuda.synchronize()
+            if call > 0:       # (the first call on a device may load the library's device code)
+                assert torch.cuda.mem_get_info(0)[0] == free_before, "the call changed the device's free memory"
             A.asap_check(ctx)
             assert int(status.item()) == 0
             assert torch.equal(keep, want.keep_idx), f"call {call}: keep_idx differs"      # indices: bit-exact
