@@ -46,6 +46,8 @@ struct asap_ctx {
                *cnt_tiles = nullptr, *cnt_work = nullptr;
   float *mass_partial = nullptr;    // [B, H, max_vis] per-head attention masses written by the score kernel
   long long fuse_mass_min_tokens = 50000;   // B * max_vis from which the attention mass rides in the score kernel
+  long long sim_pair_min_blocks = 0;        // blocks from which the similarity takes two row tiles per block (0: the SM count)
+  int sim_pair_stages = 0;                  // stages of that form (0: what fits 192 KB)
   float *sim_part = nullptr;        // partial dot products / squared norms of a sliced similarity GEMM
   size_t sim_part_bytes = 0, cap_tiles = 0;
   int32_t *role = nullptr, *seg = nullptr, *members = nullptr;
@@ -349,6 +351,42 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     // 0.56 ms against 0.92 ms).
     const bool gather_rows = splits == 1 && (long long)k * 5 >= 2LL * in->max_vis &&
                              (long long)max_mt * B > ctx->num_sms;
+    // Every visual row, two row tiles per block, the kept slots dealt in groups of at most 256 to the
+    // blocks of a pair, one pass each: fewer bytes out of L2 per product, which is what bounds the
+    // similarity of a large batch.  Taken when that grid fills the machine.
+    {
+      const int pairs = (in->max_vis + 255) / 256;
+      const int pg = (k + 255) / 256;
+      const int ptile = (((k + pg - 1) / pg) + 15) & ~15;
+      const long long min_blocks = ctx->sim_pair_min_blocks > 0 ? ctx->sim_pair_min_blocks : ctx->num_sms;
+      const int pstage = 2 * SIM_A_BYTES + ptile * 128;
+      int pstages = ctx->sim_pair_stages > 0 ? ctx->sim_pair_stages : (192 * 1024) / pstage;
+      if (pstages > SIM_MAX_STAGES) pstages = SIM_MAX_STAGES;
+      const size_t psmem = (size_t)pstages * pstage + SIM_BOOK_BYTES + 1024;
+      if (!gather_rows && splits == 1 && D % 64 == 0 && (long long)pairs * B * pg >= min_blocks &&
+          (size_t)B * pairs <= ctx->cap_tiles && pstages >= 2 && psmem <= 227 * 1024 &&
+          (size_t)B * pairs * (size_t)(pg * 512 + 256) * sizeof(float) <= ctx->sim_part_bytes &&
+          (size_t)(SIMP_THREADS / 32 + 1) * k * sizeof(int) <= (size_t)pstages * pstage) {
+        uint32_t pcols = 32;
+        while ((int)pcols < 2 * ptile) pcols <<= 1;
+        CUtensorMap map_h, map_kept;
+        if (!make_map(ctx, &map_h, in->hidden, (uint64_t)in->total_tokens, (uint64_t)D, 128) ||
+            !make_map(ctx, &map_kept, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, (uint32_t)ptile))
+          return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for hidden / kept rows");
+        SimArgs sa;
+        sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = ptile;
+        sa.n_nt = 1; sa.stages = pstages; sa.splits = 1; sa.max_mt = pairs; sa.tmem_cols = pcols;
+        sa.wide = 1; sa.groups = pg; sa.threshold = p->sim_threshold;
+        sa.drop_idx = nullptr; sa.role = ctx->role;
+        sa.hidden = static_cast<const __nv_bfloat16 *>(in->hidden); sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
+        sa.best_sim = out->best_sim; sa.seg = ctx->seg; sa.members = ctx->members; sa.counters = ctx->cnt_sim;
+        sa.tile_counters = ctx->cnt_tiles; sa.part = ctx->sim_part; sa.ss_part = nullptr; sa.smat = nullptr;
+        sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
+        mark(ctx, "sim", st);
+        launch_pdl(sim_pair_kernel, dim3(pairs * pg, B), dim3(SIMP_THREADS), psmem, st, map_h, map_kept, sa);
+        return after_launch(ctx, "sim");
+      }
+    }
     if (gather_rows) max_mt = (in->max_vis - k + 127) / 128;
     bool wide = n_nt >= 2 && n_nt * n_tile <= 512 && 3 * (SIM_A_BYTES + n_nt * n_tile * 128) <= 192 * 1024;
     // More slots than that, and enough row tiles that the hidden dimension is not sliced: the slot tiles are
@@ -591,6 +629,8 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   ctx->score_partial = reinterpret_cast<float *>(ctx->arena + o_spart);
   ctx->mass_partial = reinterpret_cast<float *>(ctx->arena + o_mpart);
   if (const char *env = getenv("ASAP_FUSE_MASS_MIN_TOKENS")) ctx->fuse_mass_min_tokens = atoll(env);
+  if (const char *env = getenv("ASAP_SIM_PAIR_MIN_BLOCKS")) ctx->sim_pair_min_blocks = atoll(env);
+  if (const char *env = getenv("ASAP_SIM_PAIR_STAGES")) ctx->sim_pair_stages = atoi(env);
   ctx->inv_norm = reinterpret_cast<float *>(ctx->arena + o_inv);
   ctx->kept_inv = reinterpret_cast<float *>(ctx->arena + o_kinv);
   ctx->counters_off = o_cnt; ctx->counters_bytes = (Bc * col_blocks + 3 * Bc + 2) * sizeof(unsigned int);
@@ -614,6 +654,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   if (e == cudaSuccess) e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(sim_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM_BYTES);

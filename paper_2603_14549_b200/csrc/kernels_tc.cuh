@@ -1130,4 +1130,257 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
             bk->scan);
 }
 
+// =======================================================================================
+// sim_pair_kernel
+//
+// The all-rows form of sim_kernel for batches large enough to fill the machine without slicing the
+// hidden dimension.  There the similarity kernel is bound by the bytes the SMs pull out of L2 (at
+// about 11 TB/s over all SMs), not by the tensor pipe: a block of sim_kernel streams 128 rows and
+// n_tile kept rows per 64 columns, (128 + n_tile) * 128 bytes for 128 * n_tile * 64 products.  This
+// kernel multiplies TWO row tiles against each stage's kept rows -- (256 + n_tile) * 128 bytes for
+// twice the products, 30 % fewer bytes per product at n_tile = 192 -- and makes a single pass over
+// the hidden dimension: the kept slots are dealt in groups of n_tile <= 256 to `groups` blocks per
+// pair of row tiles (blockIdx.x = pair * groups + group).  The blocks of a pair are neighbours in
+// launch order and stream the same rows at the same pace, so the rows come from memory once and
+// from L2 for the other groups.  Accumulators: row tile t at tensor-memory column t * n_tile.
+// Every block adds up its rows' squares from shared memory only if it is group 0, and publishes
+// its rows' best (value, slot); the block that finishes a pair last takes the maximum over the
+// groups (lowest slot among equals), looks up which rows were dropped and writes their assignment.
+// The block that finishes a sample's last pair groups the dropped tokens by destination.
+// =======================================================================================
+constexpr int SIMP_THREADS = 320;                // copy warp, MMA warp, two groups of four epilogue warps
+
+struct SimPairBook {
+  uint64_t full[SIM_MAX_STAGES], empty[SIM_MAX_STAGES], acc_full, mma_done;
+  uint32_t tmem_base;
+  int abort_flag;
+  int is_last;
+  int scan[33];
+};
+
+static_assert(sizeof(SimPairBook) <= SIM_BOOK_BYTES, "pair kernel bookkeeping exceeds its shared-memory slot");
+
+__global__ void __launch_bounds__(SIMP_THREADS, 1)
+sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_kept,
+                SimArgs a) {
+  pdl_enter();
+  extern __shared__ uint8_t smem_raw[];
+  const int pr = blockIdx.x / a.groups, b = blockIdx.y;
+  const int gz = blockIdx.x - pr * a.groups;             // group of kept slots
+  const SampleDesc d = a.desc[b];
+  if (!d.valid) return;
+  const int nd = d.nv - a.keep_k;
+  const int n_rows = d.nv;
+  if (pr * 256 >= n_rows) return;
+  if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SIM_TIMEOUT) return;
+  const bool two = pr * 256 + 128 < n_rows;              // the pair's second row tile holds visual rows
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  // a stage: [ row tile 0 | row tile 1 | kept rows ] of one 64-column block
+  const int b_bytes = a.n_tile * 128;
+  const int stage_bytes = 2 * SIM_A_BYTES + b_bytes;
+  SimPairBook *bk = reinterpret_cast<SimPairBook *>(base_ptr + (size_t)a.stages * stage_bytes);
+
+  // the epilogue warps of group 0 read their row tile from the stages (for the row norms)
+  const int n_readers = gz == 0 ? (two ? 8 : 4) : 0;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < a.stages; ++s) {
+      mbar_init(smem_u32(&bk->full[s]), 1);
+      mbar_init(smem_u32(&bk->empty[s]), 1 + n_readers);   // the MMAs that read the stage + the warps that do
+    }
+    mbar_init(smem_u32(&bk->acc_full), 1);
+    mbar_init(smem_u32(&bk->mma_done), 1);
+    bk->abort_flag = 0;
+    bk->is_last = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bk->tmem_base), a.tmem_cols);
+    tmem_relinquish();
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bk->tmem_base;
+  WaitCtx wc{&bk->abort_flag, a.status, STATUS_SIM_TIMEOUT, a.wait_limit};
+  const int n_kb = a.D / 64;
+  // the groups of a pair walk the 64-column blocks from the same starting point (they share the rows
+  // through L2); different pairs start elsewhere and spread over the memory channels
+  const int rot = (pr * 5 + b * 3) % n_kb;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tmap_h);
+      tma_prefetch_desc(&tmap_kept);
+      const int row_a = d.row0 + d.v0 + pr * 256;
+      const int row_b = b * a.keep_k + gz * a.n_tile;
+      const int tx_bytes = two ? stage_bytes : stage_bytes - SIM_A_BYTES;
+      int issued = 0;
+      for (int it = 0; it < n_kb; ++it) {
+        const int s = it % a.stages, kb = (it + rot) % n_kb;
+        const uint32_t full = smem_u32(&bk->full[s]);
+        if (it >= a.stages) mbar_wait(smem_u32(&bk->empty[s]), ((it / a.stages) - 1) & 1, wc);
+        if (bk->abort_flag) break;
+        const uint32_t dst = base + s * stage_bytes;
+        mbar_expect_tx(full, tx_bytes);
+        tma_load_2d(dst, &tmap_h, full, kb * 64, row_a);
+        if (two) tma_load_2d(dst + SIM_A_BYTES, &tmap_h, full, kb * 64, row_a + 128);
+        tma_load_2d(dst + 2 * SIM_A_BYTES, &tmap_kept, full, kb * 64, row_b);
+        issued = it + 1;
+      }
+      // drain: the last fill of every stage must have landed before the block leaves
+      for (int s = 0; s < a.stages; ++s) {
+        if (issued > s) {
+          const int last = ((issued - 1 - s) / a.stages) * a.stages + s;
+          mbar_wait_drain(smem_u32(&bk->full[s]), (last / a.stages) & 1, TC_WAIT_LIMIT);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(128, a.n_tile);
+      const int n_t = two ? 2 : 1;
+      for (int it = 0; it < n_kb; ++it) {
+        const int s = it % a.stages;
+        mbar_wait(smem_u32(&bk->full[s]), (it / a.stages) & 1, wc);
+        tc_fence_after();
+        if (!bk->abort_flag) {
+          const uint32_t sa = base + s * stage_bytes, sb = sa + 2 * SIM_A_BYTES;
+          for (int t = 0; t < n_t; ++t)
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              tc_mma_bf16(tmem_base + t * a.n_tile, umma_desc_sw128(sa + t * SIM_A_BYTES + kk * 32),
+                          umma_desc_sw128(sb + kk * 32), idesc, (it > 0 || kk > 0) ? 1u : 0u);
+          tc_commit(smem_u32(&bk->empty[s]));
+        }
+      }
+      if (!bk->abort_flag) tc_commit(smem_u32(&bk->acc_full));
+      // every MMA this thread issued has completed before tensor memory is given back
+      tc_commit(smem_u32(&bk->mma_done));
+      mbar_wait_drain(smem_u32(&bk->mma_done), 0, TC_WAIT_LIMIT);
+    }
+  } else {
+    const int grp = (warp - 2) >> 2;                     // row tile of the pair
+    const int quarter = warp & 3;                        // the tensor-memory lanes a warp may read
+    const int lrow = quarter * 32 + lane;
+    const int prow = grp * 128 + lrow;                   // row inside the pair
+    const int v = pr * 256 + prow;                       // visual token
+    const bool active = grp == 0 || two;
+    const float *kinv = a.kept_inv + (size_t)b * a.keep_k;
+    // ---- squared norm of this thread's row (group 0 only; the other groups just free the stages)
+    float ssq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    const bool norms = gz == 0 && active;
+    for (int it = 0; it < (norms ? n_kb : 0); ++it) {
+      const int s = it % a.stages;
+      mbar_wait(smem_u32(&bk->full[s]), (it / a.stages) & 1, wc);
+      if (!bk->abort_flag) {
+        const uint4 *row = reinterpret_cast<const uint4 *>(base_ptr + (size_t)s * stage_bytes +
+                                                           grp * SIM_A_BYTES + lrow * 128);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint4 x = row[c ^ (lrow & 7)];
+          float f[8];
+          unpack8(x, f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) ssq[c] = fmaf(f[e], f[e], ssq[c]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bk->empty[s]));
+    }
+    float ss = ((ssq[0] + ssq[1]) + (ssq[2] + ssq[3])) + ((ssq[4] + ssq[5]) + (ssq[6] + ssq[7]));
+
+    float best = -INFINITY;
+    int best_slot = 0;
+    mbar_wait(smem_u32(&bk->acc_full), 0, wc);
+    tc_fence_after();
+    const int slot0 = gz * a.n_tile;
+    const int ncol = max(0, min(a.n_tile, a.keep_k - slot0));
+    if (active && !bk->abort_flag) {
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + grp * a.n_tile;
+#pragma unroll 1
+      for (int c = 0; c < ncol; c += 16) {
+        uint32_t r[16];
+        tmem_ld16(taddr + c, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const int slot = slot0 + c + e;
+          if (c + e < ncol) {
+            const float val = __uint_as_float(r[e]) * __ldg(kinv + slot);
+            if (val > best) { best = val; best_slot = slot; }
+          }
+        }
+      }
+    }
+    tc_fence_before();
+    bool finalize = true;
+    if (a.groups > 1) {
+      // per pair: [group][best of 256 rows | slot of 256 rows], then the 256 squared norms
+      float *pp = a.part + ((size_t)b * a.max_mt + pr) * (size_t)(a.groups * 512 + 256);
+      pp[gz * 512 + prow] = best;
+      reinterpret_cast<int *>(pp)[gz * 512 + 256 + prow] = best_slot;
+      if (gz == 0) pp[a.groups * 512 + prow] = ss;
+      __threadfence();
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (warp == 2 && lane == 0) {
+        unsigned int *cnt = a.tile_counters + (size_t)b * a.max_mt + pr;
+        const unsigned int old = atomicAdd(cnt, 1u);
+        bk->is_last = (old == (unsigned int)(a.groups - 1));
+        if (bk->is_last) *cnt = 0u;
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      finalize = bk->is_last != 0;
+      if (finalize) {
+        __threadfence();
+        best = -INFINITY;
+        best_slot = 0;
+        for (int g2 = 0; g2 < a.groups; ++g2) {           // ascending slots: the first maximum stays
+          const float val = __ldcg(pp + g2 * 512 + prow);
+          const int slot = __ldcg(reinterpret_cast<const int *>(pp) + g2 * 512 + 256 + prow);
+          if (val > best) { best = val; best_slot = slot; }
+        }
+        ss = __ldcg(pp + a.groups * 512 + prow);
+      }
+    }
+    int dp = -1;
+    if (finalize && v < n_rows) {
+      const int role = a.role[(size_t)b * a.max_vis + v];
+      dp = role < 0 ? -role - 1 : -1;
+    }
+    if (dp >= 0 && dp < nd && !bk->abort_flag) {
+      const bool zero_row = !(ss >= 1e-24f);             // ||h|| < 1e-12: similarity 0 to every slot
+      const float sim = zero_row ? 0.f : best * rsqrtf(ss);
+      const int slot = zero_row ? 0 : best_slot;
+      const size_t o = (size_t)b * (a.max_vis - a.keep_k) + dp;
+      a.assign[o] = (sim > a.threshold) ? slot : -1;
+      if (a.best_sim) a.best_sim[o] = sim;
+    }
+    if (warp == 2 && lane == 0) bk->is_last = finalize ? 1 : 0;
+    __threadfence();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, a.tmem_cols);
+  }
+  if (!bk->is_last) return;                              // a group that did not finalize its pair
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned int n_pr = (unsigned int)((n_rows + 255) / 256);
+    const unsigned int old = atomicAdd(a.counters + b, 1u);
+    bk->is_last = (old == n_pr - 1u);
+    if (bk->is_last) a.counters[b] = 0u;
+  }
+  __syncthreads();
+  if (!bk->is_last) return;
+  __threadfence();
+  csr_block(d, b, a.max_vis, a.keep_k, a.assign, a.seg, a.members, reinterpret_cast<int *>(base_ptr),
+            bk->scan);
+}
+
 }  // namespace asap
