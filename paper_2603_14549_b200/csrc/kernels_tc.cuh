@@ -1134,12 +1134,16 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
 // sim_pair_kernel
 //
 // The all-rows form of sim_kernel for batches large enough to fill the machine without slicing the
-// hidden dimension.  There the similarity kernel is bound by the bytes the SMs pull out of L2 (at
-// about 11 TB/s over all SMs), not by the tensor pipe: a block of sim_kernel streams 128 rows and
+// hidden dimension.  There the similarity kernel is bound by the bytes an SM can take in, not by the
+// tensor pipe: measured, the tiled copies of a block deliver about 34 bytes per clock whatever the
+// stage size or count (9.6 TB/s over 148 SMs), and a block of sim_kernel streams 128 rows and
 // n_tile kept rows per 64 columns, (128 + n_tile) * 128 bytes for 128 * n_tile * 64 products.  This
 // kernel multiplies TWO row tiles against each stage's kept rows -- (256 + n_tile) * 128 bytes for
-// twice the products, 30 % fewer bytes per product at n_tile = 192 -- and makes a single pass over
-// the hidden dimension: the kept slots are dealt in groups of n_tile <= 256 to `groups` blocks per
+// twice the products, 30 % fewer bytes per product at n_tile = 192; tensor memory (512 columns =
+// 2 tiles x n_tile <= 256) allows no larger block.  (MMAs spanning a pair of CTAs, each CTA loading half
+// of the kept rows, were built and measured: the half an SM reads from its partner's shared memory
+// arrives through the same 34 bytes per clock, once per row tile, and the kernel ran 30 % slower.)
+// It makes a single pass over the hidden dimension: the kept slots are dealt in groups of n_tile <= 256 to `groups` blocks per
 // pair of row tiles (blockIdx.x = pair * groups + group).  The blocks of a pair are neighbours in
 // launch order and stream the same rows at the same pace, so the rows come from memory once and
 // from L2 for the other groups.  Accumulators: row tile t at tensor-memory column t * n_tile.
