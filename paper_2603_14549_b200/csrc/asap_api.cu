@@ -51,6 +51,7 @@ struct asap_ctx {
   float *sim_part = nullptr;        // partial dot products / squared norms of a sliced similarity GEMM
   size_t sim_part_bytes = 0, cap_tiles = 0;
   int32_t *role = nullptr, *seg = nullptr, *members = nullptr;
+  int2 *member_meta = nullptr;              // (visual index, merge weight) beside every entry of `members`
   __nv_bfloat16 *kept_rows = nullptr;
   uint32_t *status = nullptr;
   EncodeTiledFn encode = nullptr;
@@ -307,7 +308,9 @@ asap_status launch_select(asap_ctx *ctx, const asap_inputs *in, const asap_param
 }
 
 // Step 4a: kept rows gathered, cosine similarity and assignment, CSR of the assignment.
-asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
+// `salience`: the merge weights if they are complete when this is enqueued (the grouping then copies each
+// member's weight beside its index for the merge kernel), else nullptr.
+asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const float *salience,
                                const int32_t *keep_idx, const int32_t *drop_idx, const asap_outputs *out,
                                cudaStream_t st) {
   const int B = in->B, D = in->D, k = p->keep_k;
@@ -383,6 +386,7 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
         sa.hidden = static_cast<const __nv_bfloat16 *>(in->hidden); sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
         sa.best_sim = out->best_sim; sa.seg = ctx->seg; sa.members = ctx->members; sa.counters = ctx->cnt_sim;
         sa.tile_counters = ctx->cnt_tiles; sa.part = ctx->sim_part; sa.ss_part = nullptr; sa.smat = nullptr;
+        sa.drop_all = drop_idx; sa.salience = salience; sa.member_meta = salience ? ctx->member_meta : nullptr;
         sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
         mark(ctx, "sim", st);
         launch_pdl(sim_pair_kernel, dim3(pairs * pg, B), dim3(SIMP_THREADS), psmem, st, map_h, map_kept, sa);
@@ -438,6 +442,7 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     sa.tile_counters = ctx->cnt_tiles; sa.part = ctx->sim_part;
     sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
     sa.smat = nullptr;
+    sa.drop_all = drop_idx; sa.salience = salience; sa.member_meta = salience ? ctx->member_meta : nullptr;
     sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
     mark(ctx, "sim", st);
     if (gather_rows)
@@ -452,14 +457,15 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
 // Steps 4b-5: weighted merge and compaction (the first consumer of the salience).
 asap_status launch_merge_back(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                               const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
-                              const asap_outputs *out, cudaStream_t st) {
+                              const asap_outputs *out, cudaStream_t st, bool grouped_with_weights = false) {
   const int B = in->B, D = in->D, k = p->keep_k;
   const bool do_merge = merging(in, p);
   MergeArgs ma;
   ma.hidden = static_cast<const __nv_bfloat16 *>(in->hidden); ma.pos_ids = in->pos_ids; ma.desc = ctx->desc;
   ma.D = D; ma.max_vis = in->max_vis; ma.keep_k = k; ma.merge_enable = do_merge ? 1 : 0; ma.eps = p->eps;
   ma.salience = salience; ma.keep_idx = keep_idx; ma.drop_idx = drop_idx; ma.seg = ctx->seg;
-  ma.members = ctx->members; ma.out_hidden = static_cast<__nv_bfloat16 *>(out->out_hidden);
+  ma.members = ctx->members; ma.member_meta = (do_merge && grouped_with_weights) ? ctx->member_meta : nullptr;
+  ma.out_hidden = static_cast<__nv_bfloat16 *>(out->out_hidden);
   ma.out_pos = out->out_pos; ma.src_row = out->src_row;
   const int copy_rows = in->max_seq - in->min_vis;   // prefix + suffix rows of the longest sequence, at most
   const dim3 grid(k + (copy_rows + MERGE_COPY_ROWS - 1) / MERGE_COPY_ROWS, B);
@@ -477,8 +483,8 @@ asap_status launch_merge_back(asap_ctx *ctx, const asap_inputs *in, const asap_p
 asap_status launch_merge(asap_ctx *ctx, const asap_inputs *in, const asap_params *p,
                          const float *salience, const int32_t *keep_idx, const int32_t *drop_idx,
                          const asap_outputs *out, cudaStream_t st) {
-  ASAP_TRY(launch_merge_front(ctx, in, p, keep_idx, drop_idx, out, st));
-  return launch_merge_back(ctx, in, p, salience, keep_idx, drop_idx, out, st);
+  ASAP_TRY(launch_merge_front(ctx, in, p, salience, keep_idx, drop_idx, out, st));
+  return launch_merge_back(ctx, in, p, salience, keep_idx, drop_idx, out, st, true);
 }
 
 // Sec. 4.2 inside the kept set: kept rows gathered, their keep_k x keep_k cosine matrix, routing.
@@ -533,7 +539,8 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   sa.drop_idx = nullptr; sa.role = nullptr; sa.hidden = nullptr; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
   sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr; sa.tile_counters = ctx->cnt_tiles;
   sa.part = ctx->sim_part; sa.ss_part = ctx->sim_part + (size_t)B * max_mt * splits * (size_t)k * 128;
-  sa.smat = smat; sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
+  sa.smat = smat; sa.drop_all = nullptr; sa.salience = nullptr; sa.member_meta = nullptr;
+  sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
   mark(ctx, "sim_kept", st);
   launch_pdl(sim_kernel<false>, dim3(max_mt, B, splits), dim3(SIM_THREADS_TILED), smem, st, map_a, map_b, sa);
   ASAP_TRY(after_launch(ctx, "sim_kept"));
@@ -614,6 +621,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   const size_t o_role = carve(T * sizeof(int32_t));
   const size_t o_seg = carve((max_keep_rows + Bc) * sizeof(int32_t));
   const size_t o_mem = carve(T * sizeof(int32_t));
+  const size_t o_meta = carve(T * sizeof(int2));
   const size_t o_kept = carve(max_keep_rows * Dc * sizeof(__nv_bfloat16));
   ctx->cap_tiles = T / 128 + Bc;                       // row tiles of 128 visual rows in any batch that fits
   ctx->sim_part_bytes = (size_t)32 << 20;
@@ -645,6 +653,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   ctx->role = reinterpret_cast<int32_t *>(ctx->arena + o_role);
   ctx->seg = reinterpret_cast<int32_t *>(ctx->arena + o_seg);
   ctx->members = reinterpret_cast<int32_t *>(ctx->arena + o_mem);
+  ctx->member_meta = reinterpret_cast<int2 *>(ctx->arena + o_meta);
   ctx->kept_rows = reinterpret_cast<__nv_bfloat16 *>(ctx->arena + o_kept);
   ctx->cnt_tiles = reinterpret_cast<unsigned int *>(ctx->arena + o_tiles);
   ctx->sim_part = reinterpret_cast<float *>(ctx->arena + o_simpart);
@@ -835,7 +844,7 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
   if (main_status == ASAP_OK && cudaStreamWaitEvent(st, ctx->ev_desc, 0) != cudaSuccess)
     main_status = fail(ctx, ASAP_ERR_CUDA, "wait for the descriptors");
   if (main_status == ASAP_OK) main_status = launch_select(ctx, in, p, out->rank_score, out, true, true, st);
-  if (main_status == ASAP_OK) main_status = launch_merge_front(ctx, in, p, out->keep_idx, out->drop_idx, out, st);
+  if (main_status == ASAP_OK) main_status = launch_merge_front(ctx, in, p, nullptr, out->keep_idx, out->drop_idx, out, st);
   // the side stream always rejoins, also after an error, so that `stream` stays ordered behind it
   e = cudaStreamWaitEvent(st, ctx->ev_join, 0);
   if (e != cudaSuccess) return fail(ctx, ASAP_ERR_CUDA, "join with the side stream: %s", cudaGetErrorString(e));

@@ -748,11 +748,17 @@ kept_gather_kernel(const __nv_bfloat16 *__restrict__ hidden, const SampleDesc *_
 // into its own histogram, and after a scan over (slot, warp) writes its chunk's positions behind
 // those of the warps before it.  s_cnt needs (W + 1) * keep_k ints, s_scan 33 ints.
 // seg [B, keep_k+1], members [B, max_vis-keep_k] (dropped POSITIONS, ascending inside a slot).
+// With drop_idx, salience and member_meta given, member_meta [B, max_vis-keep_k] receives, beside every
+// entry of `members`, the member's visual index and its merge weight (the salience, as bits): the
+// merge kernel then reaches a member's row in two dependent loads instead of four.
 // =======================================================================================
 __device__ __forceinline__ void csr_block(const SampleDesc &d, int b, int max_vis, int keep_k,
                                           const int32_t *__restrict__ assign,
                                           int32_t *__restrict__ seg, int32_t *__restrict__ members,
-                                          int *s_cnt, int *s_scan) {
+                                          int *s_cnt, int *s_scan,
+                                          const int32_t *__restrict__ drop_idx = nullptr,
+                                          const float *__restrict__ salience = nullptr,
+                                          int2 *__restrict__ member_meta = nullptr) {
   int32_t *seg_b = seg + (size_t)b * (keep_k + 1);
   const int nd_max = max_vis - keep_k, nd = d.nv - keep_k;
   const int32_t *as_b = assign + (size_t)b * nd_max;
@@ -796,10 +802,16 @@ __device__ __forceinline__ void csr_block(const SampleDesc &d, int b, int max_vi
   if (threadIdx.x == 0) seg_b[keep_k] = total;
   __syncthreads();
   // stable fill: every warp walks its chunk 32 positions at a time in ascending order
+  const bool meta = drop_idx && salience && member_meta;
   for (int base = p_lo; base < p_hi; base += 32) {
     const int p = base + lane;
     int a = (p < p_hi) ? __ldcg(as_b + p) : -1;
     if (a >= keep_k) a = -1;
+    int2 mm = make_int2(0, 0);
+    if (meta && a >= 0) {
+      mm.x = min(max(__ldg(drop_idx + (size_t)b * nd_max + p), 0), d.nv - 1);
+      mm.y = __float_as_int(__ldcg(salience + (size_t)b * max_vis + mm.x));
+    }
     const unsigned peers = __match_any_sync(0xffffffffu, a);
     const int rank = __popc(peers & ((1u << lane) - 1u));
     int cur = 0;
@@ -807,6 +819,7 @@ __device__ __forceinline__ void csr_block(const SampleDesc &d, int b, int max_vi
     __syncwarp();
     if (a >= 0) {
       mem_b[tot[a] + cur + rank] = p;
+      if (meta) member_meta[(size_t)b * nd_max + tot[a] + cur + rank] = mm;
       if (rank == 0) hist[warp * keep_k + a] = cur + __popc(peers);
     }
     __syncwarp();
@@ -1200,6 +1213,7 @@ struct MergeArgs {
   float eps;
   const float *salience;
   const int32_t *keep_idx, *drop_idx, *seg, *members;
+  const int2 *member_meta;   // [B, max_vis-keep_k] (visual index, weight bits) beside `members`, or nullptr
   __nv_bfloat16 *out_hidden;
   int32_t *out_pos, *src_row;
 };
@@ -1292,9 +1306,15 @@ merge_compact_kernel(MergeArgs a) {
     const int cnt = min(MERGE_LIST, m_hi - base);
     __syncthreads();                      // the previous list has been consumed
     if ((int)threadIdx.x < cnt) {
-      const int j = min(max(drop_b[min(max(mem_b[base + threadIdx.x], 0), nd_max - 1)], 0), d.nv - 1);
-      s_j[threadIdx.x] = j;
-      s_w[threadIdx.x] = sal_b[j];
+      if (a.member_meta) {
+        const int2 mm = __ldg(a.member_meta + (size_t)b * nd_max + base + threadIdx.x);
+        s_j[threadIdx.x] = min(max(mm.x, 0), d.nv - 1);
+        s_w[threadIdx.x] = __int_as_float(mm.y);
+      } else {
+        const int j = min(max(drop_b[min(max(mem_b[base + threadIdx.x], 0), nd_max - 1)], 0), d.nv - 1);
+        s_j[threadIdx.x] = j;
+        s_w[threadIdx.x] = sal_b[j];
+      }
     }
     __syncthreads();
     for (int m0 = 0; m0 < cnt; m0 += BATCH) {

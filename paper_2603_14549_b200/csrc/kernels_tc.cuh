@@ -688,6 +688,7 @@ struct SimArgs {
   const int32_t *drop_idx;   // [B, max_vis-keep_k] dropped tokens, ascending: the row operand is gathered from them;
                              // nullptr: the row operand is every visual row (tiled copies), kept rows' results unused
   const int32_t *role;       // [B, max_vis] kept slot / -(dropped position + 1) of every visual token (all-rows form)
+  const int32_t *drop_all;   // [B, max_vis-keep_k] the dropped tokens whatever the form (for member_meta), or nullptr
   const __nv_bfloat16 *hidden;   // [tokens, D] (the gather warps read the dropped rows from here)
   const float *kept_inv;     // [B*keep_k]   1/||kept row||, 0 for a zero row
   int32_t *assign;           // [B, max_vis-keep_k]
@@ -699,6 +700,8 @@ struct SimArgs {
   float *part;               // [B, max_mt, splits, keep_k, 128] partial dot products (several slices only)
   float *ss_part;            // [B, max_mt, splits, 128]         partial squared norms
   float *smat;               // [B, keep_k, keep_k] or nullptr: matrix mode
+  const float *salience;     // [B, max_vis] or nullptr: with member_meta, the merge weights the grouping copies
+  int2 *member_meta;         // [B, max_vis-keep_k] or nullptr (see csr_block)
   uint32_t *status;
   long long wait_limit;      // clock cycles a wait may take before the block gives up
 };
@@ -749,7 +752,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   SimBook *bk = reinterpret_cast<SimBook *>(base_ptr + (size_t)a.stages * stage_bytes);
   if (n_rows <= 0) {
     // nothing was dropped in this sample: only the (empty) grouping has to be written
-    if (z == 0 && gz == 0) csr_block(d, b, a.max_vis, a.keep_k, a.assign, a.seg, a.members, reinterpret_cast<int *>(base_ptr), bk->scan);
+    if (z == 0 && gz == 0) csr_block(d, b, a.max_vis, a.keep_k, a.assign, a.seg, a.members, reinterpret_cast<int *>(base_ptr), bk->scan, a.drop_all, a.salience, a.member_meta);
     return;
   }
 
@@ -1127,7 +1130,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   __threadfence();
   // the tile ring is free: every copy has landed and every MMA that read it has completed
   csr_block(d, b, a.max_vis, a.keep_k, a.assign, a.seg, a.members, reinterpret_cast<int *>(base_ptr),
-            bk->scan);
+            bk->scan, a.drop_all, a.salience, a.member_meta);
 }
 
 // =======================================================================================
@@ -1384,7 +1387,7 @@ sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
   if (!bk->is_last) return;
   __threadfence();
   csr_block(d, b, a.max_vis, a.keep_k, a.assign, a.seg, a.members, reinterpret_cast<int *>(base_ptr),
-            bk->scan);
+            bk->scan, a.drop_all, a.salience, a.member_meta);
 }
 
 }  // namespace asap
