@@ -48,6 +48,7 @@ struct asap_ctx {
   long long fuse_mass_min_tokens = 50000;   // B * max_vis from which the attention mass rides in the score kernel
   long long sim_pair_min_blocks = 0;        // blocks from which the similarity takes two row tiles per block (0: half the SM count)
   int sim_pair_stages = 0;                  // stages of that form (0: what fits 192 KB)
+  int sim_cluster = 1;                      // 0: sliced similarity launches add their partials through global memory
   float *sim_part = nullptr;        // partial dot products / squared norms of a sliced similarity GEMM
   size_t sim_part_bytes = 0, cap_tiles = 0;
   int32_t *role = nullptr, *seg = nullptr, *members = nullptr;
@@ -186,6 +187,27 @@ void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cu
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);   // errors surface in after_launch
+}
+
+// The same for a kernel whose grid-z neighbours form thread-block clusters of `cluster_z` blocks.
+template <typename... KArgs, typename... Args>
+void launch_pdl_cluster_z(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_z,
+                          Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 1;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = (unsigned)cluster_z;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 asap_status after_launch(asap_ctx *ctx, const char *what) {
@@ -330,6 +352,10 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     // The slice count minimises a simple cost: streaming a row tile takes about 1 us per 128-column
     // step of the slice, and the last slice adds up keep_k * slices partial values per row at about
     // 0.5 us per 64 of them.
+    // With one slot tile (at most 256 kept slots) the slices of a row tile run as one thread-block cluster and
+    // add their partial products through distributed shared memory: no partials in global memory, no
+    // last-block pass over them; the adding then costs about a quarter of a microsecond per slice.
+    const bool cluster_ok = ctx->sim_cluster != 0 && n_nt == 1;
     int splits = 1;
     float best_cost = (float)n_kb;
     for (int c = 2; c <= 8; ++c) {
@@ -337,7 +363,7 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
       if ((long long)max_mt * B * c > 2LL * ctx->num_sms) break;
       if ((size_t)B * max_mt * c * ((size_t)k + 1) * 128 * sizeof(float) > ctx->sim_part_bytes) break;
       if ((size_t)B * max_mt > ctx->cap_tiles) break;
-      const float cost = (float)n_kb / c + 0.5f * (float)k * c / 64.f;
+      const float cost = (float)n_kb / c + (cluster_ok ? 0.25f * c : 0.5f * (float)k * c / 64.f);
       if (cost < best_cost) { best_cost = cost; splits = c; }
     }
     // a grid between one and two blocks per SM runs as one wave if two blocks fit on an SM:
@@ -381,7 +407,7 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
         SimArgs sa;
         sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = ptile;
         sa.n_nt = 1; sa.stages = pstages; sa.splits = 1; sa.max_mt = pairs; sa.tmem_cols = pcols;
-        sa.wide = 1; sa.groups = pg; sa.threshold = p->sim_threshold;
+        sa.wide = 1; sa.groups = pg; sa.cluster = 0; sa.threshold = p->sim_threshold;
         sa.drop_idx = nullptr; sa.role = ctx->role;
         sa.hidden = static_cast<const __nv_bfloat16 *>(in->hidden); sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
         sa.best_sim = out->best_sim; sa.seg = ctx->seg; sa.members = ctx->members; sa.counters = ctx->cnt_sim;
@@ -435,6 +461,9 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     sa.n_nt = n_nt; sa.stages = stages; sa.splits = splits; sa.max_mt = max_mt; sa.tmem_cols = tmem_cols;
     sa.wide = wide ? 1 : 0;
     sa.groups = groups;
+    const bool cluster = cluster_ok && splits > 1 && !wide && !gather_rows &&
+                         (size_t)k * 512 + 4096 + (size_t)splits * 1536 <= (size_t)stages * stage_bytes_used;
+    sa.cluster = cluster ? 1 : 0;
     sa.threshold = p->sim_threshold;
     sa.drop_idx = gather_rows ? drop_idx : nullptr; sa.role = ctx->role;
     sa.hidden = static_cast<const __nv_bfloat16 *>(in->hidden); sa.kept_inv = ctx->kept_inv; sa.assign = out->assign;
@@ -447,6 +476,9 @@ asap_status launch_merge_front(asap_ctx *ctx, const asap_inputs *in, const asap_
     mark(ctx, "sim", st);
     if (gather_rows)
       launch_pdl(sim_kernel<true>, dim3(max_mt * groups, B, splits), dim3(SIM_THREADS), smem, st, map_h, map_kept, sa);
+    else if (cluster)
+      launch_pdl_cluster_z(sim_kernel<false>, dim3(max_mt, B, splits), dim3(SIM_THREADS_TILED), smem, st, splits, map_h,
+                           map_kept, sa);
     else
       launch_pdl(sim_kernel<false>, dim3(max_mt * groups, B, splits), dim3(SIM_THREADS_TILED), smem, st, map_h, map_kept, sa);
     ASAP_TRY(after_launch(ctx, "sim"));
@@ -535,6 +567,7 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   sa.n_nt = n_nt; sa.stages = stages; sa.splits = splits; sa.max_mt = max_mt; sa.tmem_cols = tmem_cols;
   sa.wide = 0;
   sa.groups = 1;
+  sa.cluster = 0;
   sa.threshold = p->sim_threshold;
   sa.drop_idx = nullptr; sa.role = nullptr; sa.hidden = nullptr; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
   sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr; sa.tile_counters = ctx->cnt_tiles;
@@ -641,6 +674,7 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   if (const char *env = getenv("ASAP_FUSE_MASS_MIN_TOKENS")) ctx->fuse_mass_min_tokens = atoll(env);
   if (const char *env = getenv("ASAP_SIM_PAIR_MIN_BLOCKS")) ctx->sim_pair_min_blocks = atoll(env);
   if (const char *env = getenv("ASAP_SIM_PAIR_STAGES")) ctx->sim_pair_stages = atoi(env);
+  if (const char *env = getenv("ASAP_SIM_CLUSTER")) ctx->sim_cluster = atoi(env);
   ctx->inv_norm = reinterpret_cast<float *>(ctx->arena + o_inv);
   ctx->kept_inv = reinterpret_cast<float *>(ctx->arena + o_kinv);
   ctx->counters_off = o_cnt; ctx->counters_bytes = (Bc * col_blocks + 3 * Bc + 2) * sizeof(unsigned int);

@@ -683,6 +683,8 @@ struct SimArgs {
   int D, max_vis, keep_k, n_tile, n_nt, stages, splits, max_mt;
   int wide;                  // 1: one pass, all slot tiles' accumulators live at once
   int groups;                // > 1: slot tiles dealt to `groups` blocks per row tile (n_nt counts one group's tiles)
+  int cluster;               // 1: the `splits` slices of a row tile form a thread-block cluster (grid z) and add their
+                             // partial products through distributed shared memory instead of `part`
   uint32_t tmem_cols;        // power of two >= 2 * n_tile: two accumulators
   float threshold;
   const int32_t *drop_idx;   // [B, max_vis-keep_k] dropped tokens, ascending: the row operand is gathered from them;
@@ -711,6 +713,7 @@ struct SimBook {
   uint32_t tmem_base;
   int abort_flag;
   int is_last;
+  int skip;                  // cluster form: an earlier similarity kernel of this call gave up
   int scan[33];
   int rows[128];             // packed row of each of the tile's dropped tokens (main mode)
 };
@@ -740,7 +743,8 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   constexpr bool gather = GATHER;                        // a.drop_idx given, not matrix mode
   const int n_rows = a.smat ? a.keep_k : (gather ? nd : d.nv);   // rows of the row operand
   if (mt * 128 >= max(n_rows, 1)) return;
-  if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SIM_TIMEOUT) return;
+  // (in the cluster form the blocks of a cluster must leave together: decided below, by the cluster's first block)
+  if (!a.cluster && (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SIM_TIMEOUT)) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -768,7 +772,15 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     mbar_init(smem_u32(&bk->mma_done), 1);
     bk->abort_flag = 0;
     bk->is_last = 0;
+    bk->skip = (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SIM_TIMEOUT) ? 1 : 0;
     fence_barrier_init();
+  }
+  if (a.cluster) {
+    cluster_sync_all();
+    if (ld_cluster_s32(cluster_map(smem_u32(&bk->skip), 0))) {
+      cluster_sync_all();                                // the first block's shared memory has been read by all
+      return;
+    }
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(&bk->tmem_base), a.tmem_cols);
@@ -779,6 +791,17 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   tc_fence_after();
   const uint32_t tmem_base = bk->tmem_base;
   WaitCtx wc{&bk->abort_flag, a.status, STATUS_SIM_TIMEOUT, a.wait_limit};
+  // cluster form, in the tile ring once it is free: this slice's partial products [keep_k][128]; per quarter
+  // of this block's share of the slots the rows' best (value [4][128], slot [4][128]); and, filled by all
+  // blocks in the cluster's first block, every slice's partial squared norms and every block's best
+  // (value, slot) ([splits][128] each)
+  const int cl_per = (a.keep_k + a.splits - 1) / a.splits;
+  float *cl_p = reinterpret_cast<float *>(base_ptr);
+  float *cl_wv = cl_p + (size_t)a.keep_k * 128;
+  int *cl_ws = reinterpret_cast<int *>(cl_wv + 4 * 128);
+  float *cl_ss = reinterpret_cast<float *>(cl_ws + 4 * 128);
+  float *cl_bv = cl_ss + a.splits * 128;
+  int *cl_bs = reinterpret_cast<int *>(cl_bv + a.splits * 128);
   // steps of this slice: 128 columns each, or 64 in the one-pass layout
   const int n_kb = a.wide ? (a.D / 64) / a.splits : (a.D / 128) / a.splits;
   const int kb0 = z * n_kb;
@@ -828,6 +851,8 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
         }
       }
     }
+    __syncwarp();
+    if (a.cluster) { cluster_sync_all(); cluster_sync_all(); }   // the two barriers of the epilogue warps' reduction
   } else if (warp >= 6) {
     // ---- gather warps (main mode): warp g fetches its share of the tile's rows (128 / SIM_GWARPS hidden rows
     // of dropped tokens), one stage's columns at a time.  A warp instruction covers whole rows
@@ -925,6 +950,8 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       tc_commit(smem_u32(&bk->mma_done));
       mbar_wait_drain(smem_u32(&bk->mma_done), 0, TC_WAIT_LIMIT);
     }
+    __syncwarp();
+    if (a.cluster) { cluster_sync_all(); cluster_sync_all(); }
   } else {
     const int quarter = warp & 3;
     const int lrow = quarter * 32 + lane;
@@ -960,7 +987,12 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     float best = -INFINITY;
     int best_slot = 0;
     float *part = nullptr;
-    if (a.splits > 1) {
+    if (a.cluster) {
+      // the four epilogue warps are done reading the row tiles for the norms: from here on the ring only
+      // holds stages the MMAs still read, and those are complete once acc_full has been passed
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      part = cl_p;
+    } else if (a.splits > 1) {
       const size_t tile = ((size_t)b * a.max_mt + mt) * a.splits + z;
       part = a.part + tile * (size_t)a.keep_k * 128;
       a.ss_part[tile * 128 + lrow] = ss;
@@ -1007,7 +1039,71 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
     }
     float ss_tot = ss;
     bool finalize = true;
-    if (a.splits > 1) {
+    if (a.cluster) {
+      // ---- the slices of this row tile are the blocks of one cluster.  Block r adds, in slice order, the
+      // partial products of ITS share of the kept slots, read from every block's shared memory: warp q takes
+      // every fourth slot of the share, a lane four neighbouring rows (one 16-byte load per slice).  The
+      // warps' bests per row are merged (larger value, lower slot among equals), handed to the cluster's
+      // first block, and that block takes the maximum over the blocks in ascending slots.
+      const int rank = (int)cluster_cta_rank(), S = a.splits;
+      st_cluster_f32(cluster_map(smem_u32(cl_ss), 0) + (uint32_t)(rank * 128 + lrow) * 4u, ss);
+      cluster_sync_all();
+      const int s_lo = min(a.keep_k, rank * cl_per), n_mine = min(a.keep_k, s_lo + cl_per) - s_lo;
+      uint32_t pz[8];
+#pragma unroll
+      for (int zz = 0; zz < 8; ++zz)
+        pz[zz] = cluster_map(smem_u32(cl_p), (uint32_t)min(zz, S - 1)) + (uint32_t)lane * 16u;
+      float wb[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      int wsl[4] = {0, 0, 0, 0};
+      for (int i = quarter; i < n_mine; i += 4) {
+        const int slot = s_lo + i;
+        float4 x[8];
+#pragma unroll
+        for (int zz = 0; zz < 8; ++zz)
+          if (zz < S) x[zz] = ld_cluster_v4f32(pz[zz] + (uint32_t)slot * 512u);
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int zz = 0; zz < 8; ++zz)
+          if (zz < S) { acc[0] += x[zz].x; acc[1] += x[zz].y; acc[2] += x[zz].z; acc[3] += x[zz].w; }
+        const float ks = __ldg(kinv + slot);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (a.smat) {
+            const int vr = mt * 128 + lane * 4 + j;
+            if (vr < a.keep_k && !bk->abort_flag)
+              a.smat[((size_t)b * a.keep_k + vr) * a.keep_k + slot] = acc[j] * (__ldg(kinv + vr) * ks);
+          } else {
+            const float val = acc[j] * ks;
+            if (val > wb[j]) { wb[j] = val; wsl[j] = slot; }
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        cl_wv[quarter * 128 + lane * 4 + j] = wb[j];
+        cl_ws[quarter * 128 + lane * 4 + j] = wsl[j];
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      for (int q2 = 0; q2 < 4; ++q2) {
+        const float val = cl_wv[q2 * 128 + lrow];
+        const int sl = cl_ws[q2 * 128 + lrow];
+        if (val > best || (val == best && val > -INFINITY && sl < best_slot)) { best = val; best_slot = sl; }
+      }
+      st_cluster_f32(cluster_map(smem_u32(cl_bv), 0) + (uint32_t)(rank * 128 + lrow) * 4u, best);
+      st_cluster_s32(cluster_map(smem_u32(cl_bs), 0) + (uint32_t)(rank * 128 + lrow) * 4u, best_slot);
+      cluster_sync_all();
+      finalize = rank == 0;
+      if (finalize) {
+        ss_tot = 0.f;
+        for (int r2 = 0; r2 < S; ++r2) ss_tot += cl_ss[r2 * 128 + lrow];
+        best = -INFINITY;
+        best_slot = 0;
+        for (int r2 = 0; r2 < S; ++r2) {                    // ascending slots: the first maximum stays
+          const float val = cl_bv[r2 * 128 + lrow];
+          if (val > best) { best = val; best_slot = cl_bs[r2 * 128 + lrow]; }
+        }
+      }
+    } else if (a.splits > 1) {
       // publish this slice; the last slice to arrive for the row tile reduces all of them
       __threadfence();
       asm volatile("bar.sync 1, 128;" ::: "memory");
