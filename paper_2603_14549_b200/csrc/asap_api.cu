@@ -541,6 +541,7 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   // slices of the hidden dimension, chosen by the cost model of the similarity launch
   const int max_mt = (k + 127) / 128;
   const int n_kb = D / 128;
+  const bool cluster_ok = ctx->sim_cluster != 0 && n_nt == 1;   // slices as a thread-block cluster (see the similarity launch)
   int splits = 1;
   float best_cost = (float)n_kb;
   for (int c = 2; c <= 8; ++c) {
@@ -548,7 +549,7 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
     if ((long long)max_mt * B * c > 2LL * ctx->num_sms) break;
     if ((size_t)B * max_mt * c * ((size_t)k + 1) * 128 * sizeof(float) > ctx->sim_part_bytes) break;
     if ((size_t)B * max_mt > ctx->cap_tiles) break;
-    const float cost = (float)n_kb / c + 0.5f * (float)k * c / 64.f;
+    const float cost = (float)n_kb / c + (cluster_ok ? 0.25f * c : 0.5f * (float)k * c / 64.f);
     if (cost < best_cost) { best_cost = cost; splits = c; }
   }
   const long long ctas = (long long)max_mt * B * splits;
@@ -567,7 +568,9 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   sa.n_nt = n_nt; sa.stages = stages; sa.splits = splits; sa.max_mt = max_mt; sa.tmem_cols = tmem_cols;
   sa.wide = 0;
   sa.groups = 1;
-  sa.cluster = 0;
+  const bool cluster = cluster_ok && splits > 1 &&
+                       (size_t)k * 512 + 4096 + (size_t)splits * 1536 <= (size_t)stages * stage_bytes;
+  sa.cluster = cluster ? 1 : 0;
   sa.threshold = p->sim_threshold;
   sa.drop_idx = nullptr; sa.role = nullptr; sa.hidden = nullptr; sa.kept_inv = ctx->kept_inv; sa.assign = nullptr; sa.best_sim = nullptr;
   sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr; sa.tile_counters = ctx->cnt_tiles;
@@ -575,7 +578,10 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   sa.smat = smat; sa.drop_all = nullptr; sa.salience = nullptr; sa.member_meta = nullptr;
   sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
   mark(ctx, "sim_kept", st);
-  launch_pdl(sim_kernel<false>, dim3(max_mt, B, splits), dim3(SIM_THREADS_TILED), smem, st, map_a, map_b, sa);
+  if (cluster)
+    launch_pdl_cluster_z(sim_kernel<false>, dim3(max_mt, B, splits), dim3(SIM_THREADS_TILED), smem, st, splits, map_a, map_b, sa);
+  else
+    launch_pdl(sim_kernel<false>, dim3(max_mt, B, splits), dim3(SIM_THREADS_TILED), smem, st, map_a, map_b, sa);
   ASAP_TRY(after_launch(ctx, "sim_kept"));
 
   RouteArgs ra;
