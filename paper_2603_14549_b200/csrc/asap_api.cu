@@ -533,6 +533,40 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
              static_cast<const __nv_bfloat16 *>(in->hidden), ctx->desc, D, k, keep_idx, ctx->kept_rows, ctx->kept_inv);
   ASAP_TRY(after_launch(ctx, "kept_gather"));
 
+  float *smat = static_cast<float *>(scratch);
+  {
+    // large batches: two row tiles per block, the slots dealt in groups to neighbouring blocks (see the similarity
+    // launch of the merge); here every product is used, the matrix being square
+    const int pairs = (k + 255) / 256;
+    const int pg = (k + 255) / 256;
+    const int ptile = (((k + pg - 1) / pg) + 15) & ~15;
+    const long long min_blocks = ctx->sim_pair_min_blocks > 0 ? ctx->sim_pair_min_blocks : (ctx->num_sms + 1) / 2;
+    const int pstage = 2 * SIM_A_BYTES + ptile * 128;
+    int pstages = ctx->sim_pair_stages > 0 ? ctx->sim_pair_stages : (192 * 1024) / pstage;
+    if (pstages > SIM_MAX_STAGES) pstages = SIM_MAX_STAGES;
+    const size_t psmem = (size_t)pstages * pstage + SIM_BOOK_BYTES + 1024;
+    if (D % 64 == 0 && (long long)pairs * B * pg >= min_blocks && pstages >= 2 && psmem <= 227 * 1024) {
+      uint32_t pcols = 32;
+      while ((int)pcols < 2 * ptile) pcols <<= 1;
+      CUtensorMap map_a, map_b;
+      if (!make_map(ctx, &map_a, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, 128) ||
+          !make_map(ctx, &map_b, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, (uint32_t)ptile))
+        return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for the kept rows");
+      SimArgs sa;
+      sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = ptile;
+      sa.n_nt = 1; sa.stages = pstages; sa.splits = 1; sa.max_mt = pairs; sa.tmem_cols = pcols;
+      sa.wide = 1; sa.groups = pg; sa.cluster = 0; sa.threshold = p->sim_threshold;
+      sa.drop_idx = nullptr; sa.role = nullptr; sa.drop_all = nullptr; sa.hidden = nullptr; sa.kept_inv = ctx->kept_inv;
+      sa.assign = nullptr; sa.best_sim = nullptr; sa.seg = nullptr; sa.members = nullptr; sa.counters = nullptr;
+      sa.tile_counters = nullptr; sa.part = nullptr; sa.ss_part = nullptr; sa.smat = smat; sa.salience = nullptr;
+      sa.member_meta = nullptr; sa.status = ctx->status; sa.wait_limit = ctx->wait_limit;
+      mark(ctx, "sim_kept", st);
+      launch_pdl(sim_pair_kernel, dim3(pairs * pg, B), dim3(SIMP_THREADS), psmem, st, map_a, map_b, sa);
+      ASAP_TRY(after_launch(ctx, "sim_kept"));
+      goto routing;
+    }
+  }
+  {
   const int n_nt = (k + 255) / 256;
   const int n_tile = (((k + n_nt - 1) / n_nt) + 15) & ~15;
   const int stage_bytes = 2 * (SIM_A_BYTES + n_tile * 128);
@@ -562,7 +596,6 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   if (!make_map(ctx, &map_a, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, 128) ||
       !make_map(ctx, &map_b, ctx->kept_rows, (uint64_t)B * (uint64_t)k, (uint64_t)D, (uint32_t)n_tile))
     return fail(ctx, ASAP_ERR_CUDA, "cuTensorMapEncodeTiled failed for the kept rows");
-  float *smat = static_cast<float *>(scratch);
   SimArgs sa;
   sa.desc = ctx->desc; sa.D = D; sa.max_vis = in->max_vis; sa.keep_k = k; sa.n_tile = n_tile;
   sa.n_nt = n_nt; sa.stages = stages; sa.splits = splits; sa.max_mt = max_mt; sa.tmem_cols = tmem_cols;
@@ -583,7 +616,8 @@ asap_status launch_consolidate_front(asap_ctx *ctx, const asap_inputs *in, const
   else
     launch_pdl(sim_kernel<false>, dim3(max_mt, B, splits), dim3(SIM_THREADS_TILED), smem, st, map_a, map_b, sa);
   ASAP_TRY(after_launch(ctx, "sim_kept"));
-
+  }
+routing:
   RouteArgs ra;
   ra.desc = ctx->desc; ra.max_vis = in->max_vis; ra.keep_k = k; ra.kw = (k + 31) / 32;
   ra.threshold = p->sim_threshold; ra.smat = smat;

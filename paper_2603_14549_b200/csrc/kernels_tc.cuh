@@ -1250,6 +1250,8 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
 // its rows' best (value, slot); the block that finishes a pair last takes the maximum over the
 // groups (lowest slot among equals), looks up which rows were dropped and writes their assignment.
 // The block that finishes a sample's last pair groups the dropped tokens by destination.
+// Matrix mode (a.smat set): the row operand is the dense kept-row array too (`tmap_h` maps it with a 128-row box)
+// and every block writes its 256 x n_tile piece of the sample's keep_k x keep_k cosine matrix; nothing else.
 // =======================================================================================
 constexpr int SIMP_THREADS = 320;                // copy warp, MMA warp, two groups of four epilogue warps
 
@@ -1273,7 +1275,7 @@ sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
   const SampleDesc d = a.desc[b];
   if (!d.valid) return;
   const int nd = d.nv - a.keep_k;
-  const int n_rows = d.nv;
+  const int n_rows = a.smat ? a.keep_k : d.nv;           // matrix mode: the row operand is the dense kept-row array
   if (pr * 256 >= n_rows) return;
   if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SIM_TIMEOUT) return;
   const bool two = pr * 256 + 128 < n_rows;              // the pair's second row tile holds visual rows
@@ -1287,7 +1289,7 @@ sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
   SimPairBook *bk = reinterpret_cast<SimPairBook *>(base_ptr + (size_t)a.stages * stage_bytes);
 
   // the epilogue warps of group 0 read their row tile from the stages (for the row norms)
-  const int n_readers = gz == 0 ? (two ? 8 : 4) : 0;
+  const int n_readers = (gz == 0 && !a.smat) ? (two ? 8 : 4) : 0;   // (matrix mode takes the norms from kept_inv)
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.stages; ++s) {
       mbar_init(smem_u32(&bk->full[s]), 1);
@@ -1317,7 +1319,7 @@ sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
     if (lane == 0) {
       tma_prefetch_desc(&tmap_h);
       tma_prefetch_desc(&tmap_kept);
-      const int row_a = d.row0 + d.v0 + pr * 256;
+      const int row_a = a.smat ? b * a.keep_k + pr * 256 : d.row0 + d.v0 + pr * 256;
       const int row_b = b * a.keep_k + gz * a.n_tile;
       const int tx_bytes = two ? stage_bytes : stage_bytes - SIM_A_BYTES;
       int issued = 0;
@@ -1374,7 +1376,7 @@ sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
     const float *kinv = a.kept_inv + (size_t)b * a.keep_k;
     // ---- squared norm of this thread's row (group 0 only; the other groups just free the stages)
     float ssq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    const bool norms = gz == 0 && active;
+    const bool norms = gz == 0 && active && !a.smat;
     for (int it = 0; it < (norms ? n_kb : 0); ++it) {
       const int s = it % a.stages;
       mbar_wait(smem_u32(&bk->full[s]), (it / a.stages) & 1, wc);
@@ -1403,11 +1405,32 @@ sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
     const int ncol = max(0, min(a.n_tile, a.keep_k - slot0));
     if (active && !bk->abort_flag) {
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + grp * a.n_tile;
+      const float inv_p = (a.smat && v < a.keep_k) ? __ldg(kinv + v) : 0.f;
 #pragma unroll 1
       for (int c = 0; c < ncol; c += 16) {
         uint32_t r[16];
         tmem_ld16(taddr + c, r);
         tmem_wait_ld();
+        if (a.smat) {
+          // matrix mode: S[p][q] = <h_p, h_q> * (1/||h_p|| * 1/||h_q||) for this thread's kept row p
+          if (v < a.keep_k) {
+            float *srow = a.smat + ((size_t)b * a.keep_k + v) * a.keep_k + slot0 + c;
+            if (c + 16 <= ncol && (reinterpret_cast<size_t>(srow) & 15) == 0) {
+#pragma unroll
+              for (int e = 0; e < 16; e += 4)         // 16-byte stores: a quarter of the store requests
+                reinterpret_cast<float4 *>(srow)[e >> 2] =
+                    make_float4(__uint_as_float(r[e]) * (inv_p * __ldg(kinv + slot0 + c + e)),
+                                __uint_as_float(r[e + 1]) * (inv_p * __ldg(kinv + slot0 + c + e + 1)),
+                                __uint_as_float(r[e + 2]) * (inv_p * __ldg(kinv + slot0 + c + e + 2)),
+                                __uint_as_float(r[e + 3]) * (inv_p * __ldg(kinv + slot0 + c + e + 3)));
+            } else {
+#pragma unroll
+              for (int e = 0; e < 16; ++e)
+                if (c + e < ncol) srow[e] = __uint_as_float(r[e]) * (inv_p * __ldg(kinv + slot0 + c + e));
+            }
+          }
+          continue;
+        }
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
           const int slot = slot0 + c + e;
@@ -1419,8 +1442,8 @@ sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
       }
     }
     tc_fence_before();
-    bool finalize = true;
-    if (a.groups > 1) {
+    bool finalize = !a.smat;
+    if (a.groups > 1 && !a.smat) {
       // per pair: [group][best of 256 rows | slot of 256 rows], then the 256 squared norms
       float *pp = a.part + ((size_t)b * a.max_mt + pr) * (size_t)(a.groups * 512 + 256);
       pp[gz * 512 + prow] = best;
@@ -1470,7 +1493,7 @@ sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
     tc_fence_after();
     tmem_dealloc(tmem_base, a.tmem_cols);
   }
-  if (!bk->is_last) return;                              // a group that did not finalize its pair
+  if (!bk->is_last) return;                              // a group that did not finalize its pair (or matrix mode)
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
