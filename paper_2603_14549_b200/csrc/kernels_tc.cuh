@@ -247,6 +247,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       int kc = 0, qc = 0, g = 0, ic = 0, mc = 0;      // mc: items whose summed-query rows were waited for
       bool issued_any = false;
       const uint32_t idesc1 = umma_idesc_bf16(128, 128);
+      const uint64_t qdesc = umma_desc_sw128(q_smem);          // (every tile lies below 256 KB: offsets never carry out of the address field)
       while (true) {
         const int slot = ic % SC_ITEM_SLOTS;
         const bool got = mbar_wait_drain(smem_u32(&bk->item_full[slot]), (ic / SC_ITEM_SLOTS) & 1, TC_WAIT_LIMIT);
@@ -276,18 +277,13 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             if (!bk->abort_flag) {
               const uint32_t ks = k_smem + s * SC_TILE_BYTES;
               const uint32_t dcol = tmem_base + hh * 256;
+              const uint64_t kdesc = umma_desc_sw128(ks);
               if (pass1) {
-                for (int rt = 0; rt < T.nrt; ++rt)
-#pragma unroll
-                  for (int kk = 0; kk < 8; ++kk)
-                    tc_mma_bf16(dcol + rt * 128,
-                                umma_desc_sw128(q_smem + (kk >> 2) * SC_Q_HALF_BYTES + rt * SC_HALF_BYTES + (kk & 3) * 32),
-                                umma_desc_sw128(ks + (kk >> 2) * SC_HALF_BYTES + (kk & 3) * 32), idesc1, kk > 0);
+                tc_mma_bf16_k128<SC_Q_HALF_BYTES, SC_HALF_BYTES>(dcol, qdesc, kdesc, idesc1);
+                if (T.nrt == 2)
+                  tc_mma_bf16_k128<SC_Q_HALF_BYTES, SC_HALF_BYTES>(dcol + 128, qdesc + (SC_HALF_BYTES >> 4), kdesc, idesc1);
               } else {
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                  tc_mma_bf16(dcol, umma_desc_sw128(ks + (kk >> 2) * SC_HALF_BYTES + (kk & 3) * 32),
-                              umma_desc_sw128(q_smem + (kk >> 2) * SC_Q_HALF_BYTES + (kk & 3) * 32), idesc2, kk > 0);
+                tc_mma_bf16_k128<SC_HALF_BYTES, SC_Q_HALF_BYTES>(dcol, kdesc, qdesc, idesc2);
               }
               tc_commit(smem_u32(&bk->empty[s]));
               tc_commit(smem_u32(&bk->acc_full[hh]));
