@@ -505,7 +505,12 @@ asap_status launch_merge_back(asap_ctx *ctx, const asap_inputs *in, const asap_p
   mark(ctx, "merge_compact", st);
   switch (nv) {
     case 1: launch_pdl(merge_compact_kernel<1>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
-    case 2: launch_pdl(merge_compact_kernel<2>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
+    case 2:
+      if ((long long)grid.x * grid.y >= 32LL * 3 * ctx->num_sms)       // more than 32 waves of three blocks per SM
+        launch_pdl(merge_compact_kernel<2, true>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma);
+      else
+        launch_pdl(merge_compact_kernel<2>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma);
+      break;
     case 3: launch_pdl(merge_compact_kernel<3>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
     default: launch_pdl(merge_compact_kernel<4>, dim3(grid), dim3(MERGE_THREADS), 0, st, ma); break;
   }

@@ -1220,10 +1220,13 @@ struct MergeArgs {
 
 // NV: 16-byte vectors per thread (D <= NV * 256 * 8); wide rows keep fewer member rows in flight per thread
 // so that three blocks still fit the register file of an SM.
-template <int NV>
-__global__ void __launch_bounds__(MERGE_THREADS, NV >= 4 ? 2 : 3)
+// LEAN (rows of at most 4096 elements, launches of many waves): two member rows in flight as well, 60 registers,
+// four blocks per SM -- more blocks in their dependent look-ups at any time (c4 398 -> 369 us); on launches of a
+// few waves the shorter batches cost more than the occupancy gives (c2 24.8 -> 26.6 us), so those keep four rows.
+template <int NV, bool LEAN = false>
+__global__ void __launch_bounds__(MERGE_THREADS, NV >= 4 ? 2 : (LEAN ? 4 : 3))
 merge_compact_kernel(MergeArgs a) {
-  constexpr int BATCH = NV >= 3 ? 2 : MERGE_BATCH;
+  constexpr int BATCH = (NV >= 3 || LEAN) ? 2 : MERGE_BATCH;
   pdl_enter();
   __shared__ int s_j[MERGE_LIST];
   __shared__ float s_w[MERGE_LIST];
