@@ -1219,14 +1219,16 @@ struct MergeArgs {
 };
 
 // NV: 16-byte vectors per thread (D <= NV * 256 * 8); wide rows keep fewer member rows in flight per thread
-// so that three blocks still fit the register file of an SM.
+// so that three or four blocks still fit the register file of an SM.
 // LEAN (rows of at most 4096 elements, launches of many waves): two member rows in flight as well, 60 registers,
 // four blocks per SM -- more blocks in their dependent look-ups at any time (c4 398 -> 369 us); on launches of a
 // few waves the shorter batches cost more than the occupancy gives (c2 24.8 -> 26.6 us), so those keep four rows.
+// Rows of 4097-6144 elements (NV = 3): one member row in flight, 64 registers, four blocks per SM as well
+// (D = 5120, 1152 of 2304 kept: 280 -> 241 us; 576 of 1152: 151 -> 133 us; 288 of 576: 85 -> 75 us).
 template <int NV, bool LEAN = false>
-__global__ void __launch_bounds__(MERGE_THREADS, NV >= 4 ? 2 : (LEAN ? 4 : 3))
+__global__ void __launch_bounds__(MERGE_THREADS, NV >= 4 ? 2 : ((LEAN || NV == 3) ? 4 : 3))
 merge_compact_kernel(MergeArgs a) {
-  constexpr int BATCH = (NV >= 3 || LEAN) ? 2 : MERGE_BATCH;
+  constexpr int BATCH = NV == 3 ? 1 : ((NV >= 4 || LEAN) ? 2 : MERGE_BATCH);
   pdl_enter();
   __shared__ int s_j[MERGE_LIST];
   __shared__ float s_w[MERGE_LIST];
