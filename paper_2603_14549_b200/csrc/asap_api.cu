@@ -250,17 +250,30 @@ asap_status launch_prepare(asap_ctx *ctx, const asap_inputs *in, const asap_para
 
 // Steps 1a-1b: query sum, attention mass, salience, mask vector.  With `fold_prepare` the query-sum
 // kernel also carries the device-side validation and writes the descriptors.
+
+// Rows a block of the query-sum kernel adds up: 32, doubled (up to 128) while the grid still has eight blocks per
+// SM -- every chunk costs a partial row written and read back (32 rows: 12 % on top of the queries themselves).
+int qsum_rows_per_chunk(const asap_ctx *ctx, const asap_inputs *in) {
+  const long long col_blocks = (in->D + QSUM_COLS - 1) / QSUM_COLS;
+  int rows = QSUM_ROWS;
+  while (rows < 4 * QSUM_ROWS &&
+         (long long)((in->max_vis + 2 * rows - 1) / (2 * rows)) * col_blocks * in->B >= 8LL * ctx->num_sms)
+    rows *= 2;
+  return rows;
+}
+
 asap_status launch_mass(asap_ctx *ctx, const asap_inputs *in, const asap_params *p, const asap_outputs *out,
                         bool fold_prepare, int32_t *out_cu, int out_capacity, cudaStream_t st,
                         cudaEvent_t after_qsum = nullptr) {
   const int D = in->D, B = in->B;
-  const int max_chunks = (in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS;
+  const int qrows = qsum_rows_per_chunk(ctx, in);
+  const int max_chunks = (in->max_vis + qrows - 1) / qrows;
   const int col_blocks = (D + QSUM_COLS - 1) / QSUM_COLS;
   PrepareArgs pa = prepare_args(ctx, in, p, out_cu, out_capacity);
   pa.write_desc = fold_prepare ? 1 : 0;
   mark(ctx, "qsum", st);
   launch_pdl(qsum_kernel, dim3(max_chunks, col_blocks, B), dim3(QSUM_THREADS), 0, st,
-             static_cast<const __nv_bfloat16 *>(in->q), pa, D, max_chunks, ctx->qsum_partial, ctx->qbar,
+             static_cast<const __nv_bfloat16 *>(in->q), pa, D, max_chunks, qrows, ctx->qsum_partial, ctx->qbar,
              ctx->cnt_qsum);
   ASAP_TRY(after_launch(ctx, "qsum"));
   if (after_qsum && cudaEventRecord(after_qsum, st) != cudaSuccess)
@@ -885,10 +898,11 @@ asap_status asap_prune_step(asap_ctx *ctx, const asap_inputs *in, const asap_par
     // query sum (carrying the validation) -> score kernel with two more columns per key tile -> Eq. 2-3.
     PrepareArgs pa = prepare_args(ctx, in, p, out->out_cu_seqlens, out->out_rows_capacity);
     pa.write_desc = 1;
-    const int max_chunks = (in->max_vis + QSUM_ROWS - 1) / QSUM_ROWS;
+    const int qrows = qsum_rows_per_chunk(ctx, in);
+    const int max_chunks = (in->max_vis + qrows - 1) / qrows;
     mark(ctx, "qsum", st);
     launch_pdl(qsum_kernel, dim3(max_chunks, (in->D + QSUM_COLS - 1) / QSUM_COLS, in->B), dim3(QSUM_THREADS), 0, st,
-               static_cast<const __nv_bfloat16 *>(in->q), pa, in->D, max_chunks, ctx->qsum_partial, ctx->qbar, ctx->cnt_qsum);
+               static_cast<const __nv_bfloat16 *>(in->q), pa, in->D, max_chunks, qrows, ctx->qsum_partial, ctx->qbar, ctx->cnt_qsum);
     ASAP_TRY(after_launch(ctx, "qsum"));
     ASAP_TRY(launch_rank(ctx, in, p, out, false, st, true));
     mark(ctx, "salience", st);

@@ -95,7 +95,7 @@ constexpr int QSUM_COLS = QSUM_THREADS * 8;
 
 __global__ void __launch_bounds__(QSUM_THREADS)
 qsum_kernel(const __nv_bfloat16 *__restrict__ q, PrepareArgs pa, int D,
-            int max_chunks, float *__restrict__ partial /*[B, max_chunks, D]*/,
+            int max_chunks, int rows_per_chunk /* a multiple of QSUM_ROWS */, float *__restrict__ partial /*[B, max_chunks, D]*/,
             float *__restrict__ qbar /*[B, D]*/, unsigned int *__restrict__ counters) {
   pdl_enter();
   const int b = blockIdx.z, cb = blockIdx.y, chunk = blockIdx.x;
@@ -104,14 +104,14 @@ qsum_kernel(const __nv_bfloat16 *__restrict__ q, PrepareArgs pa, int D,
   if (pa.write_desc && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) prepare_block(pa);
   const SampleDesc d = make_desc(pa, b);
   if (!d.valid) return;
-  const int nchunks = (d.nv + QSUM_ROWS - 1) / QSUM_ROWS;
+  const int nchunks = (d.nv + rows_per_chunk - 1) / rows_per_chunk;
   if (chunk >= nchunks) return;
   const int col = cb * QSUM_COLS + threadIdx.x * 8;
   const bool active = col < D;
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   if (active) {
-    const int r_lo = chunk * QSUM_ROWS;
-    const int r_hi = min(d.nv, r_lo + QSUM_ROWS);
+    const int r_lo = chunk * rows_per_chunk;
+    const int r_hi = min(d.nv, r_lo + rows_per_chunk);
     const uint4 *base =
         reinterpret_cast<const uint4 *>(q + (size_t)(d.row0 + d.v0) * D + col);
     const size_t pitch = (size_t)D / 8;
