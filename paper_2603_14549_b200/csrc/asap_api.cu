@@ -761,6 +761,24 @@ asap_status asap_init(asap_ctx **ctx_out, int device, size_t max_total_tokens, i
   if (e == cudaSuccess) e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM_BYTES);
+  if (e == cudaSuccess && ctx->sim_cluster) {
+    // the cluster form of the sliced similarity launch needs eight co-resident blocks of up to 195 KB each in one
+    // cluster; where the device (or the partition of it this process sees) cannot place one, the form is not used
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1, 1, 8);
+    cfg.blockDim = dim3(SIM_THREADS_TILED);
+    cfg.dynamicSmemBytes = 195 * 1024;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 8;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, sim_kernel<false>, &cfg) != cudaSuccess || clusters < 1) {
+      ctx->sim_cluster = 0;
+      cudaGetLastError();
+    }
+  }
   // lowest priority: when both streams have blocks to place, the score kernel's go first and the
   // mass kernels fill what is left of each SM
   int prio_least = 0, prio_greatest = 0;
