@@ -1,7 +1,9 @@
 """The similarity launch picks one of several kernel forms from the problem size.  The large-batch form
 (two row tiles per block, kept slots in groups, Sec. 4.2's assignment) is forced here onto small ragged
 inputs, so that its edges are compared with the oracle element by element: a second row tile that is
-empty, one that is partly filled, several slot groups with a ragged last group, nothing dropped."""
+empty, one that is partly filled, several slot groups with a ragged last group, nothing dropped.  The
+small-problem form whose slices of the hidden dimension are a thread-block cluster (2, 4 or 8 blocks adding
+their partial products through distributed shared memory) is reached with wider hidden states."""
 import os
 
 import numpy as np
@@ -33,16 +35,9 @@ def ctx_pair_form():
     A.asap_free(c)
 
 
-@pytest.mark.parametrize("n_vis,k", [
-    ([520, 300, 257], 40),      # three / two / two row tiles: pairs with a full, a partial and an empty second tile
-    ([600, 513], 257),          # two groups of 144 slots, the second ragged (113 slots)
-    ([256, 300], 256),          # sample 0 drops nothing
-    ([129, 1000], 17),          # one group narrower than an MMA's smallest useful width
-])
-def test_pair_form_matches_the_oracle(ctx_pair_form, n_vis, k):
-    ctx = ctx_pair_form
+def _merge_matches_oracle(ctx, n_vis, k, H, seed):
     B = len(n_vis)
-    batch = W.tiny(B=B, n_vis=n_vis, text_lens=[5 + 3 * b for b in range(B)], H=2, keep_k=k, seed=911, centres=9)
+    batch = W.tiny(B=B, n_vis=n_vis, text_lens=[5 + 3 * b for b in range(B)], H=H, keep_k=k, seed=seed, centres=9)
     p = A.Params(keep_k=k)
     inp = A.make_inputs(batch, DEV)
     mv = inp.max_vis
@@ -82,6 +77,33 @@ def test_pair_form_matches_the_oracle(ctx_pair_form, n_vis, k):
         gh = O.bf16_bits_to_f64(bits(out.out_hidden[int(ocu[b]):int(ocu[b + 1])].cpu()))
         assert np.all(np.abs(gh - ref2["out_hidden"]) <= merged_tolerance(ref2["out_hidden"])), b
         assert np.array_equal(out.out_pos[int(ocu[b]):int(ocu[b + 1])].cpu().numpy(), ref2["out_pos"])
+
+
+@pytest.fixture(scope="module")
+def ctx_default():
+    c = A.asap_init(0, max_total_tokens=40000, max_B=8, max_H=8, max_D=1024, max_keep_rows=8000)
+    yield c
+    A.asap_free(c)
+
+
+@pytest.mark.parametrize("n_vis,k,H", [
+    ([300, 129], 100, 8),        # hidden size 1024: eight slices per row tile, ragged last row tiles
+    ([640], 256, 8),             # the widest single slot tile, 384 dropped rows
+    ([200, 130, 131], 16, 4),    # hidden size 512: four slices, one narrow slot tile
+    ([129, 129, 129, 129, 129, 129, 129, 129], 33, 8),   # sixteen row tiles: fewer slices per tile
+])
+def test_cluster_form_matches_the_oracle(ctx_default, n_vis, k, H):
+    _merge_matches_oracle(ctx_default, n_vis, k, H, seed=933)
+
+
+@pytest.mark.parametrize("n_vis,k", [
+    ([520, 300, 257], 40),      # three / two / two row tiles: pairs with a full, a partial and an empty second tile
+    ([600, 513], 257),          # two groups of 144 slots, the second ragged (113 slots)
+    ([256, 300], 256),          # sample 0 drops nothing
+    ([129, 1000], 17),          # one group narrower than an MMA's smallest useful width
+])
+def test_pair_form_matches_the_oracle(ctx_pair_form, n_vis, k):
+    _merge_matches_oracle(ctx_pair_form, n_vis, k, H=2, seed=911)
 
 
 def test_pair_form_gives_up_and_the_context_recovers(ctx_pair_form):
