@@ -131,7 +131,15 @@ typedef struct {
 
 /* Creates a context on `device` and takes all scratch memory the step will ever need for
  * problems with total_tokens <= max_total_tokens, B <= max_B, H <= max_H, D <= max_D and
- * B * keep_k <= max_keep_rows (0 = max_total_tokens).  The only call that allocates. */
+ * B * keep_k <= max_keep_rows (0 = max_total_tokens).  The only call that allocates.
+ * Which kernel form a launch takes is decided from the problem size; four environment variables, read
+ * here once per context, move those decisions for measurements (results are the same up to rounding order):
+ *   ASAP_FUSE_MASS_MIN_TOKENS   B * max_vis from which Eq. 1's key side rides in the score kernel (default 50000)
+ *   ASAP_SIM_PAIR_MIN_BLOCKS    blocks from which the similarity takes two row tiles per block (default: half the SMs)
+ *   ASAP_SIM_PAIR_STAGES        tile stages of that form (default: what fits 192 KB)
+ *   ASAP_SIM_CLUSTER            0: sliced similarity launches add their partial products through global memory
+ *                               instead of a thread-block cluster's shared memory (default 1, if the device can
+ *                               place such a cluster) */
 asap_status asap_init(asap_ctx **ctx, int device, size_t max_total_tokens, int max_B, int max_H,
                       int max_D, size_t max_keep_rows);
 
