@@ -1002,18 +1002,23 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
       const int slot0 = (tile0 + nt) * a.n_tile;
       const int ncol = min(a.n_tile, a.keep_k - slot0);   // kept slots in this accumulator (none in a group's ragged end)
       int c0 = 0;
-      if (!a.smat && !part) {
+      if (!a.smat || part) {
         // 32 columns per tensor-memory wait while they last (see sim_pair_kernel)
 #pragma unroll 1
         for (; c0 + 32 <= ncol; c0 += 32) {
           uint32_t r[32];
           tmem_ld32(taddr + c0, r);
           tmem_wait_ld();
+          if (part) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const int slot = slot0 + c0 + e;
-            const float val = __uint_as_float(r[e]) * __ldg(kinv + slot);
-            if (val > best) { best = val; best_slot = slot; }
+            for (int e = 0; e < 32; ++e) part[(size_t)(slot0 + c0 + e) * 128 + lrow] = __uint_as_float(r[e]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const int slot = slot0 + c0 + e;
+              const float val = __uint_as_float(r[e]) * __ldg(kinv + slot);
+              if (val > best) { best = val; best_slot = slot; }
+            }
           }
         }
       }
