@@ -133,7 +133,7 @@ __device__ __forceinline__ RowPair score_row_pair(const SampleDesc &d, int rp, i
 __global__ void __launch_bounds__(SC_THREADS, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
              ScoreArgs a) {
-  pdl_enter();
+  // (the wait for the preceding kernel comes after the block's set-up, which reads nothing that kernel writes)
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_items = a.B * a.H;
@@ -182,6 +182,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   WaitCtx wc{&bk->abort_flag, a.status, STATUS_SCORE_TIMEOUT, a.wait_limit};
   if (*reinterpret_cast<volatile uint32_t *>(a.status) & STATUS_SCORE_TIMEOUT) bk->abort_flag = 1;   // benign race: same value
   __syncthreads();
+  pdl_enter();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer: items, queries, key tiles
@@ -726,7 +727,9 @@ template <bool GATHER>
 __global__ void __launch_bounds__(GATHER ? SIM_THREADS : SIM_THREADS_TILED, 1)
 sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_kept,
            SimArgs a) {
-  pdl_enter();
+  // (the wait for the preceding kernel comes after this block's set-up, which reads nothing that kernel
+  // writes: descriptors and status word are older; barriers, tensor memory and the cluster's first barrier
+  // are then ready when the kept rows are)
   extern __shared__ uint8_t smem_raw[];
   // the groups of a row tile are neighbours in launch order (blockIdx.x = row tile * groups + group)
   const int mt = blockIdx.x / a.groups, b = blockIdx.y;
@@ -752,6 +755,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   SimBook *bk = reinterpret_cast<SimBook *>(base_ptr + (size_t)a.stages * stage_bytes);
   if (n_rows <= 0) {
     // nothing was dropped in this sample: only the (empty) grouping has to be written
+    pdl_enter();
     if (z == 0 && gz == 0) csr_block(d, b, a.max_vis, a.keep_k, a.assign, a.seg, a.members, reinterpret_cast<int *>(base_ptr), bk->scan, a.drop_all, a.salience, a.member_meta);
     return;
   }
@@ -785,6 +789,7 @@ sim_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ C
   }
   __syncthreads();
   tc_fence_after();
+  pdl_enter();
   const uint32_t tmem_base = bk->tmem_base;
   WaitCtx wc{&bk->abort_flag, a.status, STATUS_SIM_TIMEOUT, a.wait_limit};
   // cluster form, in the tile ring once it is free: this slice's partial products [keep_k][128]; per quarter
@@ -1285,7 +1290,7 @@ static_assert(sizeof(SimPairBook) <= SIM_BOOK_BYTES, "pair kernel bookkeeping ex
 __global__ void __launch_bounds__(SIMP_THREADS, 1)
 sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_kept,
                 SimArgs a) {
-  pdl_enter();
+  // (the wait for the preceding kernel comes after the block's set-up, which reads nothing that kernel writes)
   extern __shared__ uint8_t smem_raw[];
   const int pr = blockIdx.x / a.groups, b = blockIdx.y;
   const int gz = blockIdx.x - pr * a.groups;             // group of kept slots
@@ -1325,6 +1330,7 @@ sim_pair_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
   }
   __syncthreads();
   tc_fence_after();
+  pdl_enter();
   const uint32_t tmem_base = bk->tmem_base;
   WaitCtx wc{&bk->abort_flag, a.status, STATUS_SIM_TIMEOUT, a.wait_limit};
   const int n_kb = a.D / 64;
